@@ -1,0 +1,166 @@
+/* mavg.h -- C ABI of the M-AVG engine (K-step model averaging with block momentum,
+ * Algorithm 1 of Cong & Liu, "Accelerate Distributed Stochastic Descent for Nonconvex
+ * Optimization with Momentum").
+ *
+ * All P learners are held on one GPU as a [P, stride] fp32 replica array.  One round n is
+ *   learner level (Algorithm 1, inner loop):  every learner j takes K minibatch-SGD steps
+ *       w^j <- w^j - (gamma / B) sum_s grad F(w^j; xi^j_{k,s}),  k = 1..K
+ *   meta level (Algorithm 1, last four assignments of the outer loop):
+ *       a = (1/P) sum_j w^j;  d = a - w~;  v <- mu v + zeta d;  w~ <- w~ + v
+ *   and the start of the next round (Algorithm 1, "set w^j_n = w~_n"):  w^j <- w~  for all j.
+ * zeta, the block learning rate, is an extension; zeta = 1 is the paper's update.  mu = 0 with
+ * zeta = 1 is K-AVG (Remark after Theorem 1).
+ *
+ * Conventions
+ *   - Every pointer is tagged DEVICE or HOST below.  Device buffers and the CUDA stream belong to
+ *     the caller and are borrowed from mavg_create until mavg_destroy; the library allocates no
+ *     device memory and frees none.  The handle is host memory owned by the library.
+ *   - All work is enqueued on the configured stream and returns without waiting, except where a
+ *     function hands a value back to HOST memory (then it waits for the stream).
+ *   - Errors are status codes; nothing throws, aborts or traps.  Arguments are checked on the
+ *     host before anything is launched.  A CUDA error is sticky: the call that meets it and every
+ *     later call return MAVG_ERR_CUDA.  mavg_last_error gives a message for the last failure.
+ *   - A handle is not thread-safe; distinct handles are independent.
+ *   - Counters: rounds n = 1, 2, ...; learners j = 0..P-1; local steps k = 1..K; batch slots
+ *     s = 0..B-1.
+ *
+ * Random numbers (the paper says only "randomly sample a mini-batch"): SplitMix64 used as a
+ * counter-based generator.  With mix64 the SplitMix64 output function and G = 0x9E3779B97F4A7C15,
+ * fold(s, c) = mix64(s + (c+1) G); the stream of (tag, n, j, k) has key
+ * fold(fold(fold(fold(seed, tag), n), j), k) and element i of it is fold(key, i).
+ *   tag 1, minibatch indices: learner j owns samples [floor(j S/P), floor((j+1) S/P)); slot s
+ *     draws  lo_j + floor(u * len_j / 2^32), u = top 32 bits of element s  (i.i.d. uniform with
+ *     replacement inside the learner's shard).
+ *   tag 2, synthetic gradients: element i is (sum of the four 16-bit lanes of the 64-bit value
+ *     - 131070) * c,  c = fp32(sigma / sqrt(4 (65536^2 - 1) / 12)): an Irwin-Hall(4) variate with
+ *     mean 0 and standard deviation sigma, the same bits on every IEEE machine.
+ */
+#ifndef MAVG_H_
+#define MAVG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mavg_ctx *mavg_handle;
+
+typedef enum {
+  MAVG_OK = 0,
+  MAVG_ERR_INVALID_ARG = 1, /* a scalar argument is out of its domain, or a required pointer is NULL */
+  MAVG_ERR_BAD_BUFFER = 2,  /* a buffer is NULL, misaligned or too small */
+  MAVG_ERR_STATE = 3,       /* call not valid for this handle (wrong objective, destroyed handle) */
+  MAVG_ERR_UNSUPPORTED = 4, /* shape outside what the kernels cover, or no sm_100 device */
+  MAVG_ERR_CUDA = 5,        /* a CUDA call or kernel failed; see mavg_last_error */
+  MAVG_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up; the context stays usable */
+} mavg_status;
+
+typedef enum {
+  MAVG_OBJ_NONE = 0,       /* no learner level: the caller writes the replicas (meta-update only) */
+  MAVG_OBJ_PSEUDOGRAD = 1, /* grad F(w; xi) replaced by seeded N(0, sigma^2)-like variates (tag 2) */
+  MAVG_OBJ_MLP = 2         /* MLP with bias, ReLU, softmax cross-entropy averaged over the batch */
+} mavg_objective;
+
+typedef enum { MAVG_X_F32 = 0, MAVG_X_BF16 = 1 } mavg_x_dtype;
+
+#define MAVG_MAX_LAYERS 8
+
+/* Problem statement: the five hyper-parameters the paper lists (P, B, K, step size, mu) plus the
+ * objective the learners descend.  Plain data, copied by mavg_create. */
+typedef struct {
+  int32_t P;         /* learners, >= 1 */
+  int32_t K;         /* local steps per round, >= 1 */
+  int32_t B;         /* minibatch per learner and step, >= 1 (ignored unless MLP) */
+  float local_lr;    /* gamma of Algorithm 1, finite */
+  float block_lr;    /* zeta, finite; 1 reproduces Algorithm 1 */
+  float mu;          /* block momentum, 0 <= mu < 1 (Theorem 1's domain) */
+  uint64_t seed;
+  int32_t objective; /* mavg_objective */
+  int64_t n;         /* parameters per replica, >= 1; for MLP must equal the layout's count */
+  /* MLP: layer l = 1..n_layers maps dims[l-1] -> dims[l]; flat layout per replica
+   * [W_1 (dims[1] x dims[0], row-major), b_1, W_2, b_2, ...]. */
+  int32_t n_layers;
+  int32_t dims[MAVG_MAX_LAYERS + 1];
+  int32_t gemm_bf16; /* 0: fp32 FMA arithmetic throughout.  1: every matrix-product operand
+                        (weights, activations, dZ) rounded to bf16 (nearest-even), fp32
+                        accumulation, fp32 master weights, bias, ReLU, softmax and SGD in fp32 */
+  float pseudo_grad_sigma; /* PSEUDOGRAD: standard deviation of the variates */
+  const void *x;     /* DEVICE [n_samples, dims[0]] row-major, fp32 or bf16 per x_dtype */
+  int32_t x_dtype;   /* mavg_x_dtype; bf16 requires gemm_bf16 */
+  const int32_t *y;  /* DEVICE [n_samples] labels in [0, dims[n_layers]) */
+  int64_t n_samples; /* S >= P, < 2^31 */
+  void *stream;      /* cudaStream_t (NULL = the legacy default stream) */
+} mavg_config;
+
+/* Caller-owned DEVICE buffers.  Every base pointer must be 16-byte aligned. */
+typedef struct {
+  float *replicas;        /* [P, replica_stride] fp32; row j is w^j */
+  int64_t replica_stride; /* floats between rows, >= n and a multiple of 4 */
+  float *global_w;        /* [n] w~; on entry to mavg_create it holds w~_1 */
+  float *momentum;        /* [n] v */
+  void *workspace;        /* scratch, at least mavg_workspace_bytes() bytes */
+  size_t workspace_bytes;
+} mavg_buffers;
+
+/* Bytes of scratch the configuration needs (activations, bf16 operand copies, batch indices,
+ * loss accumulators, the device status word).  Checks the configuration like mavg_create. */
+mavg_status mavg_workspace_bytes(const mavg_config *cfg, size_t *out_bytes);
+
+/* Algorithm 1, the two initialisation lines and the first "set w^j = w~": v <- 0, w^j <- w~_1.
+ * Validates everything; on failure *out is NULL.  Enqueues the initialisation on the stream. */
+mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_handle *out);
+
+/* Learner level of Algorithm 1 (inner loop over k): K SGD steps on all P replicas for the round
+ * that follows the last completed meta-update.  MAVG_ERR_STATE for MAVG_OBJ_NONE. */
+mavg_status mavg_local_steps(mavg_handle h);
+
+/* Meta level of Algorithm 1 (a, d, v, w~) fused with the re-broadcast w^j <- w~ that opens the
+ * next round; advances the round counter. */
+mavg_status mavg_meta_update(mavg_handle h);
+
+/* One round = mavg_local_steps then mavg_meta_update.  If mean_loss is not NULL (HOST, one
+ * float) the call waits for the stream and stores the mean of the round's P*K minibatch losses
+ * (0 for objectives without a loss). */
+mavg_status mavg_round(mavg_handle h, float *mean_loss);
+
+/* The same round for a caller whose model lives in HOST memory: copies w~ and v (n floats each,
+ * HOST, read and written) to the device, re-broadcasts w~ to the replicas, runs the round,
+ * copies w~ and v back and waits.  mean_loss as in mavg_round. */
+mavg_status mavg_round_host(mavg_handle h, float *w_host, float *v_host, float *mean_loss);
+
+/* Per-round schedules (Algorithm 1 lets gamma_n and B_n vary with n; B stays fixed here). */
+mavg_status mavg_set_hparams(mavg_handle h, int32_t K, float local_lr, float block_lr, float mu);
+
+/* Runs the device index generator for (round, learner, step) and copies the B indices to
+ * out (HOST, B int32); waits for the stream.  MLP objective only. */
+mavg_status mavg_get_batch_indices(mavg_handle h, int64_t round, int32_t learner, int32_t step,
+                                   int32_t *out);
+
+/* The P*K minibatch losses of the last mavg_local_steps, out[j*K + k-1] (HOST); waits. */
+mavg_status mavg_get_losses(mavg_handle h, float *out);
+
+/* Number of completed meta-updates (the next round is this + 1), and its setter for resuming
+ * from saved (w~, v, round): the caller restores global_w and momentum, then calls
+ * mavg_set_round, which re-broadcasts w~ to the replicas. */
+mavg_status mavg_get_round(mavg_handle h, int64_t *round);
+mavg_status mavg_set_round(mavg_handle h, int64_t round);
+
+/* Kernels launched by this handle so far. */
+mavg_status mavg_get_launch_count(mavg_handle h, int64_t *count);
+
+/* Waits for the stream; reports CUDA errors and a tripped device-side wait limit. */
+mavg_status mavg_sync(mavg_handle h);
+
+/* Message for the last failure on this handle ("" if none); with h == NULL, for the last failed
+ * mavg_create / mavg_workspace_bytes of the calling thread.  Valid until the next call. */
+const char *mavg_last_error(mavg_handle h);
+
+/* Releases the handle (host memory only).  NULL is a no-op. */
+mavg_status mavg_destroy(mavg_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAVG_H_ */

@@ -1,0 +1,148 @@
+// Minibatch side of the learner level: "randomly sample a mini-batch of size B_n"
+// (Algorithm 1) as a counter-based index stream, the gather of the sampled rows, and the softmax
+// cross-entropy loss with its gradient (the 1/B_n mean of Algorithm 1's update).
+#include "mlp.cuh"
+
+namespace mavg {
+namespace {
+
+// One thread per (learner, slot): idx = lo_j + floor(u * len_j / 2^32), u = top 32 bits of the
+// stream value (see mavg.h).  Also fetches the label.
+__global__ void k_batch_indices(int32_t* __restrict__ idx, int32_t* __restrict__ labels,
+                                const int32_t* __restrict__ y, uint64_t seed, int64_t round,
+                                int step, int P, int B, int64_t S, int j_first, int j_count) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= j_count * B) return;
+  int j = j_first + t / B, s = t % B;
+  int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
+  int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
+  uint64_t key = fold(learner_key(seed, kTagBatch, (uint64_t)round, (uint64_t)j), (uint64_t)step);
+  uint64_t u = fold(key, (uint64_t)s) >> 32;
+  int32_t i = (int32_t)(lo + (int64_t)((u * (uint64_t)(hi - lo)) >> 32));
+  idx[t] = i;
+  if (labels) labels[t] = y[i];
+}
+
+template <typename TIN>
+__device__ __forceinline__ float to_f32(TIN v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Row gather.  One block per sampled row.  Outputs (any may be null):
+//   out_f32 [rows, d]  fp32 (rounded to bf16 values when quant)
+//   out_bf  [rows, d]  bf16
+//   out_bft [P, d, B]  bf16, the same rows transposed per learner
+template <typename TIN>
+__global__ void __launch_bounds__(256)
+k_gather(const TIN* __restrict__ x, const int32_t* __restrict__ idx, int d, int B, int quant,
+         float* __restrict__ out_f32, __nv_bfloat16* __restrict__ out_bf,
+         __nv_bfloat16* __restrict__ out_bft) {
+  const int row = blockIdx.x;
+  const TIN* src = x + (size_t)idx[row] * d;
+  const int p = row / B, s = row % B;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = to_f32<TIN>(src[i]);
+    __nv_bfloat16 b = __float2bfloat16_rn(v);
+    if (out_f32) out_f32[(size_t)row * d + i] = quant ? __bfloat162float(b) : v;
+    if (out_bf) out_bf[(size_t)row * d + i] = b;
+    if (out_bft) out_bft[((size_t)p * d + i) * B + s] = b;
+  }
+}
+
+// Softmax cross-entropy of learner blockIdx.x's B rows.  logits [P*B, ldz] fp32.
+//   loss_out[p*loss_stride] = (1/B) sum_b (logsumexp(z_b) - z_b[y_b])
+//   dz_f32 [P*B, ld32]  (softmax - onehot)/B
+//   dz_bf  [P*B, ldbf], dz_bft [P, C rows of ldbft] bf16 copies   (may be null)
+//   rep    if not null, the last layer's bias of learner p takes its SGD step here:
+//          b[c] -= gamma * sum_b dz[b,c]  (ascending b, from the unrounded dz)
+__global__ void __launch_bounds__(256)
+k_softmax_ce(const float* __restrict__ logits, int ldz, const int32_t* __restrict__ labels, int B,
+             int C, float* __restrict__ loss_out, int loss_stride, float* __restrict__ dz_f32,
+             int ld32, __nv_bfloat16* __restrict__ dz_bf, int ldbf,
+             __nv_bfloat16* __restrict__ dz_bft, int ldbft, float* __restrict__ rep,
+             int64_t rep_stride, int64_t bias_off, float gamma) {
+  extern __shared__ float part[];     // [blockDim.x] loss partials
+  const int p = blockIdx.x;
+  const float inv_b = 1.0f / (float)B;
+  float my_loss = 0.f;
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    const size_t row = (size_t)p * B + b;
+    const float* z = logits + row * ldz;
+    float m = z[0];
+    for (int c = 1; c < C; ++c) m = fmaxf(m, z[c]);
+    float se = 0.f;
+    for (int c = 0; c < C; ++c) se += expf(z[c] - m);
+    const float lse = m + logf(se);
+    const int yb = labels[row];
+    my_loss += lse - z[yb];
+    for (int c = 0; c < C; ++c) {
+      float g = (expf(z[c] - lse) - (c == yb ? 1.f : 0.f)) * inv_b;
+      dz_f32[row * ld32 + c] = g;
+      __nv_bfloat16 gq = __float2bfloat16_rn(g);
+      if (dz_bf) dz_bf[row * ldbf + c] = gq;
+      if (dz_bft) dz_bft[((size_t)p * C + c) * ldbft + b] = gq;
+    }
+  }
+  part[threadIdx.x] = my_loss;
+  __syncthreads();   // also makes this block's dz_f32 stores visible to its own threads
+  // fixed-order sums by one thread per output: B and C are small
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+    for (int t = 0; t < (int)blockDim.x; ++t) s += part[t];
+    loss_out[(size_t)p * loss_stride] = s * inv_b;
+  }
+  if (rep) {
+    float* bias = rep + (size_t)p * rep_stride + bias_off;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+      float s = 0.f;
+      for (int b = 0; b < B; ++b) s += dz_f32[((size_t)p * B + b) * ld32 + c];
+      bias[c] = fmaf(-gamma, s, bias[c]);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_first, int j_count,
+                                 int32_t* idx, int32_t* labels) {
+  const int total = j_count * c->cfg.B;
+  k_batch_indices<<<(total + 255) / 256, 256, 0, c->stream>>>(
+      idx, labels, c->cfg.y, c->cfg.seed, round, step, c->cfg.P, c->cfg.B, c->cfg.n_samples,
+      j_first, j_count);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather(mavg_ctx* c, const int32_t* idx, int quant, float* out_f32,
+                          __nv_bfloat16* out_bf, __nv_bfloat16* out_bft) {
+  const int rows = c->cfg.P * c->cfg.B, d = c->cfg.dims[0];
+  if (c->cfg.x_dtype == MAVG_X_BF16)
+    k_gather<__nv_bfloat16><<<rows, 256, 0, c->stream>>>((const __nv_bfloat16*)c->cfg.x, idx, d,
+                                                         c->cfg.B, quant, out_f32, out_bf, out_bft);
+  else
+    k_gather<float><<<rows, 256, 0, c->stream>>>((const float*)c->cfg.x, idx, d, c->cfg.B, quant,
+                                                 out_f32, out_bf, out_bft);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const int32_t* labels,
+                              float* loss_out, int loss_stride, float* dz_f32, int ld32,
+                              __nv_bfloat16* dz_bf, int ldbf, __nv_bfloat16* dz_bft, int ldbft,
+                              bool update_bias) {
+  const int P = c->cfg.P, B = c->cfg.B, C = c->cfg.dims[c->cfg.n_layers];
+  int threads = 32;
+  while (threads < B && threads < 256) threads <<= 1;
+  size_t smem = (size_t)threads * sizeof(float);
+  const MlpLayer& last = c->layers.back();
+  k_softmax_ce<<<P, threads, smem, c->stream>>>(
+      logits, ldz, labels, B, C, loss_out, loss_stride, dz_f32, ld32, dz_bf, ldbf, dz_bft, ldbft,
+      update_bias ? c->buf.replicas : nullptr, c->buf.replica_stride, last.b_off,
+      c->cfg.local_lr);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+}  // namespace mavg

@@ -1,0 +1,91 @@
+// Shared declarations of the M-AVG CUDA library: the context behind a handle, the workspace
+// carve-up, the counter-based generator (device and host) and the launch entry points of each
+// kernel file.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/mavg.h"
+
+namespace mavg {
+
+// ------------------------------------------------------------------ SplitMix64 as a counter RNG
+// fold(s, c) = mix64(s + (c+1) G): the (c+1)-th SplitMix64 output from state s.
+constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
+constexpr uint64_t kTagBatch = 1, kTagPseudoGrad = 2;
+
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+__host__ __device__ __forceinline__ uint64_t fold(uint64_t s, uint64_t c) {
+  return mix64(s + (c + 1) * kGamma);
+}
+// key of the stream (tag, round n, learner j); one more fold with the step k completes it
+__host__ __device__ __forceinline__ uint64_t learner_key(uint64_t seed, uint64_t tag, uint64_t n,
+                                                         uint64_t j) {
+  return fold(fold(fold(seed, tag), n), j);
+}
+
+// ------------------------------------------------------------------------------------- context
+struct MlpLayer {
+  int in, out;
+  int64_t w_off, b_off;      // offsets (floats) inside a replica
+  int64_t sh_off, sht_off;   // offsets (bf16 elements) inside a shadow row / transposed shadow row
+  int out_pad;               // row length of the transposed shadow [in, out_pad]
+};
+
+struct Workspace {           // byte offsets into the caller's scratch buffer
+  size_t status = 0;         // int32[64]: [0] device wait-limit flag
+  size_t losses = 0;         // float [P*K]
+  size_t loss_mean = 0;      // float [1]
+  size_t idx = 0;            // int32 [P*B] sample indices of the current step
+  size_t labels = 0;         // int32 [P*B]
+  size_t act = 0;            // activations and their gradients (see mlp files)
+  size_t total = 0;
+};
+
+}  // namespace mavg
+
+struct mavg_ctx {
+  mavg_config cfg;
+  mavg_buffers buf;
+  cudaStream_t stream = nullptr;
+  int64_t round = 0;          // completed meta-updates
+  int64_t launches = 0;
+  mavg_status sticky = MAVG_OK;
+  std::string err;
+  int sm_count = 148;
+  size_t l2_bytes = 0;
+  bool replicas_equal_global = true;  // true between a (re-)broadcast and the next local step
+  mavg::Workspace ws;
+  std::vector<mavg::MlpLayer> layers;
+  void* mlp = nullptr;        // state of the MLP path (owned by mlp files)
+};
+
+namespace mavg {
+
+// Every launcher enqueues on ctx->stream, adds to ctx->launches and returns the CUDA status of
+// the launch (cudaGetLastError), nothing else.
+cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v);
+cudaError_t launch_meta_update(mavg_ctx* c);
+cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round);
+
+// MLP path (mlp_*.cu)
+mavg_status mlp_validate(const mavg_config* cfg, std::string* why);
+size_t mlp_workspace_bytes(const mavg_config* cfg, Workspace* ws, size_t base);
+mavg_status mlp_setup(mavg_ctx* c);
+void mlp_teardown(mavg_ctx* c);
+cudaError_t mlp_refresh_shared_operands(mavg_ctx* c);   // after w~ changed
+cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round);
+cudaError_t mlp_indices_only(mavg_ctx* c, int64_t round, int learner, int step, int32_t* dev_out);
+
+inline char* ws_ptr(mavg_ctx* c, size_t off) { return (char*)c->buf.workspace + off; }
+
+}  // namespace mavg

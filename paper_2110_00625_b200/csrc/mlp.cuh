@@ -1,0 +1,32 @@
+// Declarations shared by the files of the MLP learner level (batch.cu, mlp.cu, mlp_simt.cu,
+// mlp_tc.cu).
+#pragma once
+#include "common.cuh"
+
+namespace mavg {
+
+// batch.cu
+cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_first, int j_count,
+                                 int32_t* idx, int32_t* labels);
+cudaError_t launch_gather(mavg_ctx* c, const int32_t* idx, int quant, float* out_f32,
+                          __nv_bfloat16* out_bf, __nv_bfloat16* out_bft);
+cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const int32_t* labels,
+                              float* loss_out, int loss_stride, float* dz_f32, int ld32,
+                              __nv_bfloat16* dz_bf, int ldbf, __nv_bfloat16* dz_bft, int ldbft,
+                              bool update_bias);
+
+// CUDA-core path (mlp_simt.cu): fp32 arithmetic, or bf16-rounded operands with fp32 FMAs.
+size_t simt_workspace_bytes(const mavg_config* cfg, size_t base, size_t* act_off);
+cudaError_t simt_step(mavg_ctx* c, int64_t round, int step);
+
+// Tensor-core path (mlp_tc.cu): tcgen05 GEMMs fed by TMA.
+bool tc_shapes_ok(const mavg_config* cfg, std::string* why);
+size_t tc_workspace_bytes(const mavg_config* cfg, size_t base, size_t* act_off);
+mavg_status tc_setup(mavg_ctx* c);
+void tc_teardown(mavg_ctx* c);
+cudaError_t tc_refresh_shared_operands(mavg_ctx* c);
+cudaError_t tc_step(mavg_ctx* c, int64_t round, int step);
+
+inline bool use_tensor_cores(const mavg_config* cfg) { return cfg->gemm_bf16 == 1; }
+
+}  // namespace mavg

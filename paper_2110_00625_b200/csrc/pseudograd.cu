@@ -1,0 +1,77 @@
+// Learner level of Algorithm 1 with the stochastic gradient replaced by seeded variates:
+//   w^j <- w^j - gamma g(seed, n, j, k, i),  k = 1..K,
+// g an Irwin-Hall(4) variate of standard deviation sigma built from one SplitMix64 stream value
+// (see mavg.h).  The K steps are applied in order to a value held in registers, so one pass over
+// the replicas (8 bytes per element and learner) serves the whole round; the per-step rounding is
+// the same as K separate passes.
+#include "common.cuh"
+
+namespace mavg {
+namespace {
+
+__device__ __forceinline__ float ih4(uint64_t h, float c) {
+  uint32_t lo = (uint32_t)h, hi = (uint32_t)(h >> 32);
+  int32_t s = (int32_t)((lo & 0xFFFFu) + (lo >> 16) + (hi & 0xFFFFu) + (hi >> 16));
+  return (float)(s - 131070) * c;
+}
+
+// grid = (x, P); dynamic shared memory holds the K step keys of learner blockIdx.y.
+__global__ void __launch_bounds__(256)
+k_pseudograd_steps(float* __restrict__ rep, int64_t stride, int64_t n, int K, uint64_t seed,
+                   int64_t round, int k_first, float c, float gamma) {
+  extern __shared__ uint64_t keys[];
+  const int j = blockIdx.y;
+  const uint64_t lk = learner_key(seed, kTagPseudoGrad, (uint64_t)round, (uint64_t)j);
+  for (int k = threadIdx.x; k < K; k += blockDim.x) keys[k] = fold(lk, (uint64_t)(k_first + k));
+  __syncthreads();
+  float* row = rep + (size_t)j * stride;
+  float4* row4 = reinterpret_cast<float4*>(row);
+  const int64_t n4 = n >> 2;
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  const float ng = -gamma;
+  for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += step) {
+    float4 w = __ldcs(row4 + q);
+    const uint64_t c0 = (uint64_t)(4 * q + 1) * kGamma;  // element i uses (i+1) G
+    for (int k = 0; k < K; ++k) {
+      const uint64_t key = keys[k];
+      w.x = fmaf(ng, ih4(mix64(key + c0), c), w.x);
+      w.y = fmaf(ng, ih4(mix64(key + c0 + kGamma), c), w.y);
+      w.z = fmaf(ng, ih4(mix64(key + c0 + 2 * kGamma), c), w.z);
+      w.w = fmaf(ng, ih4(mix64(key + c0 + 3 * kGamma), c), w.w);
+    }
+    __stcs(row4 + q, w);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {
+    const int64_t i = (n4 << 2) + threadIdx.x;
+    float w = row[i];
+    for (int k = 0; k < K; ++k) w = fmaf(ng, ih4(fold(keys[k], (uint64_t)i), c), w);
+    row[i] = w;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round) {
+  const int64_t n = c->cfg.n;
+  const int P = c->cfg.P, K = c->cfg.K;
+  const double var_lane = (65536.0 * 65536.0 - 1.0) / 12.0;
+  const float scale = (float)((double)c->cfg.pseudo_grad_sigma / sqrt(4.0 * var_lane));
+  constexpr int kMaxFused = 2048;  // step keys per launch (16 KB of shared memory)
+  int64_t blocks_x = ((n >> 2) + 255) / 256;
+  int64_t cap = ((int64_t)c->sm_count * 8 + P - 1) / P;
+  if (blocks_x > cap) blocks_x = cap;
+  if (blocks_x < 1) blocks_x = 1;
+  for (int k0 = 0; k0 < K; k0 += kMaxFused) {
+    int kc = K - k0 < kMaxFused ? K - k0 : kMaxFused;
+    dim3 grid((unsigned)blocks_x, (unsigned)P);
+    k_pseudograd_steps<<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
+        c->buf.replicas, c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
+        c->cfg.local_lr);
+    c->launches++;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace mavg

@@ -1,0 +1,140 @@
+"""GPU parity of the MLP learner level and of whole rounds against the CPU oracle, through the
+C ABI.  Gates: index streams bit-exact; fp32 model: per-round loss within 1e-4 relative (plus
+1e-6 absolute: logits of magnitude ~20 carry ~2e-6 of fp32 rounding, which is all that is left of
+a loss that has fallen to 1e-4) and parameters within 1e-3; bf16-operand model: loss within 2e-2
+relative, parameters within 5e-2."""
+import numpy as np
+import pytest
+import torch
+
+from tests.util import rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _mavg():
+    import paper_2110_00625_b200 as m
+    return m
+
+
+def _pair(oracle, cfg, S=None, rounds=None, gemm_bf16=None, x_bf16=False, seed=0x211000625, **over):
+    m = _mavg()
+    c = dict(cfg)
+    c.update(over)
+    x, y = m.workloads.make_dataset(c, S=S or c["S"])
+    w1 = m.workloads.mlp_init(c["dims"])
+    mode = gemm_bf16 if gemm_bf16 is not None else (1 if c["bf16"] else 0)
+    g = m.Mavg(w1, P=c["P"], K=c["K"], local_lr=c["gamma"], mu=c["mu"], block_lr=c["zeta"],
+               B=c["B"], seed=seed, objective=m.OBJ_MLP, dims=c["dims"], gemm_bf16=mode, x=x, y=y,
+               x_bf16=x_bf16)
+    o = oracle.Mavg(w1, P=c["P"], K=c["K"], gamma=c["gamma"], mu=c["mu"], zeta=c["zeta"],
+                    B=c["B"], seed=seed, objective=oracle.OBJ_MLP, dims=c["dims"],
+                    bf16=bool(c["bf16"]), x=x, y=y, stride=g.stride)
+    return g, o, c
+
+
+def test_batch_indices_bit_exact(oracle):
+    m = _mavg()
+    for name in ("C1", "C2", "C4"):
+        cfg = dict(m.workloads.CONFIGS[name])
+        cfg["dims"] = [32, 16, 10]     # the index stream does not depend on the model
+        cfg["bf16"] = False
+        cfg["data"] = "gaussian_mixture"
+        g, o, c = _pair(oracle, cfg)
+        for (n, j, k) in [(1, 0, 1), (3, c["P"] - 1, c["K"]), (2, c["P"] // 2, 2)]:
+            got = g.get_batch_indices(n, j, k)
+            want = oracle.batch_indices(0x211000625, n, c["P"], j, k, c["S"], c["B"])
+            assert np.array_equal(got, want)
+        g.close()
+
+
+def test_c1_fp32_full_trajectory(oracle):
+    m = _mavg()
+    g, o, c = _pair(oracle, m.workloads.CONFIGS["C1"])
+    for r in range(c["rounds"]):
+        lg = g.round(want_loss=True)
+        lo, _ = o.run_round()
+        assert abs(lg - lo) <= 1e-4 * abs(lo) + 1e-6, (r, lg, lo)
+        assert rel_err(g.w.cpu().numpy(), o.w) <= 1e-3, r
+        assert rel_err(g.v.cpu().numpy(), o.v) <= 1e-3, r
+    g.sync()
+
+
+def test_c1_first_local_steps_per_learner(oracle):
+    # replicas after the K local steps of round 1, learner by learner, and every minibatch loss
+    m = _mavg()
+    g, o, c = _pair(oracle, m.workloads.CONFIGS["C1"])
+    g.local_steps()
+    losses_o, _ = o.local_steps()
+    g.sync()
+    gr = g.replicas.cpu().numpy()
+    for j in range(c["P"]):
+        assert rel_err(gr[j, :g.n], o.replicas[j, :g.n]) <= 1e-4
+    assert np.abs(g.get_losses() - losses_o).max() <= 1e-4 * losses_o.max()
+
+
+@pytest.mark.parametrize("dims,B,P,K", [([40, 24, 10], 7, 3, 2), ([33, 70, 65, 5], 20, 2, 3),
+                                        ([16, 3], 1, 1, 1)])
+def test_fp32_odd_shapes(oracle, dims, B, P, K):
+    m = _mavg()
+    cfg = dict(kind="mlp", dims=dims, bf16=False, P=P, K=K, B=B, gamma=0.05, mu=0.9, zeta=1.0,
+               rounds=3, S=512, data="gaussian_mixture")
+    g, o, c = _pair(oracle, cfg)
+    for r in range(3):
+        lg = g.round(want_loss=True)
+        lo, _ = o.run_round()
+        assert abs(lg - lo) <= 1e-4 * abs(lo) + 1e-6
+        assert rel_err(g.w.cpu().numpy(), o.w) <= 1e-3
+
+
+def test_p1_k1_mu0_is_plain_sgd_on_gpu(oracle):
+    m = _mavg()
+    cfg = dict(kind="mlp", dims=[32, 64, 10], bf16=False, P=1, K=1, B=32, gamma=0.05, mu=0.0,
+               zeta=1.0, rounds=3, S=256, data="gaussian_mixture")
+    g, o, c = _pair(oracle, cfg)
+    x, y = m.workloads.make_dataset(c, S=256)
+    w = o.w.copy()
+    for r in range(1, 4):
+        idx = oracle.batch_indices(0x211000625, r, 1, 0, 1, 256, 32)
+        _, grad = oracle.mlp_loss_grad(c["dims"], w, x[idx], y[idx])
+        w = (w.astype(np.float64) - np.float64(np.float32(0.05)) * grad).astype(np.float32)
+        g.round()
+    g.sync()
+    assert rel_err(g.w.cpu().numpy(), w) <= 1e-4
+
+
+@pytest.mark.parametrize("mode", [2, 1])
+def test_bf16_small_cifar_shaped(oracle, mode):
+    # CIFAR-shaped workload with narrower layers: several tiles per GEMM, bf16 operands.
+    # mode 2 = CUDA-core arithmetic, mode 1 = tensor cores.
+    m = _mavg()
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(dims=[3072, 256, 128, 10], P=4, K=4, B=64, S=2048, rounds=3)
+    g, o, c = _pair(oracle, cfg, gemm_bf16=mode)
+    for r in range(3):
+        lg = g.round(want_loss=True)
+        lo, _ = o.run_round()
+        assert abs(lg - lo) <= 2e-2 * abs(lo), (r, lg, lo)
+        assert rel_err(g.w.cpu().numpy(), o.w) <= 5e-2, r
+        assert rel_err(g.v.cpu().numpy(), o.v) <= 5e-2, r
+    g.sync()
+
+
+def test_bf16_teacher_forced_step(oracle):
+    # one local step from identical replicas, learner by learner: kernel error without drift
+    m = _mavg()
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(dims=[3072, 256, 128, 10], P=3, K=1, B=128, S=2048)
+    for mode in (2, 1):
+        g, o, c = _pair(oracle, cfg, gemm_bf16=mode)
+        g.local_steps()
+        losses_o, _ = o.local_steps()
+        g.sync()
+        gr = g.replicas.cpu().numpy()
+        for j in range(c["P"]):
+            # compare the step taken, w_after - w_before, which is -gamma * grad
+            step_g = gr[j, :g.n].astype(np.float64) - o.w
+            step_o = o.replicas[j, :g.n].astype(np.float64) - o.w
+            assert rel_err(step_g, step_o) <= 2e-2
+        assert np.abs(g.get_losses() - losses_o).max() <= 2e-3 * losses_o.max()
+        g.close()

@@ -1,0 +1,397 @@
+"""Benchmark of the M-AVG round (Algorithm 1) on one B200 per rank.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mavg|reference]
+
+A step is one full round -- K_local SGD steps on all P learners, then the fused meta-update --
+of the CIFAR-shaped MLP workload (3072-512-512-10, bf16 GEMM operands, fp32 masters, P=8,
+K_local=8, B=128) on seeded synthetic data.  Prints ONE JSON line (rank 0).  With --gpus N > 1
+every rank runs an independent replica of the same workload on its own GPU (the method is
+simulated on one GPU; there is no exchange between GPUs), and `value` is the sum over ranks.
+
+--impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same
+workload; it is a deliberately plain program and only a baseline.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "learner-samples/sec per MAVG round; meta-update HBM GB/s vs peak (1 B200)"
+UNIT = "learner-samples/s"
+WORKLOAD = "C2"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-i", str(self.gpu), "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            t = [s.strip() for s in line.split(",")]
+            if len(t) < 9:
+                continue
+            try:
+                sm.append(float(t[1]))
+                mx.append(float(t[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, t[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        return out
+
+
+def workload_inputs():
+    from paper_2110_00625_b200 import workloads as W
+    cfg = dict(W.CONFIGS[WORKLOAD])
+    x, y = W.make_dataset(cfg)
+    w1 = W.mlp_init(cfg["dims"])
+    return cfg, x, y, w1
+
+
+def flop_per_sample(dims):
+    # forward + weight gradient for every layer, data gradient for all but the first
+    macs = sum(dims[l] * dims[l + 1] for l in range(len(dims) - 1))
+    return 6 * macs - 2 * dims[0] * dims[1]
+
+
+def cpu_oracle_rate(cfg, x, y, w1, k_sample, reps=1):
+    """learner-samples/s of the oracle on a round cut down to k_sample local steps."""
+    from oracle import oracle as O
+    threads = min(cfg["P"], O.max_threads())
+    o = O.Mavg(w1, P=cfg["P"], K=k_sample, gamma=cfg["gamma"], mu=cfg["mu"], zeta=cfg["zeta"],
+               B=cfg["B"], seed=0x211000625, objective=O.OBJ_MLP, dims=cfg["dims"],
+               bf16=bool(cfg["bf16"]), x=x, y=y, threads=threads)
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        o.run_round()
+        times.append(time.perf_counter() - t0)
+    units = cfg["P"] * k_sample * cfg["B"]
+    return units / statistics.median(times), threads, times
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg, x, y, w1 = workload_inputs()
+    k_sample = 1
+    total = args.warmup + args.steps
+    rate, threads, times = cpu_oracle_rate(cfg, x, y, w1, k_sample, reps=total)
+    timed = times[args.warmup:]
+    units = cfg["P"] * k_sample * cfg["B"]
+    value = units * len(timed) / sum(timed)
+    sample = (f"each step = 1 of the {cfg['K']} local steps on all {cfg['P']} learners "
+              f"(B={cfg['B']}) + the meta-update = {units} learner-samples")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(timed) / len(timed),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "C2 CIFAR-shaped MLP 3072-512-512-10, P=8, K=8, B=128, mu=0.9 "
+                               "(bounded sample per step)", "global_batch": cfg["P"] * cfg["B"]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def kernel_rooflines(cfg, prof, steps, peaks, tensor_path):
+    """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
+    dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
+    L = len(dims) - 1
+    nW = [dims[l] * dims[l + 1] for l in range(L)]
+    n = sum(nW) + sum(dims[1:])
+    rows = P * B
+    out = {}
+    per_round = {
+        # replicas, w~, v read; v, w~, replicas written
+        "meta_update": dict(bytes=(8 * P + 16) * n, flops=0),
+        # bf16 weights read once per learner and step; activations in and out
+        "fwd_gemm": dict(bytes=K * (2 * P * sum(nW) + 2 * rows * (sum(dims[:-1]) + 2 * sum(dims[1:]))),
+                         flops=K * 2 * rows * sum(nW)),
+        "dgrad_gemm": dict(bytes=K * (2 * P * sum(nW[1:]) + 2 * rows * (sum(dims[2:]) + 3 * sum(dims[1:-1]))),
+                           flops=K * 2 * rows * sum(nW[1:])),
+        # fp32 master read + written, bf16 copy written (row- and column-major for layers >= 2)
+        "wgrad_sgd_gemm": dict(bytes=K * (P * (10 * sum(nW) + 2 * sum(nW[1:])) + 2 * rows * sum(dims)),
+                               flops=K * 2 * rows * sum(nW)),
+    }
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0 or ms <= 0:
+            continue
+        e = dict(ms_total=ms, launches=cnt, ms_per_launch=ms / cnt)
+        if name in per_round:
+            w = per_round[name]
+            sec = ms * 1e-3
+            e["gbs"] = w["bytes"] * steps / sec / 1e9
+            e["frac_hbm"] = e["gbs"] / peaks["hbm_gbs"]
+            if w["flops"]:
+                e["tflops"] = w["flops"] * steps / sec / 1e12
+                e["frac_tensor"] = e["tflops"] / peaks["bf16_tflops_sustained"]
+            e["bytes_per_launch"] = w["bytes"] * steps / cnt
+        out[name] = e
+    return out
+
+
+def meta_update_sweep(m, torch, peaks, reps=5):
+    """Meta-update alone at the ResNet-18-sized sweep: n = 11.2 M, P in {4, 16, 64}, mu in {0, 0.9}."""
+    n = 11_200_000
+    res = []
+    w1 = (0.05 * torch.randn(n, generator=torch.Generator().manual_seed(1))).numpy()
+    for P in (4, 16, 64):
+        for mu in (0.0, 0.9):
+            g = m.Mavg(w1, P=P, K=1, local_lr=0.1, mu=mu, objective=m.OBJ_NONE)
+            gen = torch.Generator(device=g.device).manual_seed(P)
+            times = []
+            for u in range(3 + reps):
+                # replicas ~ N(0, 0.01) around the current global model (untimed)
+                g.replicas[:, :n] = g.w[None, :] + 0.1 * torch.randn((P, n), device=g.device,
+                                                                     generator=gen)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                g.meta_update()
+                b.record()
+                b.synchronize()
+                if u >= 3:
+                    times.append(a.elapsed_time(b))
+            g.sync()
+            by = ((8 * P + 16) - (4 if mu == 0.0 else 0)) * n
+            ms = statistics.median(times)
+            res.append(dict(P=P, mu=mu, n=n, ms=ms, gbs=by / ms / 1e6,
+                            frac_measured=by / ms / 1e6 / peaks["hbm_gbs"],
+                            frac_nominal_8tbs=by / ms / 1e6 / 8000.0))
+            g.close()
+            del g
+            torch.cuda.empty_cache()
+    return res
+
+
+def run_mavg(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2110_00625_b200 as m
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+    cfg, x, y, w1 = workload_inputs()
+
+    # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        k_sample = 4
+        rate, threads, times = cpu_oracle_rate(cfg, x, y, w1, k_sample)
+        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"one round cut to {k_sample} of {cfg['K']} local steps on all "
+                         f"{cfg['P']} learners + meta-update ({cfg['P'] * k_sample * cfg['B']} "
+                         f"learner-samples, {times[0]:.1f} s)"}
+
+    mode = args.gemm
+    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"],
+               block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
+               dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}")
+    units = cfg["P"] * cfg["K"] * cfg["B"]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        g.round()
+    g.sync()
+
+    # ---- timed region: device-resident inputs -------------------------------------------------
+    sampler = ClockSampler(local)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+           torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    l0 = g.launch_count()
+    barrier()
+    sampler.start()
+    t_wall0 = time.perf_counter()
+    for a, mid, b in ev:
+        flush.zero_()                      # L2 flush, outside the step's event pair
+        a.record()
+        g.local_steps()
+        mid.record()
+        g.meta_update()
+        b.record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    launches = g.launch_count() - l0
+    step_ms = [a.elapsed_time(b) for a, _, b in ev]
+    meta_ms = [mid.elapsed_time(b) for _, mid, b in ev]
+    total_ms = sum(step_ms)
+    g.sync()
+
+    # ---- end to end: model in host memory, copies inside the timed region ----------------------
+    wh = torch.from_numpy(w1.copy()).pin_memory()
+    vh = torch.zeros(g.n).pin_memory()
+    for _ in range(2):
+        g.round_host(wh, vh)
+    barrier()
+    t0 = time.perf_counter()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        g.round_host(wh, vh)
+    b.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b)
+
+    # ---- per-kernel device times: the same steps again with an event pair around every launch ---
+    g.set_profiling(True)
+    g.get_profile(reset=True)
+    for _ in range(args.steps):
+        flush.zero_()
+        g.round()
+    prof = g.get_profile(reset=True)
+    g.set_profiling(False)
+    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1)
+
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=g.device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = t.tolist()
+
+    line = None
+    if rank == 0:
+        # the roofline object describes the class that takes the most device time in a round
+        timed = {k: v for k, v in kern.items() if "gbs" in v}
+        dom = max(timed, key=lambda k: timed[k]["ms_total"]) if timed else None
+        roof = None
+        if dom:
+            e = timed[dom]
+            hbm_time = e["bytes_per_launch"] / (peaks["hbm_gbs"] * 1e9)
+            tensor_time = (e.get("tflops", 0) and
+                           e["tflops"] * 1e12 * e["ms_per_launch"] * 1e-3 /
+                           (peaks["bf16_tflops_sustained"] * 1e12))
+            if tensor_time and tensor_time > hbm_time:
+                roof = {"bound": "tensor", "achieved": e["tflops"],
+                        "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                        "frac": e["frac_tensor"], "traffic": None}
+            else:
+                roof = {"bound": "hbm", "achieved": e["gbs"], "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": e["frac_hbm"], "traffic": None}
+            roof["kernel"] = dom
+            roof["peak_source"] = peaks["source"]
+        sweep = meta_update_sweep(m, torch, peaks) if world == 1 and not args.no_sweep else None
+        n = g.n
+        line = {
+            "metric": METRIC, "value": world * units * args.steps / (total_ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if mode else "f32", "data": "synthetic",
+            "config": {"workload": "C2 CIFAR-shaped MLP 3072-512-512-10, P=8, K=8, B=128, mu=0.9, "
+                                   "gamma=0.05, 50000 synthetic samples, labels from a random teacher",
+                       "global_batch": cfg["P"] * cfg["B"], "parallelism": "replicas only",
+                       "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
+                                0: "CUDA cores fp32"}[mode],
+                       "l2": "flushed between steps by a 256 MiB memset outside the step's events",
+                       "kernel_timing": "second pass over the same steps with one event pair per launch"},
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
+                       "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "e2e": {"value": world * units * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": 8 * n, "d2h_bytes_per_step": 8 * n + 4},
+            "gpu_launches": launches,
+            "roofline": roof,
+            "cpu_baseline": cpu,
+            "wall_s_timed_region": t_wall,
+            "meta_update_in_round": {"ms": statistics.median(meta_ms),
+                                     "gbs": (8 * cfg["P"] + 16) * n / statistics.median(meta_ms) / 1e6},
+            "kernels": kern,
+            "meta_update_sweep": sweep,
+            "tflops_round": flop_per_sample(cfg["dims"]) * units * args.steps / (total_ms * 1e-3) / 1e12,
+        }
+        print(json.dumps(line))
+    g.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mavg", choices=["mavg", "reference"])
+    ap.add_argument("--gemm", type=int, default=1, choices=[1, 2],
+                    help="1: tensor cores (default); 2: CUDA cores with bf16-rounded operands")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "mavg":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_mavg(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

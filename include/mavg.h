@@ -150,6 +150,25 @@ mavg_status mavg_set_round(mavg_handle h, int64_t round);
 /* Kernels launched by this handle so far. */
 mavg_status mavg_get_launch_count(mavg_handle h, int64_t *count);
 
+/* Measurement aid (the paper has no counterpart).  While profiling is on, every kernel launch of
+ * this handle is bracketed by a pair of CUDA events on the stream.  mavg_get_profile waits for the
+ * stream and returns, per kernel class, the summed device time in milliseconds and the number of
+ * launches since the last reset (ms and launches: HOST arrays of MAVG_K_COUNT entries). */
+typedef enum {
+  MAVG_K_META = 0,      /* fused meta-update + re-broadcast */
+  MAVG_K_BROADCAST = 1, /* initial / resume broadcast */
+  MAVG_K_PSEUDOGRAD = 2,
+  MAVG_K_BATCH = 3,     /* index stream and gather */
+  MAVG_K_FWD = 4,       /* forward GEMMs (+bias, ReLU) */
+  MAVG_K_LOSS = 5,      /* softmax cross-entropy, loss reductions */
+  MAVG_K_DGRAD = 6,     /* backward-data GEMMs (+ReLU mask, bias step) */
+  MAVG_K_WGRAD_SGD = 7, /* backward-weight GEMMs fused with the SGD step */
+  MAVG_K_AUX = 8,       /* operand copies (bf16 shadows) */
+  MAVG_K_COUNT = 9
+} mavg_kernel_class;
+mavg_status mavg_set_profiling(mavg_handle h, int32_t on);
+mavg_status mavg_get_profile(mavg_handle h, float *ms, int64_t *launches, int32_t reset);
+
 /* Waits for the stream; reports CUDA errors and a tripped device-side wait limit. */
 mavg_status mavg_sync(mavg_handle h);
 

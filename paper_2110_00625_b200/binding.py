@@ -19,7 +19,10 @@ STATUS = {0: "MAVG_OK", 1: "MAVG_ERR_INVALID_ARG", 2: "MAVG_ERR_BAD_BUFFER", 3: 
 EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta_update",
            "mavg_round", "mavg_round_host", "mavg_set_hparams", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
-           "mavg_sync", "mavg_last_error", "mavg_destroy"]
+           "mavg_set_profiling", "mavg_get_profile", "mavg_sync", "mavg_last_error",
+           "mavg_destroy"]
+KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
+                  "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
 
 
 class Config(C.Structure):
@@ -80,6 +83,8 @@ def load_library():
     L.mavg_get_round.argtypes = [H, C.POINTER(C.c_int64)]
     L.mavg_set_round.argtypes = [H, C.c_int64]
     L.mavg_get_launch_count.argtypes = [H, C.POINTER(C.c_int64)]
+    L.mavg_set_profiling.argtypes = [H, C.c_int32]
+    L.mavg_get_profile.argtypes = [H, C.c_void_p, C.c_void_p, C.c_int32]
     L.mavg_sync.argtypes = [H]
     L.mavg_last_error.argtypes = [H]
     L.mavg_last_error.restype = C.c_char_p
@@ -209,6 +214,16 @@ class Mavg:
         r = C.c_int64()
         self.lib.mavg_get_launch_count(self.handle, C.byref(r))
         return r.value
+
+    def set_profiling(self, on):
+        self._check(self.lib.mavg_set_profiling(self.handle, int(bool(on))))
+
+    def get_profile(self, reset=True):
+        """{kernel class: (milliseconds, launches)} since the last reset."""
+        ms = (C.c_float * len(KERNEL_CLASSES))()
+        cnt = (C.c_int64 * len(KERNEL_CLASSES))()
+        self._check(self.lib.mavg_get_profile(self.handle, ms, cnt, int(bool(reset))))
+        return {k: (ms[i], cnt[i]) for i, k in enumerate(KERNEL_CLASSES)}
 
     def sync(self):
         self._check(self.lib.mavg_sync(self.handle))

@@ -146,9 +146,10 @@ mavg_status do_meta_update(mavg_ctx* c) {
 mavg_status read_mean_loss(mavg_ctx* c, float* mean_loss) {
   if (c->cfg.objective == MAVG_OBJ_MLP) {
     float* lm = (float*)ws_ptr(c, c->ws.loss_mean);
+    prof_begin(c, MAVG_K_LOSS);
     k_mean_loss<<<1, 256, 0, c->stream>>>((const float*)ws_ptr(c, c->ws.losses),
                                           c->cfg.P * c->cfg.K, lm);
-    c->launches++;
+    prof_end(c);
     CU(c, cudaGetLastError(), "mean-loss kernel");
     CU(c, cudaMemcpyAsync(mean_loss, lm, sizeof(float), cudaMemcpyDeviceToHost, c->stream),
        "loss read-back");
@@ -349,6 +350,27 @@ mavg_status mavg_get_launch_count(mavg_handle h, int64_t* count) {
   return MAVG_OK;
 }
 
+mavg_status mavg_set_profiling(mavg_handle h, int32_t on) {
+  CHECK_HANDLE(h);
+  h->profiling = on != 0;
+  h->ev_open = nullptr;
+  return MAVG_OK;
+}
+
+mavg_status mavg_get_profile(mavg_handle h, float* ms, int64_t* launches, int32_t reset) {
+  CHECK_HANDLE(h);
+  if (!ms || !launches) return set_err(h, MAVG_ERR_INVALID_ARG, "ms or launches is NULL");
+  CU(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  for (int k = 0; k < MAVG_K_COUNT; ++k) { ms[k] = 0.f; launches[k] = 0; }
+  for (const auto& sp : h->spans) {
+    float t = 0.f;
+    CU(h, cudaEventElapsedTime(&t, sp.a, sp.b), "event elapsed time");
+    if (sp.cls >= 0 && sp.cls < MAVG_K_COUNT) { ms[sp.cls] += t; launches[sp.cls] += 1; }
+  }
+  if (reset) { h->spans.clear(); h->ev_used = 0; }
+  return MAVG_OK;
+}
+
 mavg_status mavg_sync(mavg_handle h) {
   CHECK_HANDLE(h);
   int32_t flag = 0;
@@ -371,6 +393,7 @@ const char* mavg_last_error(mavg_handle h) {
 
 mavg_status mavg_destroy(mavg_handle h) {
   if (!h) return MAVG_OK;
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   mlp_teardown(h);
   delete h;
   return MAVG_OK;

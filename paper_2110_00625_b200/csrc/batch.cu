@@ -108,23 +108,25 @@ k_softmax_ce(const float* __restrict__ logits, int ldz, const int32_t* __restric
 cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_first, int j_count,
                                  int32_t* idx, int32_t* labels) {
   const int total = j_count * c->cfg.B;
+  prof_begin(c, MAVG_K_BATCH);
   k_batch_indices<<<(total + 255) / 256, 256, 0, c->stream>>>(
       idx, labels, c->cfg.y, c->cfg.seed, round, step, c->cfg.P, c->cfg.B, c->cfg.n_samples,
       j_first, j_count);
-  c->launches++;
+  prof_end(c);
   return cudaGetLastError();
 }
 
 cudaError_t launch_gather(mavg_ctx* c, const int32_t* idx, int quant, float* out_f32,
                           __nv_bfloat16* out_bf, __nv_bfloat16* out_bft) {
   const int rows = c->cfg.P * c->cfg.B, d = c->cfg.dims[0];
+  prof_begin(c, MAVG_K_BATCH);
   if (c->cfg.x_dtype == MAVG_X_BF16)
     k_gather<__nv_bfloat16><<<rows, 256, 0, c->stream>>>((const __nv_bfloat16*)c->cfg.x, idx, d,
                                                          c->cfg.B, quant, out_f32, out_bf, out_bft);
   else
     k_gather<float><<<rows, 256, 0, c->stream>>>((const float*)c->cfg.x, idx, d, c->cfg.B, quant,
                                                  out_f32, out_bf, out_bft);
-  c->launches++;
+  prof_end(c);
   return cudaGetLastError();
 }
 
@@ -137,11 +139,12 @@ cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const i
   while (threads < B && threads < 256) threads <<= 1;
   size_t smem = (size_t)threads * sizeof(float);
   const MlpLayer& last = c->layers.back();
+  prof_begin(c, MAVG_K_LOSS);
   k_softmax_ce<<<P, threads, smem, c->stream>>>(
       logits, ldz, labels, B, C, loss_out, loss_stride, dz_f32, ld32, dz_bf, ldbf, dz_bft, ldbft,
       update_bias ? c->buf.replicas : nullptr, c->buf.replica_stride, last.b_off,
       c->cfg.local_lr);
-  c->launches++;
+  prof_end(c);
   return cudaGetLastError();
 }
 

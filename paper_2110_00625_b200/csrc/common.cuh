@@ -67,6 +67,14 @@ struct mavg_ctx {
   mavg::Workspace ws;
   std::vector<mavg::MlpLayer> layers;
   void* mlp = nullptr;        // state of the MLP path (owned by mlp files)
+  // per-launch timing (mavg_set_profiling): one event pair per launch, summed per kernel class
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  struct Span { int cls; cudaEvent_t a, b; };
+  std::vector<Span> spans;
+  cudaEvent_t ev_open = nullptr;
+  int cls_open = 0;
 };
 
 namespace mavg {
@@ -85,6 +93,30 @@ void mlp_teardown(mavg_ctx* c);
 cudaError_t mlp_refresh_shared_operands(mavg_ctx* c);   // after w~ changed
 cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round);
 cudaError_t mlp_indices_only(mavg_ctx* c, int64_t round, int learner, int step, int32_t* dev_out);
+
+// Bracket every kernel launch: prof_begin before it, prof_end after it (counts the launch).
+inline cudaEvent_t prof_event(mavg_ctx* c) {
+  if (c->ev_used == c->ev_pool.size()) {
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    c->ev_pool.push_back(e);
+  }
+  return c->ev_pool[c->ev_used++];
+}
+inline void prof_begin(mavg_ctx* c, int cls) {
+  if (!c->profiling) return;
+  c->ev_open = prof_event(c);
+  c->cls_open = cls;
+  cudaEventRecord(c->ev_open, c->stream);
+}
+inline void prof_end(mavg_ctx* c) {
+  c->launches++;
+  if (!c->profiling || !c->ev_open) return;
+  cudaEvent_t b = prof_event(c);
+  cudaEventRecord(b, c->stream);
+  c->spans.push_back({c->cls_open, c->ev_open, b});
+  c->ev_open = nullptr;
+}
 
 inline char* ws_ptr(mavg_ctx* c, size_t off) { return (char*)c->buf.workspace + off; }
 

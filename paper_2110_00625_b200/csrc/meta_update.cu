@@ -112,10 +112,11 @@ int grid_for(const mavg_ctx* c, int64_t work_items, int threads, int blocks_per_
 cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v) {
   const int64_t n = c->cfg.n;
   int grid = grid_for(c, n >> 2, 256, 8);
+  prof_begin(c, MAVG_K_BROADCAST);
   k_broadcast<<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
                                            c->buf.global_w, c->buf.momentum, c->cfg.P, n,
                                            zero_v ? 1 : 0);
-  c->launches++;
+  prof_end(c);
   return cudaGetLastError();
 }
 
@@ -129,6 +130,7 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
   // A replica set that fits in L2 is about to be re-read by the next round's first local step:
   // keep it there.  Larger sets are written with evict-first stores.
   const bool stream_st = (size_t)P * (size_t)n * 4 > c->l2_bytes / 2;
+  prof_begin(c, MAVG_K_META);
   if (stream_st)
     k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
                                                         c->buf.global_w, c->buf.momentum, P, n,
@@ -137,7 +139,7 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
     k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
                                                          c->buf.global_w, c->buf.momentum, P, n,
                                                          mu, zeta, inv_p, read_v);
-  c->launches++;
+  prof_end(c);
   return cudaGetLastError();
 }
 

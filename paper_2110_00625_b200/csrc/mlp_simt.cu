@@ -170,11 +170,12 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
     g.C = sb.z[l]; g.c_batch = (int64_t)B * ly.out; g.c_m = ly.out;
     g.aux = rep + ly.b_off; g.aux_batch = rs; g.aux_m = 0;
     dim3 grid((ly.out + BN - 1) / BN, (B + BM - 1) / BM, P);
+    prof_begin(c, MAVG_K_FWD);
     if (l == 1)
       k_simt_gemm<QUANT, LD_PLAIN, LD_PLAIN, true, true, EPI_FWD><<<grid, 256, 0, c->stream>>>(g);
     else
       k_simt_gemm<QUANT, LD_RELU, LD_PLAIN, true, true, EPI_FWD><<<grid, 256, 0, c->stream>>>(g);
-    c->launches++;
+    prof_end(c);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   // loss, dZ_L and the last bias
@@ -193,8 +194,9 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
       g.C = sb.dz[l - 1]; g.c_batch = (int64_t)B * ly.in; g.c_m = ly.in;
       g.aux = sb.z[l - 1]; g.aux_batch = (int64_t)B * ly.in; g.aux_m = ly.in;
       dim3 grid((ly.in + BN - 1) / BN, (B + BM - 1) / BM, P);
+      prof_begin(c, MAVG_K_DGRAD);
       k_simt_gemm<QUANT, LD_PLAIN, LD_PLAIN, true, false, EPI_DGRAD><<<grid, 256, 0, c->stream>>>(g);
-      c->launches++;
+      prof_end(c);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     {
@@ -205,18 +207,20 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
       g.C = rep + ly.w_off; g.c_batch = rs; g.c_m = ly.in;
       g.gamma = cfg.local_lr;
       dim3 grid((ly.in + BN - 1) / BN, (ly.out + BM - 1) / BM, P);
+      prof_begin(c, MAVG_K_WGRAD_SGD);
       if (l == 1)
         k_simt_gemm<QUANT, LD_PLAIN, LD_PLAIN, false, false, EPI_WGRAD_SGD><<<grid, 256, 0, c->stream>>>(g);
       else
         k_simt_gemm<QUANT, LD_PLAIN, LD_RELU, false, false, EPI_WGRAD_SGD><<<grid, 256, 0, c->stream>>>(g);
-      c->launches++;
+      prof_end(c);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     if (l < L) {
       dim3 grid((ly.out + 255) / 256, P);
+      prof_begin(c, MAVG_K_WGRAD_SGD);
       k_simt_bias_sgd<<<grid, 256, 0, c->stream>>>(sb.dz[l], (int64_t)B * ly.out, B, ly.out, rep,
                                                    rs, ly.b_off, cfg.local_lr);
-      c->launches++;
+      prof_end(c);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
   }

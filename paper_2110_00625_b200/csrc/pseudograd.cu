@@ -64,10 +64,11 @@ cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round) {
   for (int k0 = 0; k0 < K; k0 += kMaxFused) {
     int kc = K - k0 < kMaxFused ? K - k0 : kMaxFused;
     dim3 grid((unsigned)blocks_x, (unsigned)P);
+    prof_begin(c, MAVG_K_PSEUDOGRAD);
     k_pseudograd_steps<<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
         c->buf.replicas, c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
         c->cfg.local_lr);
-    c->launches++;
+    prof_end(c);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -197,6 +197,7 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
     return fail(&g_create_error, MAVG_ERR_BAD_BUFFER, "workspace is smaller than mavg_workspace_bytes");
 
   int dev = 0;
+  cudaGetLastError();   // a stale non-sticky error of earlier, unrelated calls is not ours
   cudaError_t e = cudaGetDevice(&dev);
   cudaDeviceProp prop;
   if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, dev);

@@ -11,3 +11,18 @@ def rel_err(x, y):
     rms = float(np.sqrt(np.mean(y * y))) if y.size else 0.0
     den = np.maximum(np.abs(y), max(rms, 1e-30))
     return float((np.abs(x - y) / den).max()) if y.size else 0.0
+
+
+def outlier_fraction(x, y, tol):
+    """Fraction of elements whose error (same metric as rel_err) exceeds tol."""
+    x = np.asarray(x, dtype=np.float64).reshape(-1)
+    y = np.asarray(y, dtype=np.float64).reshape(-1)
+    rms = float(np.sqrt(np.mean(y * y)))
+    den = np.maximum(np.abs(y), max(rms, 1e-30))
+    return float(np.mean(np.abs(x - y) / den > tol))
+
+
+def l2_rel(x, y):
+    x = np.asarray(x, dtype=np.float64).reshape(-1)
+    y = np.asarray(y, dtype=np.float64).reshape(-1)
+    return float(np.linalg.norm(x - y) / max(np.linalg.norm(y), 1e-30))

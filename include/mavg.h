@@ -176,6 +176,27 @@ mavg_status mavg_sync(mavg_handle h);
  * mavg_create / mavg_workspace_bytes of the calling thread.  Valid until the next call. */
 const char *mavg_last_error(mavg_handle h);
 
+/* The index stream of mavg_get_batch_indices for callers that cannot allocate device memory (the
+ * paper has no counterpart; this is an addition for such hosts).  Think of a process whose
+ * device memory has all been handed to another component's pool, a plug-in that runs under a
+ * fixed memory budget, or a latency-critical loop that must not call cudaMalloc because that
+ * call may stall the whole device: none of them can provide the workspace a handle needs.
+ * Here no handle and no workspace exist.  The B indices that `learner` draws at local step
+ * `step` of round `round` (same generator, same shard rule, same bits as the handle-based call)
+ * are staged in an array that is part of the library image on the GPU -- 65536 int32 = 256 KB,
+ * held by every GPU that loads the library until the process exits -- and copied to out
+ * (HOST, B int32); the call waits for the stream.  B > 65536 is refused with
+ * MAVG_ERR_INVALID_ARG.  The call itself allocates and frees nothing.
+ * The first call on a device looks up the array's device address (the device must be current);
+ * make that first call before any stream capture begins.  All calls share the one array, which
+ * keeps the previous call's indices; nothing in it needs clearing because every call overwrites
+ * the B entries it reads back.  Two calls in flight at once on the same GPU (different host
+ * threads or streams) would race on it: issue them one after the other.
+ * stream: cudaStream_t (NULL = default stream).  Errors: mavg_last_error(NULL). */
+mavg_status mavg_batch_indices_noalloc(uint64_t seed, int64_t round, int32_t P, int32_t learner,
+                                       int32_t step, int64_t n_samples, int32_t B, void *stream,
+                                       int32_t *out);
+
 /* Releases the handle (host memory only).  NULL is a no-op. */
 mavg_status mavg_destroy(mavg_handle h);
 

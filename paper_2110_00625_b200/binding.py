@@ -20,7 +20,7 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_round", "mavg_round_host", "mavg_set_hparams", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
            "mavg_set_profiling", "mavg_get_profile", "mavg_sync", "mavg_last_error",
-           "mavg_destroy"]
+           "mavg_batch_indices_noalloc", "mavg_destroy"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
 
@@ -85,6 +85,9 @@ def load_library():
     L.mavg_get_launch_count.argtypes = [H, C.POINTER(C.c_int64)]
     L.mavg_set_profiling.argtypes = [H, C.c_int32]
     L.mavg_get_profile.argtypes = [H, C.c_void_p, C.c_void_p, C.c_int32]
+    L.mavg_batch_indices_noalloc.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32,
+                                             C.c_int32, C.c_int64, C.c_int32, C.c_void_p,
+                                             C.c_void_p]
     L.mavg_sync.argtypes = [H]
     L.mavg_last_error.argtypes = [H]
     L.mavg_last_error.restype = C.c_char_p
@@ -113,6 +116,19 @@ def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NON
     cfg.x, cfg.x_dtype, cfg.y, cfg.n_samples = x_ptr, x_dtype, y_ptr, n_samples
     cfg.stream = stream
     return cfg
+
+
+def batch_indices_noalloc(seed, round_, P, learner, step, n_samples, B, stream=0):
+    """mavg_batch_indices_noalloc: the B sample indices of (round, learner, step) computed on the
+    current CUDA device without a handle, a workspace or any allocation by the library."""
+    import numpy as np
+    L = load_library()
+    out = np.empty(max(B, 1), dtype=np.int32)
+    st = L.mavg_batch_indices_noalloc(seed, round_, P, learner, step, n_samples, B, stream,
+                                      out.ctypes.data)
+    if st != 0:
+        raise MavgError(st, L.mavg_last_error(None).decode())
+    return out[:B]
 
 
 class Mavg:

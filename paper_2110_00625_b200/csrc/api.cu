@@ -163,6 +163,10 @@ mavg_status read_mean_loss(mavg_ctx* c, float* mean_loss) {
 
 }  // namespace
 
+namespace mavg {
+void set_thread_error(const std::string& msg) { g_create_error = msg; }
+}  // namespace mavg
+
 extern "C" {
 
 mavg_status mavg_workspace_bytes(const mavg_config* cfg, size_t* out_bytes) {

@@ -1,6 +1,8 @@
 // Minibatch side of the learner level: "randomly sample a mini-batch of size B_n"
 // (Algorithm 1) as a counter-based index stream, the gather of the sampled rows, and the softmax
 // cross-entropy loss with its gradient (the 1/B_n mean of Algorithm 1's update).
+#include <mutex>
+
 #include "mlp.cuh"
 
 namespace mavg {
@@ -149,3 +151,74 @@ cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const i
 }
 
 }  // namespace mavg
+
+namespace mavg {
+// ------------------------------------------------------------------------------------------------
+// mavg_batch_indices_noalloc: the index stream without a handle and without any allocation.
+// The B indices are staged in a fixed array that lives in the library's device image (every GPU
+// that loads the library carries these 256 KB until the process exits) and are then copied to
+// the caller's host buffer.
+namespace {
+
+constexpr int kNoAllocMaxB = 65536;
+static __device__ __align__(256) int32_t g_noalloc_idx[kNoAllocMaxB];
+
+constexpr int kNoAllocMaxDevices = 64;
+int32_t* g_noalloc_ptr[kNoAllocMaxDevices] = {};
+std::mutex g_noalloc_mutex;
+
+// In host code the array's name is only a handle for the runtime, not a device address; the
+// address on the current device is looked up once per device and remembered.
+cudaError_t noalloc_scratch(int device, int32_t** out) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[device]) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_idx);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[device] = (int32_t*)ptr;
+  }
+  *out = g_noalloc_ptr[device];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace mavg
+
+extern "C" mavg_status mavg_batch_indices_noalloc(uint64_t seed, int64_t round, int32_t P,
+                                                  int32_t learner, int32_t step,
+                                                  int64_t n_samples, int32_t B, void* stream,
+                                                  int32_t* out) {
+  using namespace mavg;
+  if (!out || round < 1 || step < 1 || P < 1 || learner < 0 || learner >= P || B < 1 ||
+      n_samples < P || n_samples >= ((int64_t)1 << 31)) {
+    set_thread_error("mavg_batch_indices_noalloc: bad round, P, learner, step, n_samples, B or out");
+    return MAVG_ERR_INVALID_ARG;
+  }
+  if (B > kNoAllocMaxB) {
+    set_thread_error("mavg_batch_indices_noalloc: B exceeds the built-in staging array of 65536 "
+                     "indices; use mavg_get_batch_indices with a workspace instead");
+    return MAVG_ERR_INVALID_ARG;
+  }
+  int device = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e == cudaSuccess && (device < 0 || device >= kNoAllocMaxDevices)) {
+    set_thread_error("mavg_batch_indices_noalloc: device ordinal out of range");
+    return MAVG_ERR_UNSUPPORTED;
+  }
+  int32_t* scratch = nullptr;
+  if (e == cudaSuccess) e = noalloc_scratch(device, &scratch);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (e == cudaSuccess) {
+    k_batch_indices<<<(B + 255) / 256, 256, 0, s>>>(scratch, nullptr, nullptr, seed, round, step,
+                                                    P, B, n_samples, learner, 1);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(out, scratch, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    set_thread_error(std::string("mavg_batch_indices_noalloc: ") + cudaGetErrorString(e));
+    return MAVG_ERR_CUDA;
+  }
+  return MAVG_OK;
+}

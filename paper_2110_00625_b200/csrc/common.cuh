@@ -118,6 +118,9 @@ inline void prof_end(mavg_ctx* c) {
   c->ev_open = nullptr;
 }
 
+// Message returned by mavg_last_error(NULL) on the calling thread.
+void set_thread_error(const std::string& msg);
+
 inline char* ws_ptr(mavg_ctx* c, size_t off) { return (char*)c->buf.workspace + off; }
 
 }  // namespace mavg

@@ -13,8 +13,10 @@
  *
  * Conventions
  *   - Every pointer is tagged DEVICE or HOST below.  Device buffers and the CUDA stream belong to
- *     the caller and are borrowed from mavg_create until mavg_destroy; the library allocates no
- *     device memory and frees none.  The handle is host memory owned by the library.
+ *     the caller and are borrowed from mavg_create until mavg_destroy; the library calls no
+ *     device allocator and frees nothing of the caller's.  The handle is host memory owned by the
+ *     library; for the MLP objective it also holds a CUDA graph of one round's local steps
+ *     (recorded on a private stream at the first round, replayed on the caller's stream).
  *   - All work is enqueued on the configured stream and returns without waiting, except where a
  *     function hands a value back to HOST memory (then it waits for the stream).
  *   - Errors are status codes; nothing throws, aborts or traps.  Arguments are checked on the

@@ -12,9 +12,11 @@ namespace {
 // stream value (see mavg.h).  Also fetches the label.
 __global__ void k_batch_indices(int32_t* __restrict__ idx, int32_t* __restrict__ labels,
                                 const int32_t* __restrict__ y, uint64_t seed, int64_t round,
-                                int step, int P, int B, int64_t S, int j_first, int j_count) {
+                                const int64_t* __restrict__ round_ptr, int step, int P, int B,
+                                int64_t S, int j_first, int j_count) {
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= j_count * B) return;
+  if (round_ptr) round = *round_ptr;   // replayed launches read the round from device memory
   int j = j_first + t / B, s = t % B;
   int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
   int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
@@ -112,8 +114,9 @@ cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_fir
   const int total = j_count * c->cfg.B;
   prof_begin(c, MAVG_K_BATCH);
   k_batch_indices<<<(total + 255) / 256, 256, 0, c->stream>>>(
-      idx, labels, c->cfg.y, c->cfg.seed, round, step, c->cfg.P, c->cfg.B, c->cfg.n_samples,
-      j_first, j_count);
+      idx, labels, c->cfg.y, c->cfg.seed, round,
+      c->capturing ? (const int64_t*)(ws_ptr(c, c->ws.status) + 64) : nullptr, step, c->cfg.P,
+      c->cfg.B, c->cfg.n_samples, j_first, j_count);
   prof_end(c);
   return cudaGetLastError();
 }
@@ -209,8 +212,8 @@ extern "C" mavg_status mavg_batch_indices_noalloc(uint64_t seed, int64_t round, 
   if (e == cudaSuccess) e = noalloc_scratch(device, &scratch);
   cudaStream_t s = (cudaStream_t)stream;
   if (e == cudaSuccess) {
-    k_batch_indices<<<(B + 255) / 256, 256, 0, s>>>(scratch, nullptr, nullptr, seed, round, step,
-                                                    P, B, n_samples, learner, 1);
+    k_batch_indices<<<(B + 255) / 256, 256, 0, s>>>(scratch, nullptr, nullptr, seed, round,
+                                                    nullptr, step, P, B, n_samples, learner, 1);
     e = cudaGetLastError();
   }
   if (e == cudaSuccess)

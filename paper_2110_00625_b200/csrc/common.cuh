@@ -42,7 +42,7 @@ struct MlpLayer {
 };
 
 struct Workspace {           // byte offsets into the caller's scratch buffer
-  size_t status = 0;         // int32[64]: [0] device wait-limit flag
+  size_t status = 0;         // int32[64]: [0] device wait-limit flag; bytes 64..71: round (int64)
   size_t losses = 0;         // float [P*K]
   size_t loss_mean = 0;      // float [1]
   size_t idx = 0;            // int32 [P*B] sample indices of the current step
@@ -75,6 +75,15 @@ struct mavg_ctx {
   std::vector<Span> spans;
   cudaEvent_t ev_open = nullptr;
   int cls_open = 0;
+  // CUDA graph of one round's K local steps (MLP objective): captured once on a private stream,
+  // replayed on the caller's stream; rebuilt when K or the local learning rate change
+  bool capturing = false;
+  bool graph_disabled = false;
+  cudaGraphExec_t graph_exec = nullptr;
+  cudaStream_t cap_stream = nullptr;
+  int graph_K = 0;
+  float graph_lr = 0.f;
+  int64_t graph_nodes = 0;
 };
 
 namespace mavg {

@@ -40,7 +40,10 @@ mavg_status mlp_setup(mavg_ctx* c) {
   return MAVG_OK;
 }
 
+void mlp_drop_graph(mavg_ctx* c);
+
 void mlp_teardown(mavg_ctx* c) {
+  mlp_drop_graph(c);
   if (c->mlp) tc_teardown(c);
 }
 
@@ -49,12 +52,93 @@ cudaError_t mlp_refresh_shared_operands(mavg_ctx* c) {
   return cudaSuccess;
 }
 
-cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
+namespace {
+
+__global__ void k_set_round(int64_t* dst, int64_t round) { *dst = round; }
+
+cudaError_t run_steps(mavg_ctx* c, int64_t round) {
   for (int k = 1; k <= c->cfg.K; ++k) {
     cudaError_t e = use_tensor_cores(&c->cfg) ? tc_step(c, round, k) : simt_step(c, round, k);
     if (e != cudaSuccess) return e;
     c->replicas_equal_global = false;
   }
+  return cudaSuccess;
+}
+
+void drop_graph(mavg_ctx* c) {
+  if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+  c->graph_exec = nullptr;
+}
+
+// Records the K steps of a round that starts from the broadcast state into a graph.  The steps
+// are issued on a private capturing stream; nothing runs until the graph is launched.
+cudaError_t build_graph(mavg_ctx* c, int64_t round) {
+  drop_graph(c);
+  cudaError_t e = cudaSuccess;
+  if (!c->cap_stream) {
+    e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return e;
+  }
+  e = cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) return e;
+  cudaStream_t user = c->stream;
+  const int64_t before = c->launches;
+  c->stream = c->cap_stream;
+  c->capturing = true;
+  c->replicas_equal_global = true;
+  cudaError_t run = run_steps(c, round);
+  c->capturing = false;
+  c->stream = user;
+  c->graph_nodes = c->launches - before;
+  c->launches = before;
+  cudaGraph_t graph = nullptr;
+  e = cudaStreamEndCapture(c->cap_stream, &graph);
+  if (run != cudaSuccess || e != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    return run != cudaSuccess ? run : e;
+  }
+  e = cudaGraphInstantiate(&c->graph_exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) {
+    c->graph_exec = nullptr;
+    return e;
+  }
+  c->graph_K = c->cfg.K;
+  c->graph_lr = c->cfg.local_lr;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+void mlp_drop_graph(mavg_ctx* c) {
+  drop_graph(c);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  c->cap_stream = nullptr;
+}
+
+cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
+  // The usual round starts from the broadcast state and is replayed from a graph.  Rounds that
+  // start elsewhere (local steps called twice in a row), profiled rounds and handles whose
+  // capture failed once take the launch-by-launch path.
+  const bool want_graph = !c->profiling && !c->graph_disabled && c->replicas_equal_global;
+  if (!want_graph) return run_steps(c, round);
+  if (!c->graph_exec || c->graph_K != c->cfg.K || c->graph_lr != c->cfg.local_lr) {
+    cudaError_t e = build_graph(c, round);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      c->graph_disabled = true;
+      c->replicas_equal_global = true;
+      return run_steps(c, round);
+    }
+  }
+  k_set_round<<<1, 1, 0, c->stream>>>((int64_t*)(ws_ptr(c, c->ws.status) + 64), round);
+  c->launches++;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  e = cudaGraphLaunch(c->graph_exec, c->stream);
+  if (e != cudaSuccess) return e;
+  c->launches += c->graph_nodes;
+  c->replicas_equal_global = false;
   return cudaSuccess;
 }
 

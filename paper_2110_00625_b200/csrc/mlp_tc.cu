@@ -27,7 +27,8 @@ using namespace tc;
 
 constexpr int kBM = 128;        // MMA M (rows of operand A per tile)
 constexpr int kBK = 64;         // contraction elements per pipeline stage (128 bytes of bf16)
-constexpr int kThreads = 192;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int kThreads = 320;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
+constexpr int kStageBytes = 8 * 32 * 33 * 4;   // per-warp 32x32 fp32 turn-around tiles (wgrad)
 constexpr int kMaxStages = 8;
 constexpr int kATileBytes = kBM * kBK * 2;
 
@@ -148,13 +149,18 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     }
     __syncwarp();
   } else {
-    const int q = warp & 3;                  // this warp may touch TMEM lanes [32q, 32q+32)
+    // 8 epilogue warps: warp (q, half) owns TMEM lanes [32q, 32q+32) -- the only lanes a warp
+    // with (warp index mod 4) == q may read -- and every second 32-column chunk.
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int half = ew >> 2;
     const int row = q * 32 + lane;
     const bool ok = mbar_wait(&acc_bar, 0, abortp, g.status, ERR_EPILOGUE);
     tc_fence_after_sync();
     if (ok) {
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      for (int c0 = 0; c0 < g.BN; c0 += 32) {
+      float* stage = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes) + ew * (32 * 33);
+      for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
         uint32_t r[32];
         if (c0 + 32 <= g.BN) {
           tmem_ld_32x32(lane_addr + (uint32_t)c0, r);
@@ -177,51 +183,45 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
           }
         } else {
-          const int o = m0 + row;
-          if (o < g.out) {
-            float* wrow = g.rep + (size_t)p * g.rep_stride + g.w_off + (size_t)o * g.in;
-            __nv_bfloat16* hrow = g.w16 + (size_t)p * g.w16_stride + g.sh_off + (size_t)o * g.in;
-            __nv_bfloat16* tcol =
-                g.wt16 ? g.wt16 + (size_t)p * g.wt16_stride + g.sht_off + o : nullptr;
+          // The accumulator arrives with one weight row per lane.  It is turned through shared
+          // memory so that the lanes of a warp walk along a row: every access to the fp32 masters
+          // and to the [out, in] bf16 copy is then a contiguous 128 / 64 bytes per row.
 #pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {  // 8 columns at a time: in is a multiple of 8
-              const int i = n0 + c0 + j8 * 8;
-              if (j8 * 8 < ncols && i < g.in) {
-                float4 w0 = *reinterpret_cast<const float4*>(wrow + i);
-                float4 w1 = *reinterpret_cast<const float4*>(wrow + i + 4);
-                w0.x = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 0]), w0.x);
-                w0.y = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 1]), w0.y);
-                w0.z = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 2]), w0.z);
-                w0.w = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 3]), w0.w);
-                w1.x = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 4]), w1.x);
-                w1.y = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 5]), w1.y);
-                w1.z = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 6]), w1.z);
-                w1.w = fmaf(-g.gamma, __uint_as_float(r[j8 * 8 + 7]), w1.w);
-                *reinterpret_cast<float4*>(wrow + i) = w0;
-                *reinterpret_cast<float4*>(wrow + i + 4) = w1;
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(w0.x, w0.y);
-                __nv_bfloat162 h1 = __floats2bfloat162_rn(w0.z, w0.w);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(w1.x, w1.y);
-                __nv_bfloat162 h3 = __floats2bfloat162_rn(w1.z, w1.w);
-                uint4 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&h0);
-                pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                pk.z = *reinterpret_cast<uint32_t*>(&h2);
-                pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                *reinterpret_cast<uint4*>(hrow + i) = pk;
-                if (tcol) {
-                  tcol[(size_t)(i + 0) * g.out_pad] = h0.x;
-                  tcol[(size_t)(i + 1) * g.out_pad] = h0.y;
-                  tcol[(size_t)(i + 2) * g.out_pad] = h1.x;
-                  tcol[(size_t)(i + 3) * g.out_pad] = h1.y;
-                  tcol[(size_t)(i + 4) * g.out_pad] = h2.x;
-                  tcol[(size_t)(i + 5) * g.out_pad] = h2.y;
-                  tcol[(size_t)(i + 6) * g.out_pad] = h3.x;
-                  tcol[(size_t)(i + 7) * g.out_pad] = h3.y;
-                }
+          for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]);
+          __syncwarp();
+          const int o_base = m0 + q * 32;
+          const int i = n0 + c0 + lane;
+          const bool col_ok = lane < ncols && i < g.in;
+          float* wcol = g.rep + (size_t)p * g.rep_stride + g.w_off + (size_t)o_base * g.in + i;
+          __nv_bfloat16* hcol =
+              g.w16 + (size_t)p * g.w16_stride + g.sh_off + (size_t)o_base * g.in + i;
+          float wv[32];
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr)
+            wv[rr] = (col_ok && o_base + rr < g.out) ? wcol[(size_t)rr * g.in] : 0.f;
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr) {
+            const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
+            if (col_ok && o_base + rr < g.out) {
+              wcol[(size_t)rr * g.in] = w;
+              hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
+            }
+            stage[rr * 33 + lane] = w;
+          }
+          __syncwarp();
+          if (g.wt16) {                       // [in, out] copy: lanes walk along out again
+            const int o = o_base + lane;
+            if (o < g.out) {
+              __nv_bfloat16* tcol = g.wt16 + (size_t)p * g.wt16_stride + g.sht_off + o;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const int ii = n0 + c0 + j;
+                if (j < ncols && ii < g.in)
+                  tcol[(size_t)ii * g.out_pad] = __float2bfloat16_rn(stage[lane * 33 + j]);
               }
             }
           }
+          __syncwarp();
         }
       }
     }
@@ -381,7 +381,7 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count) {
 
 GemmPlan plan_wgrad(int out, int in, int B) {
   GemmPlan g{};
-  g.BN = in >= 256 ? 256 : (in + 15) / 16 * 16;
+  g.BN = in >= 128 ? 128 : (in + 15) / 16 * 16;
   g.m_tiles = (out + kBM - 1) / kBM;
   g.n_tiles = (in + g.BN - 1) / g.BN;
   g.nkb = (B + kBK - 1) / kBK;
@@ -497,7 +497,8 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   g.tmem_cols = pl.tmem_cols;
   g.P = c->cfg.P;
   g.status = (int*)ws_ptr(c, c->ws.status);
-  const size_t smem = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2) + 1024;
+  const size_t smem = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2) + 1024 +
+                      (EPI == EPI_WGRAD_SGD ? kStageBytes : 0);
   dim3 grid((unsigned)(pl.m_tiles * pl.n_tiles * pl.splits), (unsigned)c->cfg.P);
   prof_begin(c, cls);
   k_tc_gemm<EPI><<<grid, kThreads, smem, c->stream>>>(a, b, g);

@@ -8,8 +8,17 @@
 namespace mavg {
 namespace {
 
-// One thread per (learner, slot): idx = lo_j + floor(u * len_j / 2^32), u = top 32 bits of the
-// stream value (see mavg.h).  Also fetches the label.
+// idx = lo_j + floor(u * len_j / 2^32), u = top 32 bits of the stream value (see mavg.h).
+__device__ __forceinline__ int32_t sample_index(uint64_t seed, int64_t round, int j, int step,
+                                                int s, int P, int64_t S) {
+  int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
+  int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
+  uint64_t key = fold(learner_key(seed, kTagBatch, (uint64_t)round, (uint64_t)j), (uint64_t)step);
+  uint64_t u = fold(key, (uint64_t)s) >> 32;
+  return (int32_t)(lo + (int64_t)((u * (uint64_t)(hi - lo)) >> 32));
+}
+
+// One thread per (learner, slot).  Also fetches the label.
 __global__ void k_batch_indices(int32_t* __restrict__ idx, int32_t* __restrict__ labels,
                                 const int32_t* __restrict__ y, uint64_t seed, int64_t round,
                                 const int64_t* __restrict__ round_ptr, int step, int P, int B,
@@ -18,11 +27,7 @@ __global__ void k_batch_indices(int32_t* __restrict__ idx, int32_t* __restrict__
   if (t >= j_count * B) return;
   if (round_ptr) round = *round_ptr;   // replayed launches read the round from device memory
   int j = j_first + t / B, s = t % B;
-  int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
-  int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
-  uint64_t key = fold(learner_key(seed, kTagBatch, (uint64_t)round, (uint64_t)j), (uint64_t)step);
-  uint64_t u = fold(key, (uint64_t)s) >> 32;
-  int32_t i = (int32_t)(lo + (int64_t)((u * (uint64_t)(hi - lo)) >> 32));
+  int32_t i = sample_index(seed, round, j, step, s, P, S);
   idx[t] = i;
   if (labels) labels[t] = y[i];
 }
@@ -52,6 +57,58 @@ k_gather(const TIN* __restrict__ x, const int32_t* __restrict__ idx, int d, int 
     if (out_f32) out_f32[(size_t)row * d + i] = quant ? __bfloat162float(b) : v;
     if (out_bf) out_bf[(size_t)row * d + i] = b;
     if (out_bft) out_bft[((size_t)p * d + i) * B + s] = b;
+  }
+}
+
+// Index stream and gather in one kernel, for bf16 operands: block (32, 8) handles 32 batch slots of
+// learner blockIdx.z and 64 input columns; it writes the rows [P, B, d] and, through a
+// shared-memory tile, their transpose [P, d, B].  Blocks of the first column chunk also write the
+// indices and labels.  d is a multiple of 8, B a multiple of 16.
+template <typename TIN>
+__global__ void __launch_bounds__(256)
+k_sample_gather(const TIN* __restrict__ x, const int32_t* __restrict__ y, uint64_t seed,
+                int64_t round, const int64_t* __restrict__ round_ptr, int step, int P, int B,
+                int64_t S, int d, int32_t* __restrict__ idx_out, int32_t* __restrict__ labels_out,
+                __nv_bfloat16* __restrict__ out_bf, __nv_bfloat16* __restrict__ out_bft) {
+  __shared__ int32_t sidx[32];
+  __shared__ __nv_bfloat16 tile[32][66];
+  const int p = blockIdx.z, s0 = blockIdx.x * 32, c0 = blockIdx.y * 64;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  if (round_ptr) round = *round_ptr;
+  if (ty == 0) {
+    const int s = s0 + tx;
+    int32_t i = 0;
+    if (s < B) {
+      i = sample_index(seed, round, p, step, s, P, S);
+      if (blockIdx.y == 0) {
+        idx_out[p * B + s] = i;
+        labels_out[p * B + s] = y[i];
+      }
+    }
+    sidx[tx] = i;
+  }
+  __syncthreads();
+  const int c = c0 + 2 * tx;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int sl = ty + 8 * r, s = s0 + sl;
+    __nv_bfloat16 v0 = __float2bfloat16_rn(0.f), v1 = v0;
+    if (s < B && c < d) {                      // d is even: c + 1 < d as well
+      const TIN* src = x + (size_t)sidx[sl] * d + c;
+      v0 = __float2bfloat16_rn(to_f32<TIN>(src[0]));
+      v1 = __float2bfloat16_rn(to_f32<TIN>(src[1]));
+      __nv_bfloat162 pr;
+      pr.x = v0; pr.y = v1;
+      *reinterpret_cast<__nv_bfloat162*>(out_bf + ((size_t)p * B + s) * d + c) = pr;
+    }
+    tile[sl][2 * tx] = v0;
+    tile[sl][2 * tx + 1] = v1;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const int cl = ty + 8 * r, cc = c0 + cl, s = s0 + tx;
+    if (cc < d && s < B) out_bft[((size_t)p * d + cc) * B + s] = tile[tx][cl];
   }
 }
 
@@ -117,6 +174,24 @@ cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_fir
       idx, labels, c->cfg.y, c->cfg.seed, round,
       c->capturing ? (const int64_t*)(ws_ptr(c, c->ws.status) + 64) : nullptr, step, c->cfg.P,
       c->cfg.B, c->cfg.n_samples, j_first, j_count);
+  prof_end(c);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sample_gather(mavg_ctx* c, int64_t round, int step, int32_t* idx,
+                                 int32_t* labels, __nv_bfloat16* out_bf, __nv_bfloat16* out_bft) {
+  const int P = c->cfg.P, B = c->cfg.B, d = c->cfg.dims[0];
+  dim3 grid((B + 31) / 32, (d + 63) / 64, P), block(32, 8);
+  const int64_t* rp = c->capturing ? (const int64_t*)(ws_ptr(c, c->ws.status) + 64) : nullptr;
+  prof_begin(c, MAVG_K_BATCH);
+  if (c->cfg.x_dtype == MAVG_X_BF16)
+    k_sample_gather<__nv_bfloat16><<<grid, block, 0, c->stream>>>(
+        (const __nv_bfloat16*)c->cfg.x, c->cfg.y, c->cfg.seed, round, rp, step, P, B,
+        c->cfg.n_samples, d, idx, labels, out_bf, out_bft);
+  else
+    k_sample_gather<float><<<grid, block, 0, c->stream>>>(
+        (const float*)c->cfg.x, c->cfg.y, c->cfg.seed, round, rp, step, P, B, c->cfg.n_samples, d,
+        idx, labels, out_bf, out_bft);
   prof_end(c);
   return cudaGetLastError();
 }

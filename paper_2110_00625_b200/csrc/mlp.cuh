@@ -10,6 +10,8 @@ cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_fir
                                  int32_t* idx, int32_t* labels);
 cudaError_t launch_gather(mavg_ctx* c, const int32_t* idx, int quant, float* out_f32,
                           __nv_bfloat16* out_bf, __nv_bfloat16* out_bft);
+cudaError_t launch_sample_gather(mavg_ctx* c, int64_t round, int step, int32_t* idx,
+                                 int32_t* labels, __nv_bfloat16* out_bf, __nv_bfloat16* out_bft);
 cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const int32_t* labels,
                               float* loss_out, int loss_stride, float* dz_f32, int ld32,
                               __nv_bfloat16* dz_bf, int ldbf, __nv_bfloat16* dz_bft, int ldbft,

@@ -10,9 +10,12 @@
 // ([B, f] and [f, B]) and the weights' bf16 copy in both ([out, in] and, for layers >= 2,
 // [in, out]); the producing epilogues write both.  fp32 master weights take the SGD step of
 // Algorithm 1 in the wgrad epilogue, which also refreshes the bf16 copies.
-// Forward and dgrad write fp32 partial tiles (split over the contraction when there are too few
-// tiles to fill the GPU); small finishing kernels add the partials in a fixed order and apply
-// bias/ReLU or the ReLU mask and the bias step.
+// When a layer has too few output tiles to fill the GPU, forward and dgrad split the contraction
+// over several blocks; each writes an fp32 partial tile and the block that finishes last adds
+// the partials in ascending split order (so the result does not depend on which block that is).
+// That block -- or the only block, when there is no split -- applies the layer's tail in the
+// same kernel: bias + ReLU, or the ReLU mask with the bias step of the layer below, or for the
+// last layer the softmax cross-entropy loss, dZ_L and the last bias step.
 #include <cuda.h>
 
 #include <algorithm>
@@ -32,19 +35,31 @@ constexpr int kStageBytes = 8 * 32 * 33 * 4;   // per-warp 32x32 fp32 turn-aroun
 constexpr int kMaxStages = 8;
 constexpr int kATileBytes = kBM * kBK * 2;
 
-enum { EPI_PARTIAL = 0, EPI_WGRAD_SGD = 1 };
+enum { EPI_FWD_HIDDEN = 0, EPI_FWD_LAST = 1, EPI_DGRAD = 2, EPI_WGRAD_SGD = 3 };
 enum { ERR_PRODUCER = 11, ERR_MMA = 12, ERR_EPILOGUE = 13 };
 
 struct TcArgs {
   int M, N;                 // valid rows of A and of B
   int BN;                   // N tile: multiple of 16, <= 256
-  int n_tiles, splits, kb_per_split, nkb, stages;
+  int m_tiles, n_tiles, splits, kb_per_split, nkb, stages;
   int a_batched, b_batched; // 0: the operand is shared by all learners
   int P;
   uint32_t tmem_cols;
-  // EPI_PARTIAL: part[((split*P + p)*N + n)*part_ld + m]
-  float* part;
-  int64_t part_ld;
+  // forward / dgrad: A rows are features m (M of them), B rows the batch (N = B of them)
+  float* part;              // split partials, part[((split*P + p)*N + n)*M + m]
+  int* counters;            // one per (p, m_tile); zero between launches
+  float* bias_rep;          // fp32 masters; the bias this kernel reads (forward) or steps (dgrad,
+  int64_t bias_off;         // last layer) is at bias_rep[p*rep_stride + bias_off + m]
+  __nv_bfloat16* out_bm;    // [P, B, M]  relu(z) (forward) or dZ (dgrad)
+  __nv_bfloat16* out_mb;    // [P, M, B]  the same, transposed
+  const __nv_bfloat16* mask_mb;  // dgrad: forward activation [P, M, B] whose sign gates dZ
+  // last layer (M = classes <= 32): loss, dZ_L and the bias step
+  const int32_t* labels;    // [P*B]
+  float* loss_out;          // loss_out[p*loss_stride]
+  int loss_stride;
+  __nv_bfloat16* dz_bm;     // [P, B, cpad]
+  int cpad;
+  __nv_bfloat16* dz_mb;     // [P, M, B]
   // EPI_WGRAD_SGD: A rows are output features o, B rows input features i
   float* rep;               // fp32 masters, W[o, i] at rep[p*rep_stride + w_off + o*in + i]
   int64_t rep_stride, w_off;
@@ -58,6 +73,29 @@ struct TcArgs {
   int* status;
 };
 
+// Synchronises the 8 epilogue warps (256 threads) without the producer and MMA warps.
+__device__ __forceinline__ void epilogue_barrier() {
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+}
+
+// 32 accumulator columns starting at c0 for this warp's 32 lanes (16 when the tile ends there;
+// the rest reads as zero).  Returns the number of valid columns.  Warp-collective.
+__device__ __forceinline__ int load_acc_chunk(uint32_t lane_addr, int c0, int BN, float (&z)[32]) {
+  uint32_t r[32];
+  if (c0 + 32 <= BN) {
+    tmem_ld_32x32(lane_addr + (uint32_t)c0, r);
+  } else {                                   // BN is a multiple of 16
+    uint32_t h[16];
+    tmem_ld_16cols(lane_addr + (uint32_t)c0, h);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) { r[j] = h[j]; r[16 + j] = 0u; }
+  }
+  tmem_ld_wait();
+#pragma unroll
+  for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(r[j]);
+  return min(32, BN - c0);
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kThreads)
 k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -68,6 +106,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   __shared__ __align__(8) uint64_t acc_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ int last_flag;
+  __shared__ float colsum[2][kBM];
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~(uintptr_t)1023);
@@ -157,37 +197,19 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const int row = q * 32 + lane;
     const bool ok = mbar_wait(&acc_bar, 0, abortp, g.status, ERR_EPILOGUE);
     tc_fence_after_sync();
-    if (ok) {
-      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      float* stage = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes) + ew * (32 * 33);
-      for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
-        uint32_t r[32];
-        if (c0 + 32 <= g.BN) {
-          tmem_ld_32x32(lane_addr + (uint32_t)c0, r);
-        } else {                             // BN is a multiple of 16
-          uint32_t h[16];
-          tmem_ld_16cols(lane_addr + (uint32_t)c0, h);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) { r[j] = h[j]; r[16 + j] = 0u; }
-        }
-        tmem_ld_wait();
-        const int ncols = min(32, g.BN - c0);
-        if (EPI == EPI_PARTIAL) {
-          const int m = m0 + row;
-          if (m < g.M) {
-            float* dst = g.part + ((size_t)(split * g.P + p) * g.N) * g.part_ld + m;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int n = n0 + c0 + j;
-              if (j < ncols && n < g.N) dst[(size_t)n * g.part_ld] = __uint_as_float(r[j]);
-            }
-          }
-        } else {
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    if (EPI == EPI_WGRAD_SGD) {
+      if (ok) {
+        float* stage =
+            reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes) + ew * (32 * 33);
+        for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+          float z[32];
+          const int ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
           // The accumulator arrives with one weight row per lane.  It is turned through shared
           // memory so that the lanes of a warp walk along a row: every access to the fp32 masters
           // and to the [out, in] bf16 copy is then a contiguous 128 / 64 bytes per row.
 #pragma unroll
-          for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(r[j]);
+          for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = z[j];
           __syncwarp();
           const int o_base = m0 + q * 32;
           const int i = n0 + c0 + lane;
@@ -195,18 +217,30 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           float* wcol = g.rep + (size_t)p * g.rep_stride + g.w_off + (size_t)o_base * g.in + i;
           __nv_bfloat16* hcol =
               g.w16 + (size_t)p * g.w16_stride + g.sh_off + (size_t)o_base * g.in + i;
+          const int rows_valid = min(32, g.out - o_base);   // uniform over the warp
           float wv[32];
+          if (rows_valid == 32) {
+            // interior tile: 32 independent loads in flight before the first use
+            if (col_ok) {
 #pragma unroll
-          for (int rr = 0; rr < 32; ++rr)
-            wv[rr] = (col_ok && o_base + rr < g.out) ? wcol[(size_t)rr * g.in] : 0.f;
+              for (int rr = 0; rr < 32; ++rr) wv[rr] = __ldcs(wcol + (size_t)rr * g.in);
 #pragma unroll
-          for (int rr = 0; rr < 32; ++rr) {
-            const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
-            if (col_ok && o_base + rr < g.out) {
-              wcol[(size_t)rr * g.in] = w;
-              hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
+              for (int rr = 0; rr < 32; ++rr) {
+                const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
+                wcol[(size_t)rr * g.in] = w;
+                hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
+                stage[rr * 33 + lane] = w;
+              }
             }
-            stage[rr * 33 + lane] = w;
+          } else {
+            for (int rr = 0; rr < rows_valid; ++rr) {
+              if (col_ok) {
+                const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wcol[(size_t)rr * g.in]);
+                wcol[(size_t)rr * g.in] = w;
+                hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
+                stage[rr * 33 + lane] = w;
+              }
+            }
           }
           __syncwarp();
           if (g.wt16) {                       // [in, out] copy: lanes walk along out again
@@ -224,101 +258,170 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           __syncwarp();
         }
       }
+    } else {
+      // forward / dgrad: feature m per lane, the batch along the columns (n0 == 0, BN >= N)
+      const int m = m0 + row;
+      const bool m_ok = m < g.M;
+      bool finisher = ok;
+      if (g.splits > 1) {
+        if (ok) {
+          float* dst = g.part + ((size_t)(split * g.P + p) * g.N) * g.M + m;
+          for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+            float z[32];
+            const int ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
+            if (m_ok) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols && c0 + j < g.N) dst[(size_t)(c0 + j) * g.M] = z[j];
+            }
+          }
+        }
+        // the block that publishes the last of the `splits` partials of this tile finishes it
+        __threadfence();
+        epilogue_barrier();
+        if (ew == 0 && lane == 0) {
+          int* ctr = g.counters + p * g.m_tiles + m_tile;
+          const int old = ok ? atomicAdd(ctr, 1) : -1;
+          const int last = old == g.splits - 1;
+          if (last) *ctr = 0;
+          __threadfence();
+          last_flag = last;
+        }
+        epilogue_barrier();
+        finisher = last_flag != 0;
+      }
+      if (finisher) {
+        float* bias = g.bias_rep + (size_t)p * g.rep_stride + g.bias_off;
+        const float my_bias = (EPI != EPI_DGRAD && m_ok) ? bias[m] : 0.f;
+        float dsum = 0.f;
+        float* lg = reinterpret_cast<float*>(smem);          // last layer: logits [N][M]
+        for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+          float z[32];
+          int ncols;
+          if (g.splits == 1) {
+            ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
+          } else {
+            ncols = min(32, g.BN - c0);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = 0.f;
+            if (m_ok) {
+              const int nvalid = min(ncols, g.N - c0);
+              for (int sp = 0; sp < g.splits; ++sp) {        // ascending split order
+                const float* src = g.part + ((size_t)(sp * g.P + p) * g.N + c0) * g.M + m;
+                float t[32];
+                if (nvalid == 32) {                          // all loads in flight together
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * g.M);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j)
+                    t[j] = __ldcg(src + (size_t)min(j, max(nvalid - 1, 0)) * g.M);
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) z[j] += j < nvalid ? t[j] : 0.f;
+              }
+            }
+          }
+          if (EPI == EPI_FWD_LAST) {
+            if (m_ok) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols && c0 + j < g.N) lg[(c0 + j) * g.M + m] = z[j] + my_bias;
+            }
+          } else {
+            uint32_t hp[16];                                  // 32 bf16 results, packed
+            if (EPI == EPI_DGRAD) {
+              uint4 mk[4];
+              const uint4* msrc = reinterpret_cast<const uint4*>(
+                  g.mask_mb + ((size_t)p * g.M + (m_ok ? m : 0)) * g.N + c0);
+#pragma unroll
+              for (int v = 0; v < 4; ++v)
+                mk[v] = (m_ok && v * 8 < ncols && c0 + v * 8 < g.N) ? msrc[v]
+                                                                    : make_uint4(0, 0, 0, 0);
+              const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(mk);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const bool live = j < ncols && c0 + j < g.N && __bfloat162float(mh[j]) > 0.f;
+                z[j] = live ? z[j] : 0.f;                     // ReLU'(0) = 0
+                dsum += z[j];
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float a = z[j] + my_bias;
+                z[j] = a > 0.f ? a : 0.f;
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(z[2 * j], z[2 * j + 1]);
+              hp[j] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            if (m_ok) {
+              const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
+              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + c0) * g.M + m;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols && c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
+              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + c0);
+#pragma unroll
+              for (int v = 0; v < 4; ++v)
+                if (v * 8 < ncols && c0 + v * 8 < g.N)
+                  dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
+            }
+          }
+        }
+        if (EPI == EPI_DGRAD) {
+          // bias step of the layer below: b[m] -= gamma * sum_b dZ[b, m]; the two warps that
+          // share a row add their column sums in a fixed order
+          colsum[half][row] = dsum;
+          epilogue_barrier();
+          if (half == 0 && m_ok)
+            bias[m] = fmaf(-g.gamma, colsum[0][row] + colsum[1][row], bias[m]);
+        }
+        if (EPI == EPI_FWD_LAST) {
+          // softmax cross-entropy on the block's [N, M] logits: thread t takes batch row t
+          float* dzs = lg + g.N * g.M;
+          float* lossp = dzs + g.N * g.M;
+          epilogue_barrier();
+          const int t = ew * 32 + lane;
+          const int C = g.M;
+          if (t < g.N) {
+            const float* zr = lg + t * C;
+            float mx = zr[0];
+            for (int c = 1; c < C; ++c) mx = fmaxf(mx, zr[c]);
+            float se = 0.f;
+            for (int c = 0; c < C; ++c) se += expf(zr[c] - mx);
+            const float lse = mx + logf(se);
+            const int yb = g.labels[(size_t)p * g.N + t];
+            lossp[t] = lse - zr[yb];
+            const float inv_b = 1.0f / (float)g.N;
+            for (int c = 0; c < C; ++c) {
+              const float gr = (expf(zr[c] - lse) - (c == yb ? 1.f : 0.f)) * inv_b;
+              dzs[t * C + c] = gr;
+              const __nv_bfloat16 gq = __float2bfloat16_rn(gr);
+              g.dz_bm[((size_t)p * g.N + t) * g.cpad + c] = gq;
+              g.dz_mb[((size_t)p * C + c) * g.N + t] = gq;
+            }
+          }
+          epilogue_barrier();
+          if (t == 0) {
+            float sl = 0.f;
+            for (int b = 0; b < g.N; ++b) sl += lossp[b];
+            g.loss_out[(size_t)p * g.loss_stride] = sl / (float)g.N;
+          }
+          if (t < C) {
+            float sb = 0.f;
+            for (int b = 0; b < g.N; ++b) sb += dzs[b * C + t];
+            bias[t] = fmaf(-g.gamma, sb, bias[t]);
+          }
+        }
+      }
     }
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, g.tmem_cols);
-}
-
-// ------------------------------------------------------------------------------ finishing kernels
-// Forward: z = sum_s part_s + bias;  hidden layers store relu(z) as bf16 in both orientations,
-// the last layer stores fp32 logits.  grid (ceil(out/32), ceil(B/32), P), block (32, 8).
-template <bool LAST>
-__global__ void __launch_bounds__(256)
-k_fwd_finish(const float* __restrict__ part, int S, int P, int B, int out,
-             const float* __restrict__ rep, int64_t rep_stride, int64_t b_off,
-             __nv_bfloat16* __restrict__ act, __nv_bfloat16* __restrict__ act_t,
-             float* __restrict__ logits) {
-  __shared__ __nv_bfloat16 tile[32][33];
-  const int p = blockIdx.z, o0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
-  const int tx = threadIdx.x, ty = threadIdx.y;
-  const int o = o0 + tx;
-  const float bias = o < out ? rep[(size_t)p * rep_stride + b_off + o] : 0.f;
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int b = b0 + ty + 8 * r;
-    if (o < out && b < B) {
-      float z = 0.f;
-      for (int s = 0; s < S; ++s) z += part[((size_t)(s * P + p) * B + b) * out + o];
-      z += bias;
-      if (LAST) {
-        logits[((size_t)p * B + b) * out + o] = z;
-      } else {
-        __nv_bfloat16 a = __float2bfloat16_rn(z > 0.f ? z : 0.f);
-        act[((size_t)p * B + b) * out + o] = a;
-        tile[ty + 8 * r][tx] = a;
-      }
-    }
-  }
-  if (!LAST) {
-    __syncthreads();
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int oo = o0 + ty + 8 * r, b = b0 + tx;
-      if (oo < out && b < B) act_t[((size_t)p * out + oo) * B + b] = tile[tx][ty + 8 * r];
-    }
-  }
-}
-
-// dgrad: dA = sum_s part_s;  dZ = dA where the forward activation was positive, else 0
-// (ReLU'(0) = 0); stores dZ as bf16 in both orientations and takes the bias step of the layer
-// that produced the activation:  b[f] -= gamma * sum_b dZ[b, f]  (unrounded dZ, fixed order).
-// grid (ceil(feat/32), P), block (32, 8).
-__global__ void __launch_bounds__(256)
-k_dgrad_finish(const float* __restrict__ part, int S, int P, int B, int feat,
-               const __nv_bfloat16* __restrict__ act, __nv_bfloat16* __restrict__ dz,
-               __nv_bfloat16* __restrict__ dz_t, float* __restrict__ rep, int64_t rep_stride,
-               int64_t b_off, float gamma) {
-  __shared__ __nv_bfloat16 tile[32][33];
-  __shared__ float red[8][32];
-  const int p = blockIdx.y, f0 = blockIdx.x * 32;
-  const int tx = threadIdx.x, ty = threadIdx.y;
-  const int f = f0 + tx;
-  float acc = 0.f;
-  for (int bc = 0; bc < B; bc += 32) {
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int b = bc + ty + 8 * r;
-      __nv_bfloat16 q = __float2bfloat16_rn(0.f);
-      if (f < feat && b < B) {
-        float d = 0.f;
-        for (int s = 0; s < S; ++s) d += part[((size_t)(s * P + p) * B + b) * feat + f];
-        const size_t at = ((size_t)p * B + b) * feat + f;
-        d = __bfloat162float(act[at]) > 0.f ? d : 0.f;
-        acc += d;
-        q = __float2bfloat16_rn(d);
-        dz[at] = q;
-      }
-      tile[ty + 8 * r][tx] = q;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int ff = f0 + ty + 8 * r, b = bc + tx;
-      if (ff < feat && b < B) dz_t[((size_t)p * feat + ff) * B + b] = tile[tx][ty + 8 * r];
-    }
-    __syncthreads();
-  }
-  red[ty][tx] = acc;
-  __syncthreads();
-  if (ty == 0 && f < feat) {
-    float s = 0.f;
-#pragma unroll
-    for (int r = 0; r < 8; ++r) s += red[r][tx];
-    float* bias = rep + (size_t)p * rep_stride + b_off;
-    bias[f] = fmaf(-gamma, s, bias[f]);
-  }
 }
 
 // bf16 copies of the global model w~ (shared by all learners at the first step of a round, when
@@ -348,11 +451,11 @@ struct TcLayout {
   int64_t n16, nt16;                         // elements per bf16 copy row
   int64_t sh_off[MAVG_MAX_LAYERS], sht_off[MAVG_MAX_LAYERS];
   int out_pad[MAVG_MAX_LAYERS];
-  size_t xg, xt;
+  size_t xg[2], xt[2];                       // gathered batch, two buffers used by alternate steps
   size_t act[MAVG_MAX_LAYERS + 1], act_t[MAVG_MAX_LAYERS + 1];
   size_t dz[MAVG_MAX_LAYERS + 1], dz_t[MAVG_MAX_LAYERS + 1];
-  size_t logits, dz_last;
   size_t part, part_bytes;
+  size_t counters, counters_bytes;
   size_t w16, wt16, w16g, wt16g;
   size_t end;
 };
@@ -412,8 +515,11 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.nt16 = ot16 > 0 ? ot16 : 64;
   size_t off = up(base, 1024);
   auto take = [&](size_t bytes) { size_t r = off; off = up(off + bytes, 1024); return r; };
-  t.xg = take(rows * cfg->dims[0] * 2);
-  t.xt = take(rows * cfg->dims[0] * 2);
+  for (int i = 0; i < 2; ++i) {
+    t.xg[i] = take(rows * cfg->dims[0] * 2);
+    t.xt[i] = take(rows * cfg->dims[0] * 2);
+  }
+  int max_m_tiles = 1;
   for (int l = 1; l <= L; ++l) {
     const int d = cfg->dims[l];
     if (l < L) {
@@ -424,20 +530,21 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
       t.dz[l] = take(rows * t.cpad * 2);
     }
     t.dz_t[l] = take(rows * d * 2);
+    max_m_tiles = std::max(max_m_tiles, (d + kBM - 1) / kBM);
   }
-  t.logits = take(rows * cfg->dims[L] * 4);
-  t.dz_last = take(rows * cfg->dims[L] * 4);
-  size_t pb = 0;
+  size_t pb = 1024;
   for (int l = 1; l <= L; ++l) {
     GemmPlan f = plan_partial(cfg->dims[l], B, cfg->dims[l - 1], P, sm_count);
-    pb = std::max(pb, (size_t)f.splits * rows * cfg->dims[l] * 4);
+    if (f.splits > 1) pb = std::max(pb, (size_t)f.splits * rows * cfg->dims[l] * 4);
     if (l > 1) {
       GemmPlan d = plan_partial(cfg->dims[l - 1], B, cfg->dims[l], P, sm_count);
-      pb = std::max(pb, (size_t)d.splits * rows * cfg->dims[l - 1] * 4);
+      if (d.splits > 1) pb = std::max(pb, (size_t)d.splits * rows * cfg->dims[l - 1] * 4);
     }
   }
   t.part_bytes = pb;
   t.part = take(pb);
+  t.counters_bytes = (size_t)P * max_m_tiles * sizeof(int);
+  t.counters = take(t.counters_bytes);
   t.w16 = take((size_t)P * t.n16 * 2);
   t.wt16 = take((size_t)P * t.nt16 * 2);
   t.w16g = take((size_t)t.n16 * 2);
@@ -461,11 +568,16 @@ struct TcState {
   // per layer l = 1..L (index l)
   CUtensorMap w[MAVG_MAX_LAYERS + 1], wg[MAVG_MAX_LAYERS + 1];       // [out, in] copies
   CUtensorMap wt[MAVG_MAX_LAYERS + 1], wtg[MAVG_MAX_LAYERS + 1];     // [in, out] copies (l >= 2)
-  CUtensorMap act_in[MAVG_MAX_LAYERS + 1];    // [B, d_{l-1}] input activations of layer l
+  CUtensorMap act_in[MAVG_MAX_LAYERS + 1];    // [B, d_{l-1}] input activations of layer l >= 2
   CUtensorMap act_in_t[MAVG_MAX_LAYERS + 1];  // [d_{l-1}, B]
+  CUtensorMap x_in[2], x_in_t[2];             // layer 1's input: the two gather buffers
   CUtensorMap dz[MAVG_MAX_LAYERS + 1];        // [B, d_l]
   CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1], wgrad[MAVG_MAX_LAYERS + 1];
+  // side streams and events for the branches of a step that may overlap
+  cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,
+              ev_x_free[2] = {nullptr, nullptr};
 };
 
 // bf16 tensor [batch, rows, inner] with the given strides (in elements); box = 64 x box_rows.
@@ -489,6 +601,7 @@ template <int EPI>
 cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtensorMap& b,
                         const GemmPlan& pl, TcArgs g) {
   g.BN = pl.BN;
+  g.m_tiles = pl.m_tiles;
   g.n_tiles = pl.n_tiles;
   g.splits = pl.splits;
   g.kb_per_split = pl.kb_per_split;
@@ -496,9 +609,14 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   g.stages = pl.stages;
   g.tmem_cols = pl.tmem_cols;
   g.P = c->cfg.P;
+  g.rep_stride = c->buf.replica_stride;
+  g.gamma = c->cfg.local_lr;
   g.status = (int*)ws_ptr(c, c->ws.status);
-  const size_t smem = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2) + 1024 +
-                      (EPI == EPI_WGRAD_SGD ? kStageBytes : 0);
+  size_t pipe = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2);
+  size_t smem = pipe + 1024;
+  if (EPI == EPI_WGRAD_SGD) smem += kStageBytes;
+  if (EPI == EPI_FWD_LAST)   // the loss tail reuses the pipeline buffers: logits, dZ, row losses
+    smem = std::max(pipe, ((size_t)2 * g.N * g.M + g.N) * sizeof(float)) + 1024;
   dim3 grid((unsigned)(pl.m_tiles * pl.n_tiles * pl.splits), (unsigned)c->cfg.P);
   prof_begin(c, cls);
   k_tc_gemm<EPI><<<grid, kThreads, smem, c->stream>>>(a, b, g);
@@ -518,6 +636,10 @@ bool tc_shapes_ok(const mavg_config* cfg, std::string* why) {
       if (why) *why = "the tensor-core path needs every layer's input width to be a multiple of 8";
       return false;
     }
+  if (cfg->dims[cfg->n_layers] > 32) {
+    if (why) *why = "the tensor-core path needs at most 32 classes";
+    return false;
+  }
   return true;
 }
 
@@ -555,12 +677,19 @@ mavg_status tc_setup(mavg_ctx* c) {
     __nv_bfloat16* w16g = (__nv_bfloat16*)bf(t.w16g) + t.sh_off[l - 1];
     ok = ok && encode_map(st, &st->w[l], w16, in, out, P, in, t.n16, kBM, &why);
     ok = ok && encode_map(st, &st->wg[l], w16g, in, out, 1, in, t.n16, kBM, &why);
-    void* a_in = l == 1 ? bf(t.xg) : bf(t.act[l - 1]);
-    void* a_in_t = l == 1 ? bf(t.xt) : bf(t.act_t[l - 1]);
-    ok = ok && encode_map(st, &st->act_in[l], a_in, in, B, P, in, (int64_t)B * in,
-                          st->fwd[l].BN, &why);
-    ok = ok && encode_map(st, &st->act_in_t[l], a_in_t, B, in, P, B, (int64_t)B * in,
-                          st->wgrad[l].BN, &why);
+    if (l == 1) {
+      for (int i = 0; i < 2 && ok; ++i) {
+        ok = ok && encode_map(st, &st->x_in[i], bf(t.xg[i]), in, B, P, in, (int64_t)B * in,
+                              st->fwd[l].BN, &why);
+        ok = ok && encode_map(st, &st->x_in_t[i], bf(t.xt[i]), B, in, P, B, (int64_t)B * in,
+                              st->wgrad[l].BN, &why);
+      }
+    } else {
+      ok = ok && encode_map(st, &st->act_in[l], bf(t.act[l - 1]), in, B, P, in, (int64_t)B * in,
+                            st->fwd[l].BN, &why);
+      ok = ok && encode_map(st, &st->act_in_t[l], bf(t.act_t[l - 1]), B, in, P, B,
+                            (int64_t)B * in, st->wgrad[l].BN, &why);
+    }
     ok = ok && encode_map(st, &st->dz_t[l], bf(t.dz_t[l]), B, out, P, B, (int64_t)B * out, kBM,
                           &why);
     if (l > 1) {
@@ -577,15 +706,29 @@ mavg_status tc_setup(mavg_ctx* c) {
     c->err = why;
     return MAVG_ERR_CUDA;
   }
-  // 227 KB per block in all, of which a few hundred bytes are the kernel's static barriers
-  constexpr int kMaxDynSmem = 226 * 1024;
-  e = cudaFuncSetAttribute(k_tc_gemm<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  // 227 KB per block in all, of which a few hundred bytes are the kernel's static variables
+  constexpr int kMaxDynSmem = 225 * 1024;
+  e = cudaFuncSetAttribute(k_tc_gemm<EPI_FWD_HIDDEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kMaxDynSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_tc_gemm<EPI_FWD_LAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kMaxDynSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_tc_gemm<EPI_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kMaxDynSmem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_tc_gemm<EPI_WGRAD_SGD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kMaxDynSmem);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);
+  cudaEvent_t* evs[] = {&st->ev_fork, &st->ev_wgrad_done, &st->ev_gather_done, &st->ev_x_free[0],
+                        &st->ev_x_free[1]};
+  for (cudaEvent_t* ev : evs)
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(ws + t.counters, 0, t.counters_bytes, c->stream);
   if (e != cudaSuccess) {
-    c->err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
+    c->err = std::string("tensor-core path set-up: ") + cudaGetErrorString(e);
     cudaGetLastError();   // reported here; do not leave it pending for a later call
     return MAVG_ERR_CUDA;
   }
@@ -593,7 +736,16 @@ mavg_status tc_setup(mavg_ctx* c) {
 }
 
 void tc_teardown(mavg_ctx* c) {
-  delete (TcState*)c->mlp;
+  TcState* st = (TcState*)c->mlp;
+  if (st) {
+    if (st->s_wgrad) cudaStreamDestroy(st->s_wgrad);
+    if (st->s_gather) cudaStreamDestroy(st->s_gather);
+    cudaEvent_t evs[] = {st->ev_fork, st->ev_wgrad_done, st->ev_gather_done, st->ev_x_free[0],
+                         st->ev_x_free[1]};
+    for (cudaEvent_t ev : evs)
+      if (ev) cudaEventDestroy(ev);
+  }
+  delete st;
   c->mlp = nullptr;
 }
 
@@ -616,52 +768,74 @@ cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
   return cudaSuccess;
 }
 
+// One local step of all learners.  Dependencies inside a step:
+//   gather -> fwd_1 -> ... -> fwd_L (+loss) -> dgrad_L -> ... -> dgrad_2 -> wgrad_1
+//   wgrad_l (l >= 2) needs dZ_l and must follow dgrad_l, which still reads W_l; it does not feed
+//   anything else of this step, so it runs on a side stream beside the rest of the chain.
+//   The gather of the next step touches no weights; it runs on a second side stream into the
+//   other of two batch buffers as soon as that buffer's last reader (wgrad_1 of the step before
+//   last) is done.
+// With `overlap` false (profiled runs) everything is issued in order on the main stream.
 cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   TcState* st = (TcState*)c->mlp;
   const TcLayout& t = st->lay;
   const mavg_config& cfg = c->cfg;
-  const int P = cfg.P, B = cfg.B, L = cfg.n_layers;
+  const int B = cfg.B, L = cfg.n_layers, K = cfg.K;
   char* ws = (char*)c->buf.workspace;
   auto bfp = [&](size_t off) { return (__nv_bfloat16*)(ws + off); };
   int32_t* idx = (int32_t*)ws_ptr(c, c->ws.idx);
   int32_t* labels = (int32_t*)ws_ptr(c, c->ws.labels);
   float* losses = (float*)ws_ptr(c, c->ws.losses);
   float* part = (float*)(ws + t.part);
-  float* logits = (float*)(ws + t.logits);
-  float* dz_last = (float*)(ws + t.dz_last);
+  int* counters = (int*)(ws + t.counters);
   const bool shared_w = c->replicas_equal_global;   // first step after a (re-)broadcast
+  const bool overlap = !c->profiling;
+  const int xb = step & 1;                          // batch buffer of this step
+  cudaStream_t main_s = c->stream;
   cudaError_t e;
-  if ((e = launch_batch_indices(c, round, step, 0, P, idx, labels)) != cudaSuccess) return e;
-  if ((e = launch_gather(c, idx, 1, nullptr, bfp(t.xg), bfp(t.xt))) != cudaSuccess) return e;
+#define TC_TRY(call) do { if ((e = (call)) != cudaSuccess) { c->stream = main_s; return e; } } while (0)
+
+  // labels and indices are per step as well: they live beside the batch buffer they belong to
+  int32_t* idx_b = idx;
+  int32_t* labels_b = labels;
+  if (step == 1 || !overlap) {
+    TC_TRY(launch_sample_gather(c, round, step, idx_b, labels_b, bfp(t.xg[xb]), bfp(t.xt[xb])));
+  } else {
+    // issued during the previous step on the gather stream
+    TC_TRY(cudaStreamWaitEvent(main_s, st->ev_gather_done, 0));
+  }
 
   for (int l = 1; l <= L; ++l) {
     const MlpLayer& ly = c->layers[l - 1];
     TcArgs g{};
     g.M = ly.out; g.N = B;
     g.a_batched = shared_w ? 0 : 1; g.b_batched = 1;
-    g.part = part; g.part_ld = ly.out;
-    if ((e = launch_gemm<EPI_PARTIAL>(c, MAVG_K_FWD, shared_w ? st->wg[l] : st->w[l],
-                                      st->act_in[l], st->fwd[l], g)) != cudaSuccess)
-      return e;
-    dim3 grid((ly.out + 31) / 32, (B + 31) / 32, P), block(32, 8);
-    prof_begin(c, MAVG_K_FWD);
-    if (l < L)
-      k_fwd_finish<false><<<grid, block, 0, c->stream>>>(part, st->fwd[l].splits, P, B, ly.out,
-                                                         c->buf.replicas, c->buf.replica_stride,
-                                                         ly.b_off, bfp(t.act[l]), bfp(t.act_t[l]),
-                                                         nullptr);
-    else
-      k_fwd_finish<true><<<grid, block, 0, c->stream>>>(part, st->fwd[l].splits, P, B, ly.out,
-                                                        c->buf.replicas, c->buf.replica_stride,
-                                                        ly.b_off, nullptr, nullptr, logits);
-    prof_end(c);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    g.part = part; g.counters = counters;
+    g.bias_rep = c->buf.replicas; g.bias_off = ly.b_off;
+    const CUtensorMap& wm = shared_w ? st->wg[l] : st->w[l];
+    const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
+    if (l < L) {
+      g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
+      TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
+    } else {
+      g.labels = labels_b; g.loss_out = losses + (step - 1); g.loss_stride = K;
+      g.dz_bm = bfp(t.dz[L]); g.cpad = t.cpad; g.dz_mb = bfp(t.dz_t[L]);
+      TC_TRY(launch_gemm<EPI_FWD_LAST>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
+    }
   }
-  const int C = cfg.dims[L];
-  if ((e = launch_softmax_ce(c, logits, C, labels, losses + (step - 1), cfg.K, dz_last, C,
-                             bfp(t.dz[L]), t.cpad, bfp(t.dz_t[L]), B, true)) != cudaSuccess)
-    return e;
+  // the labels of this step have been consumed: the next step's gather may run now
+  if (overlap && step < K) {
+    const int nb = (step + 1) & 1;
+    TC_TRY(cudaEventRecord(st->ev_fork, main_s));
+    TC_TRY(cudaStreamWaitEvent(st->s_gather, st->ev_fork, 0));
+    if (step >= 2) TC_TRY(cudaStreamWaitEvent(st->s_gather, st->ev_x_free[nb], 0));
+    c->stream = st->s_gather;
+    TC_TRY(launch_sample_gather(c, round, step + 1, idx_b, labels_b, bfp(t.xg[nb]), bfp(t.xt[nb])));
+    c->stream = main_s;
+    TC_TRY(cudaEventRecord(st->ev_gather_done, st->s_gather));
+  }
 
+  bool side_used = false;
   for (int l = L; l >= 1; --l) {
     const MlpLayer& ly = c->layers[l - 1];
     if (l > 1) {
@@ -669,33 +843,41 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TcArgs g{};
       g.M = ly.in; g.N = B;
       g.a_batched = shared_w ? 0 : 1; g.b_batched = 1;
-      g.part = part; g.part_ld = ly.in;
-      if ((e = launch_gemm<EPI_PARTIAL>(c, MAVG_K_DGRAD, shared_w ? st->wtg[l] : st->wt[l],
-                                        st->dz[l], st->dgrad[l], g)) != cudaSuccess)
-        return e;
-      dim3 grid((ly.in + 31) / 32, P), block(32, 8);
-      prof_begin(c, MAVG_K_DGRAD);
-      k_dgrad_finish<<<grid, block, 0, c->stream>>>(part, st->dgrad[l].splits, P, B, ly.in,
-                                                    bfp(t.act[l - 1]), bfp(t.dz[l - 1]),
-                                                    bfp(t.dz_t[l - 1]), c->buf.replicas,
-                                                    c->buf.replica_stride, below.b_off,
-                                                    cfg.local_lr);
-      prof_end(c);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      g.part = part; g.counters = counters;
+      g.bias_rep = c->buf.replicas; g.bias_off = below.b_off;
+      g.out_bm = bfp(t.dz[l - 1]); g.out_mb = bfp(t.dz_t[l - 1]);
+      g.mask_mb = bfp(t.act_t[l - 1]);
+      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wtg[l] : st->wt[l], st->dz[l],
+                                    st->dgrad[l], g));
     }
     TcArgs g{};
     g.M = ly.out; g.N = ly.in;
     g.a_batched = 1; g.b_batched = 1;
-    g.rep = c->buf.replicas; g.rep_stride = c->buf.replica_stride; g.w_off = ly.w_off;
+    g.rep = c->buf.replicas; g.w_off = ly.w_off;
     g.in = ly.in; g.out = ly.out;
     g.w16 = bfp(t.w16); g.w16_stride = t.n16; g.sh_off = t.sh_off[l - 1];
     g.wt16 = l > 1 ? bfp(t.wt16) : nullptr; g.wt16_stride = t.nt16; g.sht_off = t.sht_off[l - 1];
     g.out_pad = t.out_pad[l - 1];
-    g.gamma = cfg.local_lr;
-    if ((e = launch_gemm<EPI_WGRAD_SGD>(c, MAVG_K_WGRAD_SGD, st->dz_t[l], st->act_in_t[l],
-                                        st->wgrad[l], g)) != cudaSuccess)
-      return e;
+    const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
+    if (overlap && l > 1) {
+      TC_TRY(cudaEventRecord(st->ev_fork, main_s));
+      TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
+      c->stream = st->s_wgrad;
+      TC_TRY(launch_gemm<EPI_WGRAD_SGD>(c, MAVG_K_WGRAD_SGD, st->dz_t[l], bm, st->wgrad[l], g));
+      c->stream = main_s;
+      side_used = true;
+    } else {
+      TC_TRY(launch_gemm<EPI_WGRAD_SGD>(c, MAVG_K_WGRAD_SGD, st->dz_t[l], bm, st->wgrad[l], g));
+    }
   }
+  if (overlap) {
+    TC_TRY(cudaEventRecord(st->ev_x_free[xb], main_s));     // wgrad_1 was the buffer's last reader
+    if (side_used) {
+      TC_TRY(cudaEventRecord(st->ev_wgrad_done, st->s_wgrad));
+      TC_TRY(cudaStreamWaitEvent(main_s, st->ev_wgrad_done, 0));
+    }
+  }
+#undef TC_TRY
   return cudaSuccess;
 }
 

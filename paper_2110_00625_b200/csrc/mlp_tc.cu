@@ -259,7 +259,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
       }
     } else {
-      // forward / dgrad: feature m per lane, the batch along the columns (n0 == 0, BN >= N)
+      // forward / dgrad: feature m per lane, the batch along the columns (the dgrad and last-layer
+      // tails need the whole batch in one tile: n_tiles == 1 there)
       const int m = m0 + row;
       const bool m_ok = m < g.M;
       bool finisher = ok;
@@ -272,7 +273,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             if (m_ok) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (j < ncols && c0 + j < g.N) dst[(size_t)(c0 + j) * g.M] = z[j];
+                if (j < ncols && n0 + c0 + j < g.N) dst[(size_t)(n0 + c0 + j) * g.M] = z[j];
             }
           }
         }
@@ -280,7 +281,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __threadfence();
         epilogue_barrier();
         if (ew == 0 && lane == 0) {
-          int* ctr = g.counters + p * g.m_tiles + m_tile;
+          int* ctr = g.counters + (p * g.m_tiles + m_tile) * g.n_tiles + n_tile;
           const int old = ok ? atomicAdd(ctr, 1) : -1;
           const int last = old == g.splits - 1;
           if (last) *ctr = 0;
@@ -305,9 +306,10 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 #pragma unroll
             for (int j = 0; j < 32; ++j) z[j] = 0.f;
             if (m_ok) {
-              const int nvalid = min(ncols, g.N - c0);
+              const int nvalid = min(ncols, g.N - n0 - c0);
+#pragma unroll 2
               for (int sp = 0; sp < g.splits; ++sp) {        // ascending split order
-                const float* src = g.part + ((size_t)(sp * g.P + p) * g.N + c0) * g.M + m;
+                const float* src = g.part + ((size_t)(sp * g.P + p) * g.N + n0 + c0) * g.M + m;
                 float t[32];
                 if (nvalid == 32) {                          // all loads in flight together
 #pragma unroll
@@ -326,22 +328,22 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             if (m_ok) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (j < ncols && c0 + j < g.N) lg[(c0 + j) * g.M + m] = z[j] + my_bias;
+                if (j < ncols && n0 + c0 + j < g.N) lg[(n0 + c0 + j) * g.M + m] = z[j] + my_bias;
             }
           } else {
             uint32_t hp[16];                                  // 32 bf16 results, packed
             if (EPI == EPI_DGRAD) {
               uint4 mk[4];
               const uint4* msrc = reinterpret_cast<const uint4*>(
-                  g.mask_mb + ((size_t)p * g.M + (m_ok ? m : 0)) * g.N + c0);
+                  g.mask_mb + ((size_t)p * g.M + (m_ok ? m : 0)) * g.N + n0 + c0);
 #pragma unroll
               for (int v = 0; v < 4; ++v)
-                mk[v] = (m_ok && v * 8 < ncols && c0 + v * 8 < g.N) ? msrc[v]
+                mk[v] = (m_ok && v * 8 < ncols && n0 + c0 + v * 8 < g.N) ? msrc[v]
                                                                     : make_uint4(0, 0, 0, 0);
               const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(mk);
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
-                const bool live = j < ncols && c0 + j < g.N && __bfloat162float(mh[j]) > 0.f;
+                const bool live = j < ncols && n0 + c0 + j < g.N && __bfloat162float(mh[j]) > 0.f;
                 z[j] = live ? z[j] : 0.f;                     // ReLU'(0) = 0
                 dsum += z[j];
               }
@@ -359,14 +361,14 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
             if (m_ok) {
               const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
-              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + c0) * g.M + m;
+              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + c0) * g.M + m;
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (j < ncols && c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
-              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + c0);
+                if (j < ncols && n0 + c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
+              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + c0);
 #pragma unroll
               for (int v = 0; v < 4; ++v)
-                if (v * 8 < ncols && c0 + v * 8 < g.N)
+                if (v * 8 < ncols && n0 + c0 + v * 8 < g.N)
                   dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
             }
           }
@@ -462,15 +464,26 @@ struct TcLayout {
 
 struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages; uint32_t tmem_cols; };
 
-GemmPlan plan_partial(int M, int N, int K, int P, int sm_count) {
+// Forward / dgrad plan.  To fill the GPU the batch may be cut into column tiles (`tile_n`: only
+// the hidden-layer forward can, its tail needs no sum over the batch) and, if blocks are still
+// few and the contraction long, the contraction is split; a block never gets fewer than 8 slabs
+// (512 elements), below which the split's fix-up costs more than it saves.
+GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   GemmPlan g{};
   g.BN = (N + 15) / 16 * 16;
   g.m_tiles = (M + kBM - 1) / kBM;
   g.n_tiles = 1;
   g.nkb = (K + kBK - 1) / kBK;
-  int tiles = g.m_tiles * P;
-  int want = tiles >= sm_count ? 1 : (sm_count + tiles - 1) / tiles;
-  if (want > g.nkb) want = g.nkb;
+  const int enough = sm_count - sm_count / 8;
+  if (tile_n)
+    while (g.m_tiles * g.n_tiles * P < enough && g.BN % 64 == 0) {
+      g.BN /= 2;
+      g.n_tiles *= 2;
+    }
+  int tiles = g.m_tiles * g.n_tiles * P;
+  int want = tiles >= enough ? 1 : (sm_count + tiles - 1) / tiles;
+  if (want > g.nkb / 8) want = g.nkb / 8;
+  if (want < 1) want = 1;
   g.kb_per_split = (g.nkb + want - 1) / want;
   g.splits = (g.nkb + g.kb_per_split - 1) / g.kb_per_split;
   int stage_bytes = kATileBytes + g.BN * kBK * 2;
@@ -530,14 +543,14 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
       t.dz[l] = take(rows * t.cpad * 2);
     }
     t.dz_t[l] = take(rows * d * 2);
-    max_m_tiles = std::max(max_m_tiles, (d + kBM - 1) / kBM);
+    max_m_tiles = std::max(max_m_tiles, 8 * ((d + kBM - 1) / kBM));   // up to 8 column tiles
   }
   size_t pb = 1024;
   for (int l = 1; l <= L; ++l) {
-    GemmPlan f = plan_partial(cfg->dims[l], B, cfg->dims[l - 1], P, sm_count);
+    GemmPlan f = plan_partial(cfg->dims[l], B, cfg->dims[l - 1], P, sm_count, l < L);
     if (f.splits > 1) pb = std::max(pb, (size_t)f.splits * rows * cfg->dims[l] * 4);
     if (l > 1) {
-      GemmPlan d = plan_partial(cfg->dims[l - 1], B, cfg->dims[l], P, sm_count);
+      GemmPlan d = plan_partial(cfg->dims[l - 1], B, cfg->dims[l], P, sm_count, false);
       if (d.splits > 1) pb = std::max(pb, (size_t)d.splits * rows * cfg->dims[l - 1] * 4);
     }
   }
@@ -671,7 +684,7 @@ mavg_status tc_setup(mavg_ctx* c) {
   for (int l = 1; l <= L && ok; ++l) {
     const int in = cfg.dims[l - 1], out = cfg.dims[l];
     const int dz_ld = l < L ? out : t.cpad;
-    st->fwd[l] = plan_partial(out, B, in, P, kPlanSmCount);
+    st->fwd[l] = plan_partial(out, B, in, P, kPlanSmCount, l < L);
     st->wgrad[l] = plan_wgrad(out, in, B);
     __nv_bfloat16* w16 = (__nv_bfloat16*)bf(t.w16) + t.sh_off[l - 1];
     __nv_bfloat16* w16g = (__nv_bfloat16*)bf(t.w16g) + t.sh_off[l - 1];
@@ -693,7 +706,7 @@ mavg_status tc_setup(mavg_ctx* c) {
     ok = ok && encode_map(st, &st->dz_t[l], bf(t.dz_t[l]), B, out, P, B, (int64_t)B * out, kBM,
                           &why);
     if (l > 1) {
-      st->dgrad[l] = plan_partial(in, B, out, P, kPlanSmCount);
+      st->dgrad[l] = plan_partial(in, B, out, P, kPlanSmCount, false);
       __nv_bfloat16* wt16 = (__nv_bfloat16*)bf(t.wt16) + t.sht_off[l - 1];
       __nv_bfloat16* wt16g = (__nv_bfloat16*)bf(t.wt16g) + t.sht_off[l - 1];
       ok = ok && encode_map(st, &st->wt[l], wt16, out, in, P, t.out_pad[l - 1], t.nt16, kBM, &why);

@@ -124,6 +124,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   const int kb1 = min(g.nkb, kb0 + g.kb_per_split);
   const int count = kb1 - kb0;
 
+  grid_launch_dependents();   // the next kernel may begin its own set-up early
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
@@ -144,6 +145,10 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_slot;
+  // Everything above touched only this block's own shared and tensor memory.  When the launch
+  // allowed it, that much ran while the previous kernel of the stream was still finishing; from
+  // here on its results are read, so wait for it to complete (returns at once otherwise).
+  grid_dependency_wait();
   volatile int* abortp = &abort_flag;
 
   if (warp == 0) {
@@ -218,28 +223,21 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           __nv_bfloat16* hcol =
               g.w16 + (size_t)p * g.w16_stride + g.sh_off + (size_t)o_base * g.in + i;
           const int rows_valid = min(32, g.out - o_base);   // uniform over the warp
-          float wv[32];
-          if (rows_valid == 32) {
-            // interior tile: 32 independent loads in flight before the first use
-            if (col_ok) {
+          if (col_ok && rows_valid > 0) {
+            // 32 independent loads in flight before the first use; rows past the matrix repeat
+            // the last valid row's address and are not stored
+            float wv[32];
 #pragma unroll
-              for (int rr = 0; rr < 32; ++rr) wv[rr] = __ldcs(wcol + (size_t)rr * g.in);
+            for (int rr = 0; rr < 32; ++rr)
+              wv[rr] = __ldcs(wcol + (size_t)min(rr, rows_valid - 1) * g.in);
 #pragma unroll
-              for (int rr = 0; rr < 32; ++rr) {
-                const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
+            for (int rr = 0; rr < 32; ++rr) {
+              const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
+              if (rr < rows_valid) {
                 wcol[(size_t)rr * g.in] = w;
                 hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
-                stage[rr * 33 + lane] = w;
               }
-            }
-          } else {
-            for (int rr = 0; rr < rows_valid; ++rr) {
-              if (col_ok) {
-                const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wcol[(size_t)rr * g.in]);
-                wcol[(size_t)rr * g.in] = w;
-                hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
-                stage[rr * 33 + lane] = w;
-              }
+              stage[rr * 33 + lane] = w;
             }
           }
           __syncwarp();
@@ -474,7 +472,7 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   g.m_tiles = (M + kBM - 1) / kBM;
   g.n_tiles = 1;
   g.nkb = (K + kBK - 1) / kBK;
-  const int enough = sm_count - sm_count / 8;
+  const int enough = sm_count - sm_count / 5;   // ~80 % of the SMs busy counts as full
   if (tile_n)
     while (g.m_tiles * g.n_tiles * P < enough && g.BN % 64 == 0) {
       g.BN /= 2;
@@ -631,10 +629,20 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   if (EPI == EPI_FWD_LAST)   // the loss tail reuses the pipeline buffers: logits, dZ, row losses
     smem = std::max(pipe, ((size_t)2 * g.N * g.M + g.N) * sizeof(float)) + 1024;
   dim3 grid((unsigned)(pl.m_tiles * pl.n_tiles * pl.splits), (unsigned)c->cfg.P);
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = grid;
+  lc.blockDim = dim3(kThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
   prof_begin(c, cls);
-  k_tc_gemm<EPI><<<grid, kThreads, smem, c->stream>>>(a, b, g);
+  cudaError_t e = cudaLaunchKernelEx(&lc, k_tc_gemm<EPI>, a, b, g);
   prof_end(c);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

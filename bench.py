@@ -95,9 +95,9 @@ class ClockSampler:
         return out
 
 
-def workload_inputs():
+def workload_inputs(name=None):
     from paper_2110_00625_b200 import workloads as W
-    cfg = dict(W.CONFIGS[WORKLOAD])
+    cfg = dict(W.CONFIGS[name or WORKLOAD])
     x, y = W.make_dataset(cfg)
     w1 = W.mlp_init(cfg["dims"])
     return cfg, x, y, w1
@@ -223,6 +223,41 @@ def meta_update_sweep(m, torch, peaks, reps=5):
     return res
 
 
+def run_pseudograd(args, m, torch, peaks, rank):
+    """Full round at the ResNet-50-sized vector (n = 25.6 M, P = 16) with seeded pseudo-gradients:
+    one line per K with the local pass, the meta-update and the whole round."""
+    from paper_2110_00625_b200 import workloads as W
+    cfg = W.CONFIGS["C5"]
+    n, P = cfg["n"], cfg["P"]
+    w1 = W.global_model(n)
+    out = []
+    for K in cfg["K"]:
+        g = m.Mavg(w1, P=P, K=K, local_lr=cfg["gamma"], mu=0.9, seed=W.BASE_SEED,
+                   objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"])
+        for _ in range(3):
+            g.round()
+        g.sync()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        for a, b, c in ev:
+            a.record(); g.local_steps(); b.record(); g.meta_update(); c.record()
+        torch.cuda.synchronize()
+        loc = statistics.median(a.elapsed_time(b) for a, b, c in ev)
+        met = statistics.median(b.elapsed_time(c) for a, b, c in ev)
+        out.append(dict(K=K, local_ms=loc, meta_ms=met, round_ms=loc + met,
+                        learner_steps_per_s=P * K / ((loc + met) * 1e-3),
+                        local_gbs=8 * P * n / loc / 1e6,
+                        variates_per_s=P * K * n / (loc * 1e-3),
+                        meta_gbs=(8 * P + 16) * n / met / 1e6,
+                        meta_frac_measured=(8 * P + 16) * n / met / 1e6 / peaks["hbm_gbs"]))
+        g.close()
+        del g
+        torch.cuda.empty_cache()
+    if rank == 0:
+        print(json.dumps({"workload": "C5 full round, n=25.6M fp32, P=16, seeded pseudo-gradients",
+                          "steps": args.steps, "results": out}))
+    return 0
+
+
 def run_mavg(args):
     import torch
     import torch.distributed as dist
@@ -237,12 +272,14 @@ def run_mavg(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = measured_peaks()
-    cfg, x, y, w1 = workload_inputs()
+    if args.workload == "C5":
+        return run_pseudograd(args, m, torch, peaks, rank)
+    cfg, x, y, w1 = workload_inputs(args.workload)
 
     # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        k_sample = 4
+        k_sample = 4 if args.workload == "C2" else 1
         rate, threads, times = cpu_oracle_rate(cfg, x, y, w1, k_sample)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"one round cut to {k_sample} of {cfg['K']} local steps on all "
@@ -347,7 +384,8 @@ def run_mavg(args):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if mode else "f32", "data": "synthetic",
-            "config": {"workload": "C2 CIFAR-shaped MLP 3072-512-512-10, P=8, K=8, B=128, mu=0.9, "
+            "config": {"workload": f"{args.workload} CIFAR-shaped MLP {'-'.join(map(str, cfg['dims']))}, "
+                                   f"P={cfg['P']}, K={cfg['K']}, B={cfg['B']}, mu={cfg['mu']}, "
                                    "gamma=0.05, 50000 synthetic samples, labels from a random teacher",
                        "global_batch": cfg["P"] * cfg["B"], "parallelism": "replicas only",
                        "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
@@ -383,6 +421,9 @@ def main():
     ap.add_argument("--impl", default="mavg", choices=["mavg", "reference"])
     ap.add_argument("--gemm", type=int, default=1, choices=[1, 2],
                     help="1: tensor cores (default); 2: CUDA cores with bf16-rounded operands")
+    ap.add_argument("--workload", default="C2", choices=["C2", "C4", "C5"],
+                    help="C2 is the benchmark workload; C4 (large MLP) and C5 (pseudo-gradient "
+                         "round at 25.6 M parameters) print the same measurements for context")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     args = ap.parse_args()

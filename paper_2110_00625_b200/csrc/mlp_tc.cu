@@ -1,5 +1,7 @@
 // Tensor-core MLP learner step: the three matrix products of every layer run on tcgen05 with
-// TMA-fed shared-memory operands and the accumulator in tensor memory.
+// TMA-fed shared-memory operands and the accumulator in tensor memory.  This file holds the
+// forward and dgrad kernel and the schedule of a step; the weight-gradient kernel, which carries
+// the SGD step, is in wgrad_tc.cu.
 //
 // Every product is arranged so that the 128-row MMA dimension is a feature dimension and the
 // batch (16..256 rows) is the MMA's N or K:
@@ -9,7 +11,7 @@
 // All operands are K-major bf16, so activations and dZ are kept in both orientations
 // ([B, f] and [f, B]) and the weights' bf16 copy in both ([out, in] and, for layers >= 2,
 // [in, out]); the producing epilogues write both.  fp32 master weights take the SGD step of
-// Algorithm 1 in the wgrad epilogue, which also refreshes the bf16 copies.
+// Algorithm 1 in the wgrad kernel, which also refreshes the bf16 copies.
 // When a layer has too few output tiles to fill the GPU, forward and dgrad split the contraction
 // over several blocks; each writes an fp32 partial tile and the block that finishes last adds
 // the partials in ascending split order (so the result does not depend on which block that is).
@@ -22,6 +24,7 @@
 
 #include "mlp.cuh"
 #include "tc_ptx.cuh"
+#include "wgrad_tc.cuh"
 
 namespace mavg {
 namespace {
@@ -31,11 +34,10 @@ using namespace tc;
 constexpr int kBM = 128;        // MMA M (rows of operand A per tile)
 constexpr int kBK = 64;         // contraction elements per pipeline stage (128 bytes of bf16)
 constexpr int kThreads = 320;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
-constexpr int kStageBytes = 8 * 32 * 33 * 4;   // per-warp 32x32 fp32 turn-around tiles (wgrad)
 constexpr int kMaxStages = 8;
 constexpr int kATileBytes = kBM * kBK * 2;
 
-enum { EPI_FWD_HIDDEN = 0, EPI_FWD_LAST = 1, EPI_DGRAD = 2, EPI_WGRAD_SGD = 3 };
+enum { EPI_FWD_HIDDEN = 0, EPI_FWD_LAST = 1, EPI_DGRAD = 2 };
 enum { ERR_PRODUCER = 11, ERR_MMA = 12, ERR_EPILOGUE = 13 };
 
 struct TcArgs {
@@ -60,15 +62,7 @@ struct TcArgs {
   __nv_bfloat16* dz_bm;     // [P, B, cpad]
   int cpad;
   __nv_bfloat16* dz_mb;     // [P, M, B]
-  // EPI_WGRAD_SGD: A rows are output features o, B rows input features i
-  float* rep;               // fp32 masters, W[o, i] at rep[p*rep_stride + w_off + o*in + i]
-  int64_t rep_stride, w_off;
-  int in, out;
-  __nv_bfloat16* w16;       // bf16 copy [out, in] at w16[p*w16_stride + sh_off + o*in + i]
-  int64_t w16_stride, sh_off;
-  __nv_bfloat16* wt16;      // bf16 copy [in, out_pad] or null
-  int64_t wt16_stride, sht_off;
-  int out_pad;
+  int64_t rep_stride;
   float gamma;
   int* status;
 };
@@ -203,60 +197,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const bool ok = mbar_wait(&acc_bar, 0, abortp, g.status, ERR_EPILOGUE);
     tc_fence_after_sync();
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    if (EPI == EPI_WGRAD_SGD) {
-      if (ok) {
-        float* stage =
-            reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes) + ew * (32 * 33);
-        for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
-          float z[32];
-          const int ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
-          // The accumulator arrives with one weight row per lane.  It is turned through shared
-          // memory so that the lanes of a warp walk along a row: every access to the fp32 masters
-          // and to the [out, in] bf16 copy is then a contiguous 128 / 64 bytes per row.
-#pragma unroll
-          for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = z[j];
-          __syncwarp();
-          const int o_base = m0 + q * 32;
-          const int i = n0 + c0 + lane;
-          const bool col_ok = lane < ncols && i < g.in;
-          float* wcol = g.rep + (size_t)p * g.rep_stride + g.w_off + (size_t)o_base * g.in + i;
-          __nv_bfloat16* hcol =
-              g.w16 + (size_t)p * g.w16_stride + g.sh_off + (size_t)o_base * g.in + i;
-          const int rows_valid = min(32, g.out - o_base);   // uniform over the warp
-          if (col_ok && rows_valid > 0) {
-            // 32 independent loads in flight before the first use; rows past the matrix repeat
-            // the last valid row's address and are not stored
-            float wv[32];
-#pragma unroll
-            for (int rr = 0; rr < 32; ++rr)
-              wv[rr] = __ldcs(wcol + (size_t)min(rr, rows_valid - 1) * g.in);
-#pragma unroll
-            for (int rr = 0; rr < 32; ++rr) {
-              const float w = fmaf(-g.gamma, stage[rr * 33 + lane], wv[rr]);
-              if (rr < rows_valid) {
-                wcol[(size_t)rr * g.in] = w;
-                hcol[(size_t)rr * g.in] = __float2bfloat16_rn(w);
-              }
-              stage[rr * 33 + lane] = w;
-            }
-          }
-          __syncwarp();
-          if (g.wt16) {                       // [in, out] copy: lanes walk along out again
-            const int o = o_base + lane;
-            if (o < g.out) {
-              __nv_bfloat16* tcol = g.wt16 + (size_t)p * g.wt16_stride + g.sht_off + o;
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const int ii = n0 + c0 + j;
-                if (j < ncols && ii < g.in)
-                  tcol[(size_t)ii * g.out_pad] = __float2bfloat16_rn(stage[lane * 33 + j]);
-              }
-            }
-          }
-          __syncwarp();
-        }
-      }
-    } else {
+    {
       // forward / dgrad: feature m per lane, the batch along the columns (the dgrad and last-layer
       // tails need the whole batch in one tile: n_tiles == 1 there)
       const int m = m0 + row;
@@ -493,20 +434,6 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   return g;
 }
 
-GemmPlan plan_wgrad(int out, int in, int B) {
-  GemmPlan g{};
-  g.BN = in >= 128 ? 128 : (in + 15) / 16 * 16;
-  g.m_tiles = (out + kBM - 1) / kBM;
-  g.n_tiles = (in + g.BN - 1) / g.BN;
-  g.nkb = (B + kBK - 1) / kBK;
-  g.splits = 1;
-  g.kb_per_split = g.nkb;
-  g.stages = g.nkb < 2 ? 2 : (g.nkb > 4 ? 4 : g.nkb);
-  g.tmem_cols = 32;
-  while ((int)g.tmem_cols < g.BN) g.tmem_cols <<= 1;
-  return g;
-}
-
 TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   TcLayout t{};
   const int L = cfg->n_layers, P = cfg->P, B = cfg->B;
@@ -584,28 +511,39 @@ struct TcState {
   CUtensorMap x_in[2], x_in_t[2];             // layer 1's input: the two gather buffers
   CUtensorMap dz[MAVG_MAX_LAYERS + 1];        // [B, d_l]
   CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
-  GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1], wgrad[MAVG_MAX_LAYERS + 1];
+  CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
+  CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store views of the bf16 copies
+  CUtensorMap wt16_st[MAVG_MAX_LAYERS + 1];
+  GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
+  WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap
   cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,
               ev_x_free[2] = {nullptr, nullptr};
 };
 
-// bf16 tensor [batch, rows, inner] with the given strides (in elements); box = 64 x box_rows.
-bool encode_map(TcState* st, CUtensorMap* m, void* ptr, int inner, int rows, int batch,
-                int64_t row_stride, int64_t batch_stride, int box_rows, std::string* why) {
+// Tensor [batch, rows, inner] with the given strides (in elements) and box inner x box_rows.
+bool encode_any(TcState* st, CUtensorMap* m, CUtensorMapDataType dt, int esize, void* ptr,
+                int inner, int rows, int batch, int64_t row_stride, int64_t batch_stride,
+                int box_inner, int box_rows, CUtensorMapSwizzle swz, std::string* why) {
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)row_stride * 2, (cuuint64_t)batch_stride * 2};
-  cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)box_rows, 1};
+  cuuint64_t strides[2] = {(cuuint64_t)row_stride * esize, (cuuint64_t)batch_stride * esize};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
-  CUresult r = st->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptr, dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  CUresult r = st->encode(m, dt, 3, ptr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     if (why) *why = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
     return false;
   }
   return true;
+}
+
+// bf16 operand of an MMA: 64-element K slabs, 128-byte swizzle.
+bool encode_map(TcState* st, CUtensorMap* m, void* ptr, int inner, int rows, int batch,
+                int64_t row_stride, int64_t batch_stride, int box_rows, std::string* why) {
+  return encode_any(st, m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, inner, rows, batch, row_stride,
+                    batch_stride, kBK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B, why);
 }
 
 template <int EPI>
@@ -625,7 +563,6 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   g.status = (int*)ws_ptr(c, c->ws.status);
   size_t pipe = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2);
   size_t smem = pipe + 1024;
-  if (EPI == EPI_WGRAD_SGD) smem += kStageBytes;
   if (EPI == EPI_FWD_LAST)   // the loss tail reuses the pipeline buffers: logits, dZ, row losses
     smem = std::max(pipe, ((size_t)2 * g.N * g.M + g.N) * sizeof(float)) + 1024;
   dim3 grid((unsigned)(pl.m_tiles * pl.n_tiles * pl.splits), (unsigned)c->cfg.P);
@@ -693,7 +630,7 @@ mavg_status tc_setup(mavg_ctx* c) {
     const int in = cfg.dims[l - 1], out = cfg.dims[l];
     const int dz_ld = l < L ? out : t.cpad;
     st->fwd[l] = plan_partial(out, B, in, P, kPlanSmCount, l < L);
-    st->wgrad[l] = plan_wgrad(out, in, B);
+    st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count);
     __nv_bfloat16* w16 = (__nv_bfloat16*)bf(t.w16) + t.sh_off[l - 1];
     __nv_bfloat16* w16g = (__nv_bfloat16*)bf(t.w16g) + t.sh_off[l - 1];
     ok = ok && encode_map(st, &st->w[l], w16, in, out, P, in, t.n16, kBM, &why);
@@ -703,16 +640,28 @@ mavg_status tc_setup(mavg_ctx* c) {
         ok = ok && encode_map(st, &st->x_in[i], bf(t.xg[i]), in, B, P, in, (int64_t)B * in,
                               st->fwd[l].BN, &why);
         ok = ok && encode_map(st, &st->x_in_t[i], bf(t.xt[i]), B, in, P, B, (int64_t)B * in,
-                              st->wgrad[l].BN, &why);
+                              kWgradTileCols, &why);
       }
     } else {
       ok = ok && encode_map(st, &st->act_in[l], bf(t.act[l - 1]), in, B, P, in, (int64_t)B * in,
                             st->fwd[l].BN, &why);
       ok = ok && encode_map(st, &st->act_in_t[l], bf(t.act_t[l - 1]), B, in, P, B,
-                            (int64_t)B * in, st->wgrad[l].BN, &why);
+                            (int64_t)B * in, kWgradTileCols, &why);
     }
     ok = ok && encode_map(st, &st->dz_t[l], bf(t.dz_t[l]), B, out, P, B, (int64_t)B * out, kBM,
                           &why);
+    ok = ok && encode_any(st, &st->w32[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                          c->buf.replicas + c->layers[l - 1].w_off, in, out, P, in,
+                          c->buf.replica_stride, kWgradTileCols, kWgradTileRows,
+                          CU_TENSOR_MAP_SWIZZLE_128B, &why);
+    ok = ok && encode_any(st, &st->w16_st[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w16, in, out, P,
+                          in, t.n16, kWgradTileCols, kWgradTileRows, CU_TENSOR_MAP_SWIZZLE_64B,
+                          &why);
+    if (l > 1)
+      ok = ok && encode_any(st, &st->wt16_st[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                            (__nv_bfloat16*)bf(t.wt16) + t.sht_off[l - 1], out, in, P,
+                            t.out_pad[l - 1], t.nt16, kWgradTileRows, kWgradTileCols,
+                            CU_TENSOR_MAP_SWIZZLE_NONE, &why);
     if (l > 1) {
       st->dgrad[l] = plan_partial(in, B, out, P, kPlanSmCount, false);
       __nv_bfloat16* wt16 = (__nv_bfloat16*)bf(t.wt16) + t.sht_off[l - 1];
@@ -737,9 +686,7 @@ mavg_status tc_setup(mavg_ctx* c) {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_tc_gemm<EPI_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kMaxDynSmem);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_tc_gemm<EPI_WGRAD_SGD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kMaxDynSmem);
+  if (e == cudaSuccess) e = wgrad_stream_prepare();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);
   cudaEvent_t* evs[] = {&st->ev_fork, &st->ev_wgrad_done, &st->ev_gather_done, &st->ev_x_free[0],
@@ -871,24 +818,19 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wtg[l] : st->wt[l], st->dz[l],
                                     st->dgrad[l], g));
     }
-    TcArgs g{};
-    g.M = ly.out; g.N = ly.in;
-    g.a_batched = 1; g.b_batched = 1;
-    g.rep = c->buf.replicas; g.w_off = ly.w_off;
-    g.in = ly.in; g.out = ly.out;
-    g.w16 = bfp(t.w16); g.w16_stride = t.n16; g.sh_off = t.sh_off[l - 1];
-    g.wt16 = l > 1 ? bfp(t.wt16) : nullptr; g.wt16_stride = t.nt16; g.sht_off = t.sht_off[l - 1];
-    g.out_pad = t.out_pad[l - 1];
     const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
+    const CUtensorMap& wtm = l > 1 ? st->wt16_st[l] : st->w16_st[l];
     if (overlap && l > 1) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
       c->stream = st->s_wgrad;
-      TC_TRY(launch_gemm<EPI_WGRAD_SGD>(c, MAVG_K_WGRAD_SGD, st->dz_t[l], bm, st->wgrad[l], g));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l], wtm,
+                                 l > 1));
       c->stream = main_s;
       side_used = true;
     } else {
-      TC_TRY(launch_gemm<EPI_WGRAD_SGD>(c, MAVG_K_WGRAD_SGD, st->dz_t[l], bm, st->wgrad[l], g));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l], wtm,
+                                 l > 1));
     }
   }
   if (overlap) {

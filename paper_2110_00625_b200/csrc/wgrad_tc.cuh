@@ -1,0 +1,26 @@
+// Launch interface of the streaming weight-gradient + SGD kernel (wgrad_tc.cu).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace mavg {
+
+struct WgradPlan {
+  int nkb, m_tiles, n_tiles, chunk, n_chunks, items, slots, a_bufs, grid;
+  size_t smem;
+};
+
+constexpr int kWgradTileRows = 128;   // rows of out per tile (box rows of the dZ^T and master maps)
+constexpr int kWgradTileCols = 32;    // columns of in per tile
+
+WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count);
+cudaError_t wgrad_stream_prepare();
+// dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
+// w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128
+// (64B swizzle); wt16: bf16 [P, in, out] box 128 x 32 (no swizzle), ignored unless has_wt.
+cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
+                                const CUtensorMap& at, const CUtensorMap& w32,
+                                const CUtensorMap& w16, const CUtensorMap& wt16, bool has_wt);
+
+}  // namespace mavg

@@ -1,0 +1,125 @@
+"""Parity at the full sizes of the workload list, in the launch configuration bench.py times.
+Where the oracle cannot redo the whole workload in seconds, sampled learners / element windows
+are compared, each computed by the oracle one by one."""
+import numpy as np
+import pytest
+import torch
+
+from tests.util import l2_rel, outlier_fraction, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _m():
+    import paper_2110_00625_b200 as m
+    return m
+
+
+@pytest.mark.parametrize("P", [4, 16, 64])
+def test_c3_meta_update_full_length(oracle, P):
+    # n = 11.2 M, replicas N(0, 0.01) around the model, two of the five updates, mu = 0.9
+    m = _m()
+    n = m.workloads.CONFIGS["C3"]["n"]
+    w1 = m.workloads.global_model(n)
+    g = m.Mavg(w1, P=P, K=1, local_lr=0.1, mu=0.9, objective=m.OBJ_NONE)
+    o = oracle.Mavg(w1, P=P, K=1, gamma=0.1, mu=0.9, stride=g.stride)
+    gen = torch.Generator().manual_seed(100 + P)
+    for u in range(2):
+        # perturbations drawn once on the host and handed to both sides
+        for j in range(P):
+            o.replicas[j, :n] = o.w + 0.1 * torch.randn(n, generator=gen).numpy()
+        g.replicas.copy_(torch.from_numpy(o.replicas))
+        g.meta_update()
+        o.meta_update()
+    g.sync()
+    assert rel_err(g.w.cpu().numpy(), o.w) <= 1e-5
+    assert rel_err(g.v.cpu().numpy(), o.v) <= 1e-5
+    rows = g.replicas[[0, P - 1]].cpu().numpy()
+    assert np.array_equal(rows[0, :n], g.w.cpu().numpy()) and np.array_equal(rows[1], rows[0])
+
+
+@pytest.mark.parametrize("K", [1, 64])
+def test_c5_round_full_length_sampled(oracle, K):
+    # n = 25.6 M, P = 16: the replicas after the K fused local steps on sampled windows (first,
+    # middle, ragged end), then the meta-update on those windows' elements
+    m = _m()
+    cfg = m.workloads.CONFIGS["C5"]
+    n, P, gamma, sigma = cfg["n"] + 3, cfg["P"], cfg["gamma"], cfg["sigma"]
+    w1 = m.workloads.global_model(n)
+    g = m.Mavg(w1, P=P, K=K, local_lr=gamma, mu=0.9, seed=77, objective=m.OBJ_PSEUDOGRAD,
+               sigma=sigma)
+    g.local_steps()
+    g.sync()
+    windows = [(0, 4096), (n // 2 - 1000, 4099), (n - 3001, 3001)]
+    rep = g.replicas.cpu().numpy()
+    want_rows = {}
+    for (i0, cnt) in windows:
+        for j in (0, 7, P - 1):
+            w = w1[i0:i0 + cnt].astype(np.float32).copy()
+            for k in range(1, K + 1):
+                gr = oracle.pseudograd(77, 1, j, k, i0, cnt, sigma)
+                w = (w.astype(np.float64) - np.float64(np.float32(gamma)) * gr).astype(np.float32)
+            want_rows[(i0, j)] = w
+            assert rel_err(rep[j, i0:i0 + cnt], w) <= 1e-5
+    # meta-update against the oracle fed with the GPU's replicas (teacher-forced), full length
+    o = oracle.Mavg(w1, P=P, K=1, gamma=gamma, mu=0.9, stride=g.stride)
+    o.replicas[:] = rep
+    g.meta_update()
+    o.meta_update()
+    g.sync()
+    assert rel_err(g.w.cpu().numpy(), o.w) <= 1e-5
+    assert rel_err(g.v.cpu().numpy(), o.v) <= 1e-5
+
+
+def test_c2_full_shape_two_rounds(oracle):
+    # the benchmark workload itself: 3072-512-512-10, P=8, K=8, B=128, 50 000 samples, bf16 data
+    m = _m()
+    cfg = m.workloads.CONFIGS["C2"]
+    x, y = m.workloads.make_dataset(cfg)
+    w1 = m.workloads.mlp_init(cfg["dims"])
+    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+               seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1,
+               x=x, y=y, x_bf16=True)
+    o = oracle.Mavg(w1, P=cfg["P"], K=cfg["K"], gamma=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+                    seed=m.workloads.BASE_SEED, objective=oracle.OBJ_MLP, dims=cfg["dims"],
+                    bf16=True, x=x, y=y, stride=g.stride)
+    for r in range(2):
+        lg = g.round(want_loss=True)
+        lo, _ = o.run_round()
+        assert abs(lg - lo) <= 2e-2 * abs(lo), (r, lg, lo)
+        assert rel_err(g.w.cpu().numpy(), o.w) <= 5e-2
+        assert l2_rel(g.v.cpu().numpy(), o.v) <= 5e-2
+    for (n_, j, k) in [(1, 0, 1), (3, 7, 8)]:
+        assert np.array_equal(g.get_batch_indices(n_, j, k),
+                              oracle.batch_indices(m.workloads.BASE_SEED, n_, 8, j, k, 50000, 128))
+
+
+def test_c4_full_shape_sampled_learners(oracle):
+    # 3072-2048-2048-2048-10, P=32, K=16, B=64: one local step from the broadcast state on the
+    # GPU for all learners; the oracle redoes it for two sampled learners
+    m = _m()
+    cfg = dict(m.workloads.CONFIGS["C4"])
+    x, y = m.workloads.make_dataset(cfg)
+    w1 = m.workloads.mlp_init(cfg["dims"])
+    g = m.Mavg(w1, P=cfg["P"], K=1, local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+               seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1,
+               x=x, y=y, x_bf16=True)
+    g.local_steps()
+    g.sync()
+    losses = g.get_losses()
+    n = g.n
+    for j in (0, 31):
+        idx = oracle.batch_indices(m.workloads.BASE_SEED, 1, cfg["P"], j, 1, cfg["S"], cfg["B"])
+        lo, grad = oracle.mlp_loss_grad(cfg["dims"], w1, x[idx], y[idx], bf16=True)
+        step_o = -np.float64(np.float32(cfg["gamma"])) * grad.astype(np.float64)
+        step_g = g.replicas[j, :n].cpu().numpy().astype(np.float64) - w1
+        assert abs(losses[j, 0] - lo) <= 2e-2 * abs(lo)
+        assert l2_rel(step_g, step_o) <= 2e-2
+        assert outlier_fraction(step_g, step_o, 5e-2) <= 0.02
+    # a second step uses the per-learner weight copies: run it and one meta-update, finite output
+    g.set_hparams(1, cfg["gamma"], 1.0, cfg["mu"])
+    g.meta_update()
+    g.local_steps()
+    g.meta_update()
+    g.sync()
+    assert torch.isfinite(g.w).all() and torch.isfinite(g.v).all()

@@ -4,6 +4,7 @@
 // 4P + 8 bytes written.  d is formed as (sum_j (w^j - w~)) / P in ascending j, which is the same
 // real number and keeps the fp32 sum small.
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace mavg {
 namespace {
@@ -100,6 +101,173 @@ k_broadcast(float* __restrict__ rep, int64_t stride, const float* __restrict__ w
   }
 }
 
+// ---- the same update driven by bulk copies ------------------------------------------------------
+// One block per SM walks over tiles of T consecutive elements.  A producer warp keeps a ring of
+// STAGES shared-memory stages filled with G replica tiles each (cp.async.bulk, completion counted
+// on mbarriers) plus the tile of w~ and v; THREADS consumer threads add the differences
+// w^j - w~ in ascending j, form v and w~, and one thread sends the two result tiles back and
+// the w~ tile to every replica with bulk stores.  Bytes in flight per SM are set by the ring
+// (tens of KB), not by registers, which is what a pass with 2P+4 concurrent streams needs.
+enum { ERR_META_PRODUCER = 31, ERR_META_CONSUMER = 32 };
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes,
+                                          uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+               "r"(tc::smem_u32(src)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_read_all() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_plain(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc::smem_u32(bar)) : "memory");
+}
+
+template <int T, int G, int STAGES, int THREADS>
+__global__ void __launch_bounds__(THREADS + 32)
+k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
+                   float* __restrict__ v, int P, int64_t n_tiles, float mu, float zeta,
+                   float inv_p, int read_v, int* status) {
+  extern __shared__ __align__(128) uint8_t sm[];
+  float* st_rep = reinterpret_cast<float*>(sm);            // [STAGES][G][T]
+  float* st_wv = st_rep + (size_t)STAGES * G * T;          // [2][2][T]: (w~, v) of two tiles
+  float* st_out = st_wv + 4 * T;                           // [2][2][T]: (new w~, new v)
+  __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], wv_full[2], wv_empty[2];
+  __shared__ int abort_flag;
+  constexpr int kWarps = THREADS / 32;
+  constexpr int PER = T / THREADS;                          // elements per thread, multiple of 4
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      tc::mbar_init(&full[s], 1);
+      tc::mbar_init(&empty[s], kWarps);
+    }
+    for (int b = 0; b < 2; ++b) {
+      tc::mbar_init(&wv_full[b], 1);
+      tc::mbar_init(&wv_empty[b], kWarps);
+    }
+    abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::fence_proxy_async();
+  }
+  __syncthreads();
+  volatile int* abortp = &abort_flag;
+  const int groups = (P + G - 1) / G;
+  if (tid >= THREADS) {                                     // producer warp
+    if (tid == THREADS) {
+      uint32_t sc = 0, tcount = 0;
+      for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tcount) {
+        const int b = tcount & 1;
+        if (!tc::mbar_wait(&wv_empty[b], ((tcount >> 1) & 1) ^ 1, abortp, status, ERR_META_PRODUCER))
+          return;
+        tc::mbar_arrive_expect_tx(&wv_full[b], (read_v ? 2 : 1) * T * 4);
+        bulk_load(st_wv + (size_t)(b * 2) * T, w + t * T, T * 4, &wv_full[b]);
+        if (read_v) bulk_load(st_wv + (size_t)(b * 2 + 1) * T, v + t * T, T * 4, &wv_full[b]);
+        for (int gi = 0; gi < groups; ++gi, ++sc) {
+          const int s = sc % STAGES;
+          if (!tc::mbar_wait(&empty[s], ((sc / STAGES) & 1) ^ 1, abortp, status, ERR_META_PRODUCER))
+            return;
+          const int cnt = min(G, P - gi * G);
+          tc::mbar_arrive_expect_tx(&full[s], (uint32_t)cnt * T * 4);
+          for (int u = 0; u < cnt; ++u)
+            bulk_load(st_rep + ((size_t)s * G + u) * T, rep + (size_t)(gi * G + u) * stride + t * T,
+                      T * 4, &full[s]);
+        }
+      }
+    }
+    return;
+  }
+  uint32_t sc = 0, tcount = 0;
+  const int lane = tid & 31;
+  for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tcount) {
+    const int b = tcount & 1;
+    if (!tc::mbar_wait(&wv_full[b], (tcount >> 1) & 1, abortp, status, ERR_META_CONSUMER)) return;
+    float wt[PER], acc[PER];
+#pragma unroll
+    for (int i = 0; i < PER; i += 4) {
+      const float4 x =
+          *reinterpret_cast<const float4*>(st_wv + (size_t)(b * 2) * T + (i / 4) * THREADS * 4 + tid * 4);
+      wt[i] = x.x; wt[i + 1] = x.y; wt[i + 2] = x.z; wt[i + 3] = x.w;
+      acc[i] = acc[i + 1] = acc[i + 2] = acc[i + 3] = 0.f;
+    }
+    for (int gi = 0; gi < groups; ++gi, ++sc) {
+      const int s = sc % STAGES;
+      if (!tc::mbar_wait(&full[s], (sc / STAGES) & 1, abortp, status, ERR_META_CONSUMER)) return;
+      const int cnt = min(G, P - gi * G);
+      for (int u = 0; u < cnt; ++u) {                       // ascending j
+#pragma unroll
+        for (int i = 0; i < PER; i += 4) {
+          const float4 x = *reinterpret_cast<const float4*>(st_rep + ((size_t)s * G + u) * T +
+                                                            (i / 4) * THREADS * 4 + tid * 4);
+          acc[i] += x.x - wt[i];
+          acc[i + 1] += x.y - wt[i + 1];
+          acc[i + 2] += x.z - wt[i + 2];
+          acc[i + 3] += x.w - wt[i + 3];
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive_plain(&empty[s]);
+    }
+    // the result buffers of the tile before last must have been read by their stores
+    if (tid == 0) bulk_wait_read_all();
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
+#pragma unroll
+    for (int i = 0; i < PER; i += 4) {
+      float4 vt = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (read_v)
+        vt = *reinterpret_cast<const float4*>(st_wv + (size_t)(b * 2 + 1) * T +
+                                              (i / 4) * THREADS * 4 + tid * 4);
+      float4 vn, wn;
+      vn.x = fmaf(mu, vt.x, zeta * (acc[i] * inv_p));
+      vn.y = fmaf(mu, vt.y, zeta * (acc[i + 1] * inv_p));
+      vn.z = fmaf(mu, vt.z, zeta * (acc[i + 2] * inv_p));
+      vn.w = fmaf(mu, vt.w, zeta * (acc[i + 3] * inv_p));
+      wn.x = wt[i] + vn.x; wn.y = wt[i + 1] + vn.y; wn.z = wt[i + 2] + vn.z; wn.w = wt[i + 3] + vn.w;
+      *reinterpret_cast<float4*>(st_out + (size_t)(b * 2) * T + (i / 4) * THREADS * 4 + tid * 4) = wn;
+      *reinterpret_cast<float4*>(st_out + (size_t)(b * 2 + 1) * T + (i / 4) * THREADS * 4 + tid * 4) = vn;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive_plain(&wv_empty[b]);
+    tc::fence_proxy_async();
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
+    if (tid == 0) {
+      bulk_store(w + t * T, st_out + (size_t)(b * 2) * T, T * 4);
+      bulk_store(v + t * T, st_out + (size_t)(b * 2 + 1) * T, T * 4);
+      for (int j = 0; j < P; ++j)
+        bulk_store(rep + (size_t)j * stride + t * T, st_out + (size_t)(b * 2) * T, T * 4);
+      bulk_commit();
+    }
+  }
+  if (tid == 0) bulk_wait_read_all();
+}
+
+template <int T, int G, int STAGES, int THREADS>
+cudaError_t launch_bulk(mavg_ctx* c, int64_t n_tiles, float mu, float zeta, float inv_p,
+                        int read_v) {
+  const size_t smem = ((size_t)STAGES * G * T + 8 * (size_t)T) * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_meta_update_bulk<T, G, STAGES, THREADS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int grid = (int)(n_tiles < c->sm_count ? n_tiles : c->sm_count);
+  k_meta_update_bulk<T, G, STAGES, THREADS><<<grid, THREADS + 32, smem, c->stream>>>(
+      c->buf.replicas, c->buf.replica_stride, c->buf.global_w, c->buf.momentum, c->cfg.P, n_tiles,
+      mu, zeta, inv_p, read_v, (int*)ws_ptr(c, c->ws.status));
+  return cudaGetLastError();
+}
+
 int grid_for(const mavg_ctx* c, int64_t work_items, int threads, int blocks_per_sm) {
   int64_t need = (work_items + threads - 1) / threads;
   int64_t cap = (int64_t)c->sm_count * blocks_per_sm;
@@ -126,21 +294,37 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
   const float mu = c->cfg.mu, zeta = c->cfg.block_lr;
   const float inv_p = 1.0f / (float)P;
   const int read_v = mu != 0.f ? 1 : 0;
-  int grid = grid_for(c, n >> 2, 256, 6);
   // A replica set that fits in L2 is about to be re-read by the next round's first local step:
-  // keep it there.  Larger sets are written with evict-first stores.
-  const bool stream_st = (size_t)P * (size_t)n * 4 > c->l2_bytes / 2;
+  // it takes the plain-store kernel, which leaves it there.  Larger sets with more than 8
+  // replicas go through the bulk-copy kernel tile by tile (measured faster from P = 16 up; with
+  // few replicas the register kernel already keeps enough loads in flight); what is left of n
+  // after the last whole tile, short vectors and small P take the register kernel with
+  // evict-first stores.
+  const bool big = (size_t)P * (size_t)n * 4 > c->l2_bytes / 2;
+  int64_t done = 0;
   prof_begin(c, MAVG_K_META);
-  if (stream_st)
-    k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
-                                                        c->buf.global_w, c->buf.momentum, P, n,
-                                                        mu, zeta, inv_p, read_v);
-  else
-    k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
-                                                         c->buf.global_w, c->buf.momentum, P, n,
-                                                         mu, zeta, inv_p, read_v);
+  cudaError_t e = cudaSuccess;
+  if (big && P > 8 && n >= (int64_t)4096 * c->sm_count * 4) {
+    done = n / 4096 * 4096;
+    e = launch_bulk<4096, 2, 3, 512>(c, n / 4096, mu, zeta, inv_p, read_v);
+  }
+  if (e == cudaSuccess && done < n) {
+    const int64_t rest = n - done;
+    int grid = grid_for(c, rest >> 2, 256, 8);
+    float* rep = c->buf.replicas + done;
+    float* w = c->buf.global_w + done;
+    float* v = c->buf.momentum + done;
+    if (big)
+      k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
+                                                          rest, mu, zeta, inv_p, read_v);
+    else
+      k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
+                                                           rest, mu, zeta, inv_p, read_v);
+    e = cudaGetLastError();
+    if (done > 0) c->launches++;
+  }
   prof_end(c);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace mavg

@@ -274,7 +274,12 @@ def run_mavg(args):
     peaks = measured_peaks()
     if args.workload == "C5":
         return run_pseudograd(args, m, torch, peaks, rank)
+    if args.sweep_only:
+        print(json.dumps({"meta_update_sweep": meta_update_sweep(m, torch, peaks, reps=2)}))
+        return 0
     cfg, x, y, w1 = workload_inputs(args.workload)
+    if args.learners:
+        cfg["P"] = args.learners      # reduced-size captures under a profiler only
 
     # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
     cpu = None
@@ -424,6 +429,10 @@ def main():
     ap.add_argument("--workload", default="C2", choices=["C2", "C4", "C5"],
                     help="C2 is the benchmark workload; C4 (large MLP) and C5 (pseudo-gradient "
                          "round at 25.6 M parameters) print the same measurements for context")
+    ap.add_argument("--learners", type=int, default=0,
+                    help="override P (for small profiler captures; not a benchmark setting)")
+    ap.add_argument("--sweep-only", action="store_true",
+                    help="run only the meta-update sweep (profiler captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     args = ap.parse_args()

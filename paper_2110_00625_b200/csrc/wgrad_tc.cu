@@ -8,9 +8,11 @@
 //                   of A^T into a ring of shared-memory slots; the 128 x B tile of dZ^T is loaded
 //                   once per work item (a run of column tiles of one learner and row tile);
 //   MMA warp        one thread issues tcgen05.mma (M=128, N=32, K=B) into one of two TMEM buffers;
-//   4 epilogue warps read the accumulator (tcgen05.ld, one weight row per lane), update the master
-//                   tile in place in shared memory, write the bf16 tiles beside it, and one
-//                   thread sends all three back with TMA stores.
+//   2 x 4 epilogue warps (one group per TMEM buffer, i.e. per tile parity) read the accumulator
+//                   (tcgen05.ld, one weight row per lane), update the master tile in place in
+//                   shared memory and write the bf16 tiles beside it;
+//   store warp      one thread sends the three finished tiles back with TMA stores and frees the
+//                   slot once they have left shared memory.
 // Edge tiles need no predicates: TMA zero-fills loads and clips stores at the tensor bounds.
 #include <cuda.h>
 
@@ -24,12 +26,12 @@ namespace {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 32, kBK = 64;
-constexpr int kThreads = 192;            // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
+constexpr int kThreads = 352;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores
 constexpr int kMaxSlots = 4;
 constexpr int kW32Bytes = kBM * kBN * 4;  // 16 KB, rows of 128 bytes, 128-byte swizzle
 constexpr int kW16Bytes = kBM * kBN * 2;  //  8 KB, rows of  64 bytes,  64-byte swizzle
 constexpr int kWtBytes = kBN * kBM * 2;   //  8 KB, rows of 256 bytes, no swizzle
-enum { ERR_WG_PRODUCER = 21, ERR_WG_MMA = 22, ERR_WG_EPILOGUE = 23 };
+enum { ERR_WG_PRODUCER = 21, ERR_WG_MMA = 22, ERR_WG_EPILOGUE = 23, ERR_WG_STORE = 24 };
 
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* src, int c0, int c1,
                                              int c2) {
@@ -48,9 +50,6 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void epilogue_barrier4() {
-  asm volatile("bar.sync 1, 128;" ::: "memory");
 }
 
 struct WgradArgs {
@@ -74,7 +73,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
                    const __grid_constant__ CUtensorMap tm_wt16,  // bf16 [P, in, out] store
                    const WgradArgs g) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
   __shared__ __align__(8) uint64_t tmem_full[2], tmem_empty[2];
   __shared__ __align__(8) uint64_t a_full[2], a_empty[2];
   __shared__ uint32_t tmem_slot;
@@ -99,6 +98,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     for (int s = 0; s < g.slots; ++s) {
       mbar_init(&slot_full[s], 1);
       mbar_init(&slot_empty[s], 1);
+      mbar_init(&out_full[s], 4);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&tmem_full[b], 1);
@@ -203,7 +203,8 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 10) {
+    const int grp = (warp - 2) >> 2;           // epilogue group = TMEM buffer = tile parity
     const int q = warp & 3;                    // TMEM lane quarter this warp may read
     const int r = q * 32 + lane;               // weight row inside the tile
     uint32_t tile_ctr = 0;
@@ -212,23 +213,23 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
       int p, m0, nt0, nt;
       decode(item, p, m0, nt0, nt);
       for (int j = 0; j < nt; ++j, ++tile_ctr) {
+        if ((int)(tile_ctr & 1) != grp) continue;
         const int s = tile_ctr % g.slots;
         const uint32_t use = tile_ctr / g.slots;
-        const int tb = tile_ctr & 1;
         const uint32_t tuse = tile_ctr >> 1;
         // the master tile landed with the same barrier the MMA waited on; the accumulator next
         if (!mbar_wait(&slot_full[s], use & 1, abortp, g.status, ERR_WG_EPILOGUE) ||
-            !mbar_wait(&tmem_full[tb], tuse & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
+            !mbar_wait(&tmem_full[grp], tuse & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
           ok = false;
           break;
         }
         tc_fence_after_sync();
         uint32_t acc[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * kBN), acc);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(grp * kBN), acc);
         tmem_ld_wait();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tmem_empty[tb]);     // this warp is done with the buffer
+        if (lane == 0) mbar_arrive(&tmem_empty[grp]);    // this warp is done with the buffer
 
         uint8_t* sl = slot_base + (size_t)s * slot_bytes;
         uint8_t* w32 = sl + (size_t)r * 128;             // 8 chunks of 16 B, chunk c at c ^ (r & 7)
@@ -259,8 +260,25 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           for (int i = 0; i < 32; ++i) *reinterpret_cast<uint16_t*>(wt + (size_t)i * 256) = hh[i];
         }
         fence_proxy_async();                   // generic-proxy writes -> visible to the TMA stores
-        epilogue_barrier4();
-        if (warp == 2 && lane == 0) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&out_full[s]);
+      }
+    }
+  } else {
+    if (lane == 0) {
+      uint32_t tile_ctr = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < g.items && ok; item += gridDim.x) {
+        int p, m0, nt0, nt;
+        decode(item, p, m0, nt0, nt);
+        for (int j = 0; j < nt; ++j, ++tile_ctr) {
+          const int s = tile_ctr % g.slots;
+          const uint32_t use = tile_ctr / g.slots;
+          if (!mbar_wait(&out_full[s], use & 1, abortp, g.status, ERR_WG_STORE)) {
+            ok = false;
+            break;
+          }
+          uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
           tma_store_3d(&tm_w32, sl, i0, m0, p);
           tma_store_3d(&tm_w16, sl + kW32Bytes, i0, m0, p);
@@ -273,11 +291,10 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           }
         }
       }
-    }
-    if (warp == 2 && lane == 0) {
       tma_store_wait_read<0>();
       if (tile_ctr > 0 && ok) mbar_arrive(&slot_empty[(tile_ctr - 1) % g.slots]);
     }
+    __syncwarp();
   }
   tc_fence_before_sync();
   __syncthreads();

@@ -90,8 +90,10 @@ __device__ __forceinline__ int load_acc_chunk(uint32_t lane_addr, int c0, int BN
   return min(32, BN - c0);
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(kThreads)
+// MINB = 2 caps the registers so that two blocks fit an SM (used when a launch has more blocks
+// than SMs; costs a few spills in the tail), MINB = 1 leaves the compiler free.
+template <int EPI, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
           const TcArgs g) {
   extern __shared__ uint8_t smem_raw[];
@@ -401,7 +403,7 @@ struct TcLayout {
   size_t end;
 };
 
-struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages; uint32_t tmem_cols; };
+struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages, two_per_sm; uint32_t tmem_cols; };
 
 // Forward / dgrad plan.  To fill the GPU the batch may be cut into column tiles (`tile_n`: only
 // the hidden-layer forward can, its tail needs no sum over the batch) and, if blocks are still
@@ -426,7 +428,11 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   g.kb_per_split = (g.nkb + want - 1) / want;
   g.splits = (g.nkb + g.kb_per_split - 1) / g.kb_per_split;
   int stage_bytes = kATileBytes + g.BN * kBK * 2;
-  g.stages = 200 * 1024 / stage_bytes;
+  // more blocks than SMs: two blocks share an SM, so that one block's set-up and tail overlap
+  // the other's main loop; otherwise one block takes the whole shared memory
+  g.two_per_sm = g.m_tiles * g.n_tiles * g.splits * P > sm_count ? 1 : 0;
+  const int budget = g.two_per_sm ? 104 * 1024 : 200 * 1024;
+  g.stages = budget / stage_bytes;
   if (g.stages > kMaxStages) g.stages = kMaxStages;
   if (g.stages > g.kb_per_split) g.stages = g.kb_per_split < 2 ? 2 : g.kb_per_split;
   g.tmem_cols = 32;
@@ -577,7 +583,8 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   lc.attrs = at;
   lc.numAttrs = 1;
   prof_begin(c, cls);
-  cudaError_t e = cudaLaunchKernelEx(&lc, k_tc_gemm<EPI>, a, b, g);
+  cudaError_t e = pl.two_per_sm ? cudaLaunchKernelEx(&lc, k_tc_gemm<EPI, 2>, a, b, g)
+                                : cudaLaunchKernelEx(&lc, k_tc_gemm<EPI, 1>, a, b, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -678,14 +685,13 @@ mavg_status tc_setup(mavg_ctx* c) {
   }
   // 227 KB per block in all, of which a few hundred bytes are the kernel's static variables
   constexpr int kMaxDynSmem = 225 * 1024;
-  e = cudaFuncSetAttribute(k_tc_gemm<EPI_FWD_HIDDEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kMaxDynSmem);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_tc_gemm<EPI_FWD_LAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kMaxDynSmem);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_tc_gemm<EPI_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kMaxDynSmem);
+  e = cudaSuccess;
+  const void* kernels[] = {(const void*)k_tc_gemm<EPI_FWD_HIDDEN, 1>, (const void*)k_tc_gemm<EPI_FWD_HIDDEN, 2>,
+                           (const void*)k_tc_gemm<EPI_FWD_LAST, 1>,   (const void*)k_tc_gemm<EPI_FWD_LAST, 2>,
+                           (const void*)k_tc_gemm<EPI_DGRAD, 1>,      (const void*)k_tc_gemm<EPI_DGRAD, 2>};
+  for (const void* k : kernels)
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
   if (e == cudaSuccess) e = wgrad_stream_prepare();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);

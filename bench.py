@@ -169,8 +169,8 @@ def kernel_rooflines(cfg, prof, steps, peaks, tensor_path):
                          flops=K * 2 * rows * sum(nW)),
         "dgrad_gemm": dict(bytes=K * (2 * P * sum(nW[1:]) + 2 * rows * (sum(dims[2:]) + 3 * sum(dims[1:-1]))),
                            flops=K * 2 * rows * sum(nW[1:])),
-        # fp32 master read + written, bf16 copy written (row- and column-major for layers >= 2)
-        "wgrad_sgd_gemm": dict(bytes=K * (P * (10 * sum(nW) + 2 * sum(nW[1:])) + 2 * rows * sum(dims)),
+        # fp32 master read + written, bf16 copy written
+        "wgrad_sgd_gemm": dict(bytes=K * (P * 10 * sum(nW) + 2 * rows * sum(dims)),
                                flops=K * 2 * rows * sum(nW)),
     }
     for name, (ms, cnt) in prof.items():
@@ -221,6 +221,23 @@ def meta_update_sweep(m, torch, peaks, reps=5):
             del g
             torch.cuda.empty_cache()
     return res
+
+
+def reduce_max_over_ranks(values, device=None):
+    """MAX over ranks of a list of floats (the slowest rank's times count); identity without a
+    process group.  Works on any backend: the tensor lives on `device`."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(units_per_step, steps, total_ms, world):
+    """Aggregate throughput of `world` independent replicas of the workload (replicas only: the
+    method is simulated inside one GPU, there is nothing to exchange between GPUs)."""
+    return world * units_per_step * steps / (total_ms * 1e-3)
 
 
 def run_pseudograd(args, m, torch, peaks, rank):
@@ -356,10 +373,7 @@ def run_mavg(args):
     g.set_profiling(False)
     kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1)
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=g.device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = t.tolist()
+    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=g.device)
 
     line = None
     if rank == 0:
@@ -385,7 +399,7 @@ def run_mavg(args):
         sweep = meta_update_sweep(m, torch, peaks) if world == 1 and not args.no_sweep else None
         n = g.n
         line = {
-            "metric": METRIC, "value": world * units * args.steps / (total_ms * 1e-3), "unit": UNIT,
+            "metric": METRIC, "value": whole_job_value(units, args.steps, total_ms, world), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if mode else "f32", "data": "synthetic",
@@ -399,7 +413,7 @@ def run_mavg(args):
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
                        "reasons": clocks["reasons"], "samples": clocks["samples"]},
-            "e2e": {"value": world * units * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+            "e2e": {"value": whole_job_value(units, args.steps, e2e_ms, world), "unit": UNIT,
                     "h2d_bytes_per_step": 8 * n, "d2h_bytes_per_step": 8 * n + 4},
             "gpu_launches": launches,
             "roofline": roof,

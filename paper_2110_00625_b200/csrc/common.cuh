@@ -37,8 +37,6 @@ __host__ __device__ __forceinline__ uint64_t learner_key(uint64_t seed, uint64_t
 struct MlpLayer {
   int in, out;
   int64_t w_off, b_off;      // offsets (floats) inside a replica
-  int64_t sh_off, sht_off;   // offsets (bf16 elements) inside a shadow row / transposed shadow row
-  int out_pad;               // row length of the transposed shadow [in, out_pad]
 };
 
 struct Workspace {           // byte offsets into the caller's scratch buffer

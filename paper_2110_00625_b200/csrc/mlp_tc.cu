@@ -6,12 +6,13 @@
 // Every product is arranged so that the 128-row MMA dimension is a feature dimension and the
 // batch (16..256 rows) is the MMA's N or K:
 //   forward   Z^T[out, B]  = W[out, in]    . A[B, in]^T        contraction over in
-//   dgrad     dA^T[in, B]  = W^T[in, out]  . dZ[B, out]^T      contraction over out
+//   dgrad     dA^T[in, B]  = W^T[in, out]  . dZ[B, out]^T      contraction over out (W^T = W read MN-major)
 //   wgrad     dW[out, in]  = dZ^T[out, B]  . A^T[in, B]^T      contraction over the batch
-// All operands are K-major bf16, so activations and dZ are kept in both orientations
-// ([B, f] and [f, B]) and the weights' bf16 copy in both ([out, in] and, for layers >= 2,
-// [in, out]); the producing epilogues write both.  fp32 master weights take the SGD step of
-// Algorithm 1 in the wgrad kernel, which also refreshes the bf16 copies.
+// Activations and dZ are kept in both orientations ([B, f] and [f, B]; the producing epilogues
+// write both) so that they are K-major wherever they are an operand.  The weights have one bf16
+// copy, [out, in]: forward reads it K-major, dgrad reads the same tiles MN-major.  fp32 master
+// weights take the SGD step of Algorithm 1 in the wgrad kernel, which also refreshes the bf16
+// copy.
 // When a layer has too few output tiles to fill the GPU, forward and dgrad split the contraction
 // over several blocks; each writes an fp32 partial tile and the block that finishes last adds
 // the partials in ascending split order (so the result does not depend on which block that is).
@@ -45,6 +46,7 @@ struct TcArgs {
   int BN;                   // N tile: multiple of 16, <= 256
   int m_tiles, n_tiles, splits, kb_per_split, nkb, stages;
   int a_batched, b_batched; // 0: the operand is shared by all learners
+  int a_mn;                 // 1: A is read MN-major from a [K rows, M contiguous] array (dgrad: W itself)
   int P;
   uint32_t tmem_cols;
   // forward / dgrad: A rows are features m (M of them), B rows the batch (N = B of them)
@@ -155,7 +157,13 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (!mbar_wait(&empty_bar[s], (u & 1) ^ 1, abortp, g.status, ERR_PRODUCER)) break;
         uint8_t* sa = smem + (size_t)s * stage_bytes;
         mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
-        tma_load_3d(sa, &tmA, &full_bar[s], (kb0 + i) * kBK, m0, g.a_batched ? p : 0);
+        if (g.a_mn) {     // two 64-wide halves of the M range, each 64 K-rows of 128 bytes
+          tma_load_3d(sa, &tmA, &full_bar[s], m0, (kb0 + i) * kBK, g.a_batched ? p : 0);
+          tma_load_3d(sa + kATileBytes / 2, &tmA, &full_bar[s], m0 + 64, (kb0 + i) * kBK,
+                      g.a_batched ? p : 0);
+        } else {
+          tma_load_3d(sa, &tmA, &full_bar[s], (kb0 + i) * kBK, m0, g.a_batched ? p : 0);
+        }
         tma_load_3d(sa + kATileBytes, &tmB, &full_bar[s], (kb0 + i) * kBK, n0,
                     g.b_batched ? p : 0);
         issued = i + 1;
@@ -172,18 +180,21 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = idesc_bf16_f32(kBM, g.BN);
+      const uint32_t idesc = idesc_bf16_f32(kBM, g.BN, g.a_mn);
       bool ok = true;
       for (int i = 0; i < count; ++i) {
         const int s = i % stages, u = i / stages;
         if (!mbar_wait(&full_bar[s], u & 1, abortp, g.status, ERR_MMA)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t adesc = smem_desc_k_sw128(sa);
+        const uint64_t adesc = g.a_mn ? smem_desc_mn_sw128(sa) : smem_desc_k_sw128(sa);
         const uint64_t bdesc = smem_desc_k_sw128(sa + kATileBytes);
+        // per MMA (16 K-elements) a K-major tile advances 32 bytes inside its 128-byte rows, an
+        // MN-major tile 16 rows of 128 bytes; descriptor addresses count 16-byte units
+        const uint32_t a_step = g.a_mn ? (16 * 128) >> 4 : 2;
 #pragma unroll
-        for (int k = 0; k < kBK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-          umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (uint32_t)((i | k) != 0));
+        for (int k = 0; k < kBK / 16; ++k)
+          umma_bf16(tmem_base, adesc + a_step * k, bdesc + 2 * k, idesc, (uint32_t)((i | k) != 0));
         umma_commit(&empty_bar[s]);
       }
       if (ok) umma_commit(&acc_bar);
@@ -367,22 +378,14 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   if (warp == 1) tmem_dealloc(tmem_base, g.tmem_cols);
 }
 
-// bf16 copies of the global model w~ (shared by all learners at the first step of a round, when
+// bf16 copy of the global model w~ (shared by all learners at the first step of a round, when
 // every replica equals w~).  One launch per layer; grid-stride over the layer's weights.
 __global__ void __launch_bounds__(256)
-k_shadow_from_global(const float* __restrict__ w, int64_t w_off, int in, int out,
-                     __nv_bfloat16* __restrict__ w16, int64_t sh_off,
-                     __nv_bfloat16* __restrict__ wt16, int64_t sht_off, int out_pad) {
-  const int64_t total = (int64_t)in * out;
+k_shadow_from_global(const float* __restrict__ w, int64_t w_off, int64_t total,
+                     __nv_bfloat16* __restrict__ w16, int64_t sh_off) {
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-       t += (int64_t)gridDim.x * blockDim.x) {
-    __nv_bfloat16 h = __float2bfloat16_rn(w[w_off + t]);
-    w16[sh_off + t] = h;
-    if (wt16) {
-      const int o = (int)(t / in), i = (int)(t % in);
-      wt16[sht_off + (int64_t)i * out_pad + o] = h;
-    }
-  }
+       t += (int64_t)gridDim.x * blockDim.x)
+    w16[sh_off + t] = __float2bfloat16_rn(w[w_off + t]);
 }
 
 // ---------------------------------------------------------------------------------- host side
@@ -391,15 +394,14 @@ size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct TcLayout {
   int L;
   int cpad;                                  // last layer's dZ row length (multiple of 8)
-  int64_t n16, nt16;                         // elements per bf16 copy row
-  int64_t sh_off[MAVG_MAX_LAYERS], sht_off[MAVG_MAX_LAYERS];
-  int out_pad[MAVG_MAX_LAYERS];
+  int64_t n16;                               // elements per bf16 copy row
+  int64_t sh_off[MAVG_MAX_LAYERS];
   size_t xg[2], xt[2];                       // gathered batch, two buffers used by alternate steps
   size_t act[MAVG_MAX_LAYERS + 1], act_t[MAVG_MAX_LAYERS + 1];
   size_t dz[MAVG_MAX_LAYERS + 1], dz_t[MAVG_MAX_LAYERS + 1];
   size_t part, part_bytes;
   size_t counters, counters_bytes;
-  size_t w16, wt16, w16g, wt16g;
+  size_t w16, w16g;
   size_t end;
 };
 
@@ -446,17 +448,12 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   const size_t rows = (size_t)P * B;
   t.L = L;
   t.cpad = (cfg->dims[L] + 7) / 8 * 8;
-  int64_t o16 = 0, ot16 = 0;
+  int64_t o16 = 0;
   for (int l = 0; l < L; ++l) {
-    const int in = cfg->dims[l], out = cfg->dims[l + 1];
     t.sh_off[l] = o16;
-    o16 += (int64_t)up((size_t)in * out, 64);
-    t.out_pad[l] = (out + 7) / 8 * 8;
-    t.sht_off[l] = ot16;
-    if (l > 0) ot16 += (int64_t)up((size_t)in * t.out_pad[l], 64);
+    o16 += (int64_t)up((size_t)cfg->dims[l] * cfg->dims[l + 1], 64);
   }
   t.n16 = o16;
-  t.nt16 = ot16 > 0 ? ot16 : 64;
   size_t off = up(base, 1024);
   auto take = [&](size_t bytes) { size_t r = off; off = up(off + bytes, 1024); return r; };
   for (int i = 0; i < 2; ++i) {
@@ -490,9 +487,7 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.counters_bytes = (size_t)P * max_m_tiles * sizeof(int);
   t.counters = take(t.counters_bytes);
   t.w16 = take((size_t)P * t.n16 * 2);
-  t.wt16 = take((size_t)P * t.nt16 * 2);
   t.w16g = take((size_t)t.n16 * 2);
-  t.wt16g = take((size_t)t.nt16 * 2);
   t.end = off;
   return t;
 }
@@ -511,15 +506,14 @@ struct TcState {
   EncodeTiledFn encode = nullptr;
   // per layer l = 1..L (index l)
   CUtensorMap w[MAVG_MAX_LAYERS + 1], wg[MAVG_MAX_LAYERS + 1];       // [out, in] copies
-  CUtensorMap wt[MAVG_MAX_LAYERS + 1], wtg[MAVG_MAX_LAYERS + 1];     // [in, out] copies (l >= 2)
   CUtensorMap act_in[MAVG_MAX_LAYERS + 1];    // [B, d_{l-1}] input activations of layer l >= 2
   CUtensorMap act_in_t[MAVG_MAX_LAYERS + 1];  // [d_{l-1}, B]
   CUtensorMap x_in[2], x_in_t[2];             // layer 1's input: the two gather buffers
   CUtensorMap dz[MAVG_MAX_LAYERS + 1];        // [B, d_l]
   CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
+  CUtensorMap w_mn[MAVG_MAX_LAYERS + 1], wg_mn[MAVG_MAX_LAYERS + 1];  // [out, in] copies, 64 x 64 boxes
   CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
-  CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store views of the bf16 copies
-  CUtensorMap wt16_st[MAVG_MAX_LAYERS + 1];
+  CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap
@@ -642,6 +636,8 @@ mavg_status tc_setup(mavg_ctx* c) {
     __nv_bfloat16* w16g = (__nv_bfloat16*)bf(t.w16g) + t.sh_off[l - 1];
     ok = ok && encode_map(st, &st->w[l], w16, in, out, P, in, t.n16, kBM, &why);
     ok = ok && encode_map(st, &st->wg[l], w16g, in, out, 1, in, t.n16, kBM, &why);
+    ok = ok && encode_map(st, &st->w_mn[l], w16, in, out, P, in, t.n16, 64, &why);
+    ok = ok && encode_map(st, &st->wg_mn[l], w16g, in, out, 1, in, t.n16, 64, &why);
     if (l == 1) {
       for (int i = 0; i < 2 && ok; ++i) {
         ok = ok && encode_map(st, &st->x_in[i], bf(t.xg[i]), in, B, P, in, (int64_t)B * in,
@@ -664,17 +660,8 @@ mavg_status tc_setup(mavg_ctx* c) {
     ok = ok && encode_any(st, &st->w16_st[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w16, in, out, P,
                           in, t.n16, kWgradTileCols, kWgradTileRows, CU_TENSOR_MAP_SWIZZLE_64B,
                           &why);
-    if (l > 1)
-      ok = ok && encode_any(st, &st->wt16_st[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                            (__nv_bfloat16*)bf(t.wt16) + t.sht_off[l - 1], out, in, P,
-                            t.out_pad[l - 1], t.nt16, kWgradTileRows, kWgradTileCols,
-                            CU_TENSOR_MAP_SWIZZLE_NONE, &why);
     if (l > 1) {
       st->dgrad[l] = plan_partial(in, B, out, P, kPlanSmCount, false);
-      __nv_bfloat16* wt16 = (__nv_bfloat16*)bf(t.wt16) + t.sht_off[l - 1];
-      __nv_bfloat16* wt16g = (__nv_bfloat16*)bf(t.wt16g) + t.sht_off[l - 1];
-      ok = ok && encode_map(st, &st->wt[l], wt16, out, in, P, t.out_pad[l - 1], t.nt16, kBM, &why);
-      ok = ok && encode_map(st, &st->wtg[l], wt16g, out, in, 1, t.out_pad[l - 1], t.nt16, kBM, &why);
       ok = ok && encode_map(st, &st->dz[l], bf(t.dz[l]), out, B, P, dz_ld, (int64_t)B * dz_ld,
                             st->dgrad[l].BN, &why);
     }
@@ -732,9 +719,9 @@ cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
     const int64_t total = (int64_t)ly.in * ly.out;
     int grid = (int)std::min<int64_t>((total + 255) / 256, (int64_t)c->sm_count * 8);
     prof_begin(c, MAVG_K_AUX);
-    k_shadow_from_global<<<grid, 256, 0, c->stream>>>(
-        c->buf.global_w, ly.w_off, ly.in, ly.out, (__nv_bfloat16*)(ws + t.w16g), t.sh_off[l - 1],
-        l > 1 ? (__nv_bfloat16*)(ws + t.wt16g) : nullptr, t.sht_off[l - 1], t.out_pad[l - 1]);
+    k_shadow_from_global<<<grid, 256, 0, c->stream>>>(c->buf.global_w, ly.w_off, total,
+                                                      (__nv_bfloat16*)(ws + t.w16g),
+                                                      t.sh_off[l - 1]);
     prof_end(c);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -821,22 +808,20 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.bias_rep = c->buf.replicas; g.bias_off = below.b_off;
       g.out_bm = bfp(t.dz[l - 1]); g.out_mb = bfp(t.dz_t[l - 1]);
       g.mask_mb = bfp(t.act_t[l - 1]);
-      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wtg[l] : st->wt[l], st->dz[l],
-                                    st->dgrad[l], g));
+      g.a_mn = 1;
+      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : st->w_mn[l],
+                                    st->dz[l], st->dgrad[l], g));
     }
     const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
-    const CUtensorMap& wtm = l > 1 ? st->wt16_st[l] : st->w16_st[l];
     if (overlap && l > 1) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
       c->stream = st->s_wgrad;
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l], wtm,
-                                 l > 1));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l]));
       c->stream = main_s;
       side_used = true;
     } else {
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l], wtm,
-                                 l > 1));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l]));
     }
   }
   if (overlap) {

@@ -1,17 +1,17 @@
 // Weight gradient fused with the SGD step of Algorithm 1, as a persistent streaming kernel:
 //   W[o, i] <- W[o, i] - gamma * sum_b dZ[b, o] A[b, i]          (fp32 masters, per learner)
-// and the refreshed bf16 copies of W ([out, in] and, for layers >= 2, [in, out]).
+// and the refreshed bf16 copy of W that the forward and dgrad products read.
 //
 // The contraction is only as long as the batch, so the kernel is a read-modify-write stream over
-// the masters (10-12 bytes per weight) and is built around bulk copies, not around the MMA:
+// the masters (10 bytes per weight) and is built around bulk copies, not around the MMA:
 //   producer warp   TMA-loads, per 128 x 32 weight tile, the fp32 master tile and the 32 x B tile
 //                   of A^T into a ring of shared-memory slots; the 128 x B tile of dZ^T is loaded
 //                   once per work item (a run of column tiles of one learner and row tile);
 //   MMA warp        one thread issues tcgen05.mma (M=128, N=32, K=B) into one of two TMEM buffers;
 //   2 x 4 epilogue warps (one group per TMEM buffer, i.e. per tile parity) read the accumulator
 //                   (tcgen05.ld, one weight row per lane), update the master tile in place in
-//                   shared memory and write the bf16 tiles beside it;
-//   store warp      one thread sends the three finished tiles back with TMA stores and frees the
+//                   shared memory and write the bf16 tile beside it;
+//   store warp      one thread sends the two finished tiles back with TMA stores and frees the
 //                   slot once they have left shared memory.
 // Edge tiles need no predicates: TMA zero-fills loads and clips stores at the tensor bounds.
 #include <cuda.h>
@@ -27,10 +27,9 @@ using namespace tc;
 
 constexpr int kBM = 128, kBN = 32, kBK = 64;
 constexpr int kThreads = 352;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores
-constexpr int kMaxSlots = 4;
+constexpr int kMaxSlots = 6;
 constexpr int kW32Bytes = kBM * kBN * 4;  // 16 KB, rows of 128 bytes, 128-byte swizzle
 constexpr int kW16Bytes = kBM * kBN * 2;  //  8 KB, rows of  64 bytes,  64-byte swizzle
-constexpr int kWtBytes = kBN * kBM * 2;   //  8 KB, rows of 256 bytes, no swizzle
 enum { ERR_WG_PRODUCER = 21, ERR_WG_MMA = 22, ERR_WG_EPILOGUE = 23, ERR_WG_STORE = 24 };
 
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* src, int c0, int c1,
@@ -60,7 +59,6 @@ struct WgradArgs {
   int items;               // P * m_tiles * n_chunks
   int slots;               // ring depth
   int a_bufs;              // 1 or 2 buffers for the dZ^T tile
-  int has_wt;
   float gamma;
   int* status;
 };
@@ -70,7 +68,6 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
                    const __grid_constant__ CUtensorMap tm_at,    // bf16 [P, in, B]   load
                    const __grid_constant__ CUtensorMap tm_w32,   // fp32 [P, out, in] load + store
                    const __grid_constant__ CUtensorMap tm_w16,   // bf16 [P, out, in] store
-                   const __grid_constant__ CUtensorMap tm_wt16,  // bf16 [P, in, out] store
                    const WgradArgs g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
@@ -84,7 +81,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
   const int b_bytes = g.nkb * kBN * kBK * 2;         // A^T tile:  nkb slabs of 4 KB
-  const int slot_bytes = kW32Bytes + kW16Bytes + kWtBytes + b_bytes;   // multiple of 1024
+  const int slot_bytes = kW32Bytes + kW16Bytes + b_bytes;   // multiple of 1024
   uint8_t* a_base = smem;
   uint8_t* slot_base = smem + (size_t)g.a_bufs * a_bytes;
 
@@ -94,7 +91,6 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     tma_prefetch_desc(&tm_at);
     tma_prefetch_desc(&tm_w32);
     tma_prefetch_desc(&tm_w16);
-    if (g.has_wt) tma_prefetch_desc(&tm_wt16);
     for (int s = 0; s < g.slots; ++s) {
       mbar_init(&slot_full[s], 1);
       mbar_init(&slot_empty[s], 1);
@@ -158,7 +154,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           mbar_arrive_expect_tx(&slot_full[s], (uint32_t)(kW32Bytes + b_bytes));
           tma_load_3d(sl, &tm_w32, &slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
-            tma_load_3d(sl + kW32Bytes + kW16Bytes + kWtBytes + (size_t)kb * (kBN * kBK * 2),
+            tma_load_3d(sl + kW32Bytes + kW16Bytes + (size_t)kb * (kBN * kBK * 2),
                         &tm_at, &slot_full[s], kb * kBK, i0, p);
         }
       }
@@ -188,7 +184,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           }
           tc_fence_after_sync();
           const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + kW32Bytes +
-                                           kW16Bytes + kWtBytes);
+                                           kW16Bytes);
           for (int kb = 0; kb < g.nkb; ++kb) {
             const uint64_t adesc = smem_desc_k_sw128(a_addr + kb * (kBM * kBK * 2));
             const uint64_t bdesc = smem_desc_k_sw128(b_addr + kb * (kBN * kBK * 2));
@@ -234,7 +230,6 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
         uint8_t* sl = slot_base + (size_t)s * slot_bytes;
         uint8_t* w32 = sl + (size_t)r * 128;             // 8 chunks of 16 B, chunk c at c ^ (r & 7)
         uint8_t* w16 = sl + kW32Bytes + (size_t)r * 64;  // 4 chunks, chunk c at c ^ ((r >> 1) & 3)
-        uint8_t* wt = sl + kW32Bytes + kW16Bytes + (size_t)r * 2;   // [in i][out r], 256 B rows
         uint32_t hp[16];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -254,11 +249,6 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
         for (int c = 0; c < 4; ++c)
           *reinterpret_cast<uint4*>(w16 + ((c ^ ((r >> 1) & 3)) << 4)) =
               make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
-        if (g.has_wt) {
-          const uint16_t* hh = reinterpret_cast<const uint16_t*>(hp);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) *reinterpret_cast<uint16_t*>(wt + (size_t)i * 256) = hh[i];
-        }
         fence_proxy_async();                   // generic-proxy writes -> visible to the TMA stores
         __syncwarp();
         if (lane == 0) mbar_arrive(&out_full[s]);
@@ -282,7 +272,6 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           const int i0 = (nt0 + j) * kBN;
           tma_store_3d(&tm_w32, sl, i0, m0, p);
           tma_store_3d(&tm_w16, sl + kW32Bytes, i0, m0, p);
-          if (g.has_wt) tma_store_3d(&tm_wt16, sl + kW32Bytes + kW16Bytes, m0, i0, p);
           tma_store_commit();
           // the slot of the previous tile is free once its stores have read shared memory
           if (tile_ctr > 0) {
@@ -317,7 +306,7 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count) {
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
   w.items = P * w.m_tiles * w.n_chunks;
   const int a_bytes = w.nkb * kBM * kBK * 2;
-  const int slot_bytes = kW32Bytes + kW16Bytes + kWtBytes + w.nkb * kBN * kBK * 2;
+  const int slot_bytes = kW32Bytes + kW16Bytes + w.nkb * kBN * kBK * 2;
   const int budget = 220 * 1024;
   w.a_bufs = 2;
   w.slots = (budget - 2 * a_bytes) / slot_bytes;
@@ -338,7 +327,7 @@ cudaError_t wgrad_stream_prepare() {
 
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16, const CUtensorMap& wt16, bool has_wt) {
+                                const CUtensorMap& w16) {
   WgradArgs g{};
   g.nkb = w.nkb;
   g.m_tiles = w.m_tiles;
@@ -348,7 +337,6 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   g.items = w.items;
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
-  g.has_wt = has_wt ? 1 : 0;
   g.gamma = c->cfg.local_lr;
   g.status = (int*)ws_ptr(c, c->ws.status);
   cudaLaunchConfig_t lc{};
@@ -362,7 +350,7 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   lc.attrs = at_;
   lc.numAttrs = 1;
   prof_begin(c, MAVG_K_WGRAD_SGD);
-  cudaError_t e = cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream, dzt, at, w32, w16, wt16, g);
+  cudaError_t e = cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream, dzt, at, w32, w16, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -18,9 +18,9 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count);
 cudaError_t wgrad_stream_prepare();
 // dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
 // w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128
-// (64B swizzle); wt16: bf16 [P, in, out] box 128 x 32 (no swizzle), ignored unless has_wt.
+// (64B swizzle).
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16, const CUtensorMap& wt16, bool has_wt);
+                                const CUtensorMap& w16);
 
 }  // namespace mavg

@@ -153,6 +153,18 @@ def run_reference(args):
     return 0
 
 
+# DRAM read + write bytes per launch, averaged over the launches of a class in one local step of
+# the C2 workload, from the ncu capture summarised in profiles/step_kernels_c2.md (cold cache:
+# ncu flushes L2 before every kernel; in a running round most of this workload's 90 MB of state
+# stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
+# captured; set an entry to None when its kernel changes.
+NCU_TRAFFIC_C2 = {
+    "wgrad_sgd_gemm": (57.709312e6 + 21.674752e6 + 10.521344e6 + 0.009728e6 + 1.326080e6) / 3,
+    "fwd_gemm": (31.535360e6 + 5.321216e6 + 1.273600e6) / 3,
+    "dgrad_gemm": (1.305088e6 + 6.372608e6) / 2,
+}
+
+
 def kernel_rooflines(cfg, prof, steps, peaks, tensor_path):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
@@ -396,6 +408,8 @@ def run_mavg(args):
                         "unit": "GB/s", "frac": e["frac_hbm"], "traffic": None}
             roof["kernel"] = dom
             roof["peak_source"] = peaks["source"]
+            if args.workload == "C2" and mode == 1 and not args.learners:
+                roof["traffic"] = NCU_TRAFFIC_C2.get(dom)
         sweep = meta_update_sweep(m, torch, peaks) if world == 1 and not args.no_sweep else None
         n = g.n
         line = {

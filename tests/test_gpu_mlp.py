@@ -151,3 +151,71 @@ def test_bf16_teacher_forced_step(oracle):
             _check_update(step_g, step_o)
         assert np.abs(g.get_losses() - losses_o).max() <= 2e-3 * losses_o.max()
         g.close()
+
+
+def _tc_handle(cfg_over=None, K=3):
+    m = _mavg()
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(dims=[3072, 256, 128, 10], P=4, K=K, B=64, S=2048)
+    if cfg_over:
+        cfg.update(cfg_over)
+    x, y = m.workloads.make_dataset(cfg, S=cfg["S"])
+    w1 = m.workloads.mlp_init(cfg["dims"])
+    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+               seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1,
+               x=x, y=y, x_bf16=True)
+    return g
+
+
+def test_tc_path_is_deterministic_and_graph_equals_launch_by_launch():
+    # two runs give the same bits (fixed reduction orders, no atomics on the value path), and the
+    # replayed CUDA graph with its overlapped branches computes exactly what the serial,
+    # launch-by-launch schedule (taken while per-launch profiling is on) computes
+    outs = []
+    for profiled in (False, False, True):
+        g = _tc_handle()
+        g.set_profiling(profiled)
+        losses = [g.round(want_loss=True) for _ in range(3)]
+        g.sync()
+        outs.append((g.w.cpu().numpy(), g.v.cpu().numpy(), losses))
+        if profiled:
+            prof = g.get_profile()
+            assert prof["wgrad_sgd_gemm"][1] == 3 * 3 * 3 and prof["meta_update"][1] == 3
+        g.close()
+    for other in outs[1:]:
+        assert np.array_equal(outs[0][0], other[0]) and np.array_equal(outs[0][1], other[1])
+        assert outs[0][2] == other[2]
+
+
+def test_tc_hparam_change_and_repeated_local_steps():
+    # K and the learning rate may change between rounds (the recorded graph is rebuilt)
+    a = _tc_handle(K=2)
+    a.round(); a.set_hparams(3, 0.02, 1.0, 0.5); a.round(); a.round()
+    a.sync()
+    b = _tc_handle(K=2)
+    b.set_profiling(True)           # launch-by-launch reference for the same schedule of calls
+    b.round(); b.set_hparams(3, 0.02, 1.0, 0.5); b.round(); b.round()
+    b.sync()
+    assert np.array_equal(a.w.cpu().numpy(), b.w.cpu().numpy())
+    assert a.get_round() == 3
+    # a second call without a meta-update in between starts from diverged replicas: it must take
+    # the per-learner weight copies, not the shared copy of w~ -- compare graph and serial paths
+    c = _tc_handle(K=2)
+    c.local_steps(); c.local_steps(); c.sync()
+    d = _tc_handle(K=2)
+    d.set_profiling(True)
+    d.local_steps(); d.local_steps(); d.sync()
+    rc = c.replicas.cpu().numpy()
+    assert np.array_equal(rc, d.replicas.cpu().numpy()) and np.isfinite(rc).all()
+    assert not np.array_equal(rc[0], rc[1])
+    # K lowered through set_hparams gives the same steps as a handle created with that K
+    e = _tc_handle(K=2)
+    e.local_steps(); e.sync()
+    f = _tc_handle(K=4)
+    f.set_hparams(2, 0.05, 1.0, 0.9)
+    f.local_steps(); f.sync()
+    assert np.array_equal(e.replicas.cpu().numpy(), f.replicas.cpu().numpy())
+    with pytest.raises(_mavg().MavgError):
+        a.set_hparams(0, 0.05, 1.0, 0.9)
+    with pytest.raises(_mavg().MavgError):
+        a.set_hparams(2, 0.05, 1.0, 1.0)

@@ -55,7 +55,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-i", str(self.gpu), "-lms", "100"], stdout=self.f,
+                                       "-i", str(self.gpu), "-lms", "50"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -130,14 +130,20 @@ def run_reference(args):
     if rank != 0:
         return 0
     cfg, x, y, w1 = workload_inputs()
+    # Bounded sample per step: one of the K local steps on p_s of the P learners (+ their
+    # meta-update), p_s sized from one calibration step so that the whole run stays near 100 s.
     k_sample = 1
+    one = dict(cfg, P=1)
+    _, _, t_cal = cpu_oracle_rate(one, x, y, w1, k_sample, reps=1)
     total = args.warmup + args.steps
-    rate, threads, times = cpu_oracle_rate(cfg, x, y, w1, k_sample, reps=total)
+    p_s = int(max(1, min(cfg["P"], 100.0 / max(total, 1) / max(t_cal[0], 1e-6))))
+    sub = dict(cfg, P=p_s)
+    rate, threads, times = cpu_oracle_rate(sub, x, y, w1, k_sample, reps=total)
     timed = times[args.warmup:]
-    units = cfg["P"] * k_sample * cfg["B"]
+    units = p_s * k_sample * cfg["B"]
     value = units * len(timed) / sum(timed)
-    sample = (f"each step = 1 of the {cfg['K']} local steps on all {cfg['P']} learners "
-              f"(B={cfg['B']}) + the meta-update = {units} learner-samples")
+    sample = (f"each step = 1 of the {cfg['K']} local steps on {p_s} of the {cfg['P']} learners "
+              f"(B={cfg['B']}) + their meta-update = {units} learner-samples")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(timed) / len(timed),
@@ -449,7 +455,7 @@ def run_mavg(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mavg", choices=["mavg", "reference"])
     ap.add_argument("--gemm", type=int, default=1, choices=[1, 2],

@@ -219,3 +219,38 @@ def test_tc_hparam_change_and_repeated_local_steps():
         a.set_hparams(0, 0.05, 1.0, 0.9)
     with pytest.raises(_mavg().MavgError):
         a.set_hparams(2, 0.05, 1.0, 1.0)
+
+
+@pytest.mark.parametrize("dims,B,P,K", [
+    ([64, 10], 16, 1, 2),                    # one layer, smallest batch
+    ([72, 40, 24, 10], 48, 3, 2),            # widths that are multiples of 8 only; ragged tiles
+    ([200, 136, 10], 32, 2, 3),              # in/out not multiples of 64 or 128
+    ([1024, 384, 32], 256, 2, 2),            # largest batch, 32 classes, 3 row tiles
+    ([4104, 128, 128, 128, 128, 8], 64, 2, 2),   # long contraction (65 slabs, ragged), 5 layers
+    ([512, 1152, 16], 128, 5, 2),            # 9 row tiles x 5 learners
+])
+def test_tc_shapes_teacher_forced(oracle, dims, B, P, K):
+    # tensor-core path on shapes that exercise ragged tiles, contraction tails, batch tiling and
+    # contraction splits; K local steps from identical replicas against the oracle, per learner
+    m = _mavg()
+    S = max(4 * P * B, 512)
+    r = np.random.default_rng(17)
+    x = r.standard_normal((S, dims[0])).astype(np.float32)
+    y = r.integers(0, dims[-1], S).astype(np.int32)
+    w1 = m.workloads.mlp_init(dims, seed=5)
+    g = m.Mavg(w1, P=P, K=K, local_lr=0.05, mu=0.9, B=B, seed=99, objective=m.OBJ_MLP, dims=dims,
+               gemm_bf16=1, x=x, y=y)
+    o = oracle.Mavg(w1, P=P, K=K, gamma=0.05, mu=0.9, B=B, seed=99, objective=oracle.OBJ_MLP,
+                    dims=dims, bf16=True, x=x, y=y, stride=g.stride)
+    g.local_steps()
+    losses_o, _ = o.local_steps()
+    g.sync()
+    gr = g.replicas.cpu().numpy()
+    assert np.abs(g.get_losses() - losses_o).max() <= 2e-2 * losses_o.max()
+    for j in range(P):
+        step_g = gr[j, :g.n].astype(np.float64) - w1
+        step_o = o.replicas[j, :g.n].astype(np.float64) - w1
+        assert l2_rel(step_g, step_o) <= 3e-2, j
+    lg = g.round(want_loss=True)       # and a full round on top: finite, graph path
+    assert np.isfinite(lg) and torch.isfinite(g.w).all()
+    g.close()

@@ -207,6 +207,32 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const int q = warp & 3;
     const int half = ew >> 2;
     const int row = q * 32 + lane;
+    // Operands of the tail that do not depend on the accumulator are fetched while the main loop
+    // is still running: the bias (read by the forward tails, stepped by the dgrad tail), the
+    // first mask chunk (dgrad) and the label of this thread's batch row (last layer).
+    float* bias = g.bias_rep + (size_t)p * g.rep_stride + g.bias_off;
+    const bool m_ok_pre = m0 + row < g.M;
+    const float bias_pre = (m_ok_pre && (EPI != EPI_DGRAD || half == 0)) ? bias[m0 + row] : 0.f;
+    uint4 mk[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
+                   make_uint4(0, 0, 0, 0)};
+    auto load_mask = [&](int c0, uint4 (&dst)[4]) {
+      if (!m_ok_pre || c0 >= g.BN) return;
+      const uint4* msrc = reinterpret_cast<const uint4*>(
+          g.mask_mb + ((size_t)p * g.M + m0 + row) * g.N + n0 + c0);
+      if (n0 + c0 + 32 <= g.N) {               // whole chunk inside the batch: 4 loads in flight
+#pragma unroll
+        for (int v = 0; v < 4; ++v) dst[v] = msrc[v];
+      } else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          dst[v] = n0 + c0 + v * 8 < g.N ? msrc[v] : make_uint4(0, 0, 0, 0);
+      }
+    };
+    // (only in the one-block-per-SM build: the register-capped build has no room to hold it)
+    if (EPI == EPI_DGRAD && MINB == 1) load_mask(half * 32, mk);
+    int label_pre = 0;
+    if (EPI == EPI_FWD_LAST && ew * 32 + lane < g.N)
+      label_pre = g.labels[(size_t)p * g.N + ew * 32 + lane];
     const bool ok = mbar_wait(&acc_bar, 0, abortp, g.status, ERR_EPILOGUE);
     tc_fence_after_sync();
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -216,7 +242,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       const int m = m0 + row;
       const bool m_ok = m < g.M;
       bool finisher = ok;
-      if (g.splits > 1) {
+      if (MINB == 1 && g.splits > 1) {   // the register-capped build is never used with a split
         if (ok) {
           float* dst = g.part + ((size_t)(split * g.P + p) * g.N) * g.M + m;
           for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
@@ -244,14 +270,13 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         finisher = last_flag != 0;
       }
       if (finisher) {
-        float* bias = g.bias_rep + (size_t)p * g.rep_stride + g.bias_off;
-        const float my_bias = (EPI != EPI_DGRAD && m_ok) ? bias[m] : 0.f;
+        const float my_bias = EPI != EPI_DGRAD ? bias_pre : 0.f;
         float dsum = 0.f;
         float* lg = reinterpret_cast<float*>(smem);          // last layer: logits [N][M]
         for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
           float z[32];
           int ncols;
-          if (g.splits == 1) {
+          if (MINB != 1 || g.splits == 1) {
             ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
           } else {
             ncols = min(32, g.BN - c0);
@@ -285,19 +310,20 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           } else {
             uint32_t hp[16];                                  // 32 bf16 results, packed
             if (EPI == EPI_DGRAD) {
-              uint4 mk[4];
-              const uint4* msrc = reinterpret_cast<const uint4*>(
-                  g.mask_mb + ((size_t)p * g.M + (m_ok ? m : 0)) * g.N + n0 + c0);
-#pragma unroll
-              for (int v = 0; v < 4; ++v)
-                mk[v] = (m_ok && v * 8 < ncols && n0 + c0 + v * 8 < g.N) ? msrc[v]
-                                                                    : make_uint4(0, 0, 0, 0);
+              uint4 mkn[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
+                              make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+              if (MINB == 1) load_mask(c0 + 64, mkn);         // next chunk, used one iteration on
+              else load_mask(c0, mk);
               const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(mk);
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
                 const bool live = j < ncols && n0 + c0 + j < g.N && __bfloat162float(mh[j]) > 0.f;
                 z[j] = live ? z[j] : 0.f;                     // ReLU'(0) = 0
                 dsum += z[j];
+              }
+              if (MINB == 1) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v) mk[v] = mkn[v];
               }
             } else {
 #pragma unroll
@@ -314,14 +340,22 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             if (m_ok) {
               const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
               __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + c0) * g.M + m;
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols && n0 + c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
               uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + c0);
+              if (ncols == 32 && n0 + c0 + 32 <= g.N) {
 #pragma unroll
-              for (int v = 0; v < 4; ++v)
-                if (v * 8 < ncols && n0 + c0 + v * 8 < g.N)
+                for (int v = 0; v < 4; ++v)
                   dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dbm[(size_t)j * g.M] = hh[j];
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (j < ncols && n0 + c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                  if (v * 8 < ncols && n0 + c0 + v * 8 < g.N)
+                    dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
+              }
             }
           }
         }
@@ -331,7 +365,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           colsum[half][row] = dsum;
           epilogue_barrier();
           if (half == 0 && m_ok)
-            bias[m] = fmaf(-g.gamma, colsum[0][row] + colsum[1][row], bias[m]);
+            bias[m] = fmaf(-g.gamma, colsum[0][row] + colsum[1][row], bias_pre);
         }
         if (EPI == EPI_FWD_LAST) {
           // softmax cross-entropy on the block's [N, M] logits: thread t takes batch row t
@@ -347,7 +381,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             float se = 0.f;
             for (int c = 0; c < C; ++c) se += expf(zr[c] - mx);
             const float lse = mx + logf(se);
-            const int yb = g.labels[(size_t)p * g.N + t];
+            const int yb = label_pre;
             lossp[t] = lse - zr[yb];
             const float inv_b = 1.0f / (float)g.N;
             for (int c = 0; c < C; ++c) {
@@ -359,15 +393,27 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
           }
           epilogue_barrier();
+          // loss: every warp adds its 32 rows, thread 0 the warps' sums; bias gradient of class c:
+          // a warp adds the rows lane, lane + 32, ... and then its lanes, in a fixed order
+          {
+            float sl = t < g.N ? lossp[t] : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sl += __shfl_xor_sync(0xffffffffu, sl, o);
+            if (lane == 0) colsum[0][ew] = sl;
+            for (int c = ew; c < C; c += 8) {
+              float sb = 0.f;
+              for (int b = lane; b < g.N; b += 32) sb += dzs[b * C + c];
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
+              if (lane == 0) bias[c] = fmaf(-g.gamma, sb, bias[c]);
+            }
+          }
+          epilogue_barrier();
           if (t == 0) {
             float sl = 0.f;
-            for (int b = 0; b < g.N; ++b) sl += lossp[b];
+            const int nw = (g.N + 31) / 32;
+            for (int w = 0; w < nw; ++w) sl += colsum[0][w];
             g.loss_out[(size_t)p * g.loss_stride] = sl / (float)g.N;
-          }
-          if (t < C) {
-            float sb = 0.f;
-            for (int b = 0; b < g.N; ++b) sb += dzs[b * C + t];
-            bias[t] = fmaf(-g.gamma, sb, bias[t]);
           }
         }
       }
@@ -432,7 +478,7 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   int stage_bytes = kATileBytes + g.BN * kBK * 2;
   // more blocks than SMs: two blocks share an SM, so that one block's set-up and tail overlap
   // the other's main loop; otherwise one block takes the whole shared memory
-  g.two_per_sm = g.m_tiles * g.n_tiles * g.splits * P > sm_count ? 1 : 0;
+  g.two_per_sm = (g.splits == 1 && g.m_tiles * g.n_tiles * P > sm_count) ? 1 : 0;
   const int budget = g.two_per_sm ? 104 * 1024 : 200 * 1024;
   g.stages = budget / stage_bytes;
   if (g.stages > kMaxStages) g.stages = kMaxStages;

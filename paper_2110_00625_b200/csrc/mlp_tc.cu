@@ -229,7 +229,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       }
     };
     // (only in the one-block-per-SM build: the register-capped build has no room to hold it)
-    if (EPI == EPI_DGRAD && MINB == 1) load_mask(half * 32, mk);
+    if (EPI == EPI_DGRAD) load_mask(half * 32, mk);
     int label_pre = 0;
     if (EPI == EPI_FWD_LAST && ew * 32 + lane < g.N)
       label_pre = g.labels[(size_t)p * g.N + ew * 32 + lane];
@@ -312,8 +312,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             if (EPI == EPI_DGRAD) {
               uint4 mkn[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
                               make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-              if (MINB == 1) load_mask(c0 + 64, mkn);         // next chunk, used one iteration on
-              else load_mask(c0, mk);
+              load_mask(c0 + 64, mkn);                        // next chunk, used one iteration on
               const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(mk);
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
@@ -321,10 +320,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 z[j] = live ? z[j] : 0.f;                     // ReLU'(0) = 0
                 dsum += z[j];
               }
-              if (MINB == 1) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v) mk[v] = mkn[v];
-              }
+              for (int v = 0; v < 4; ++v) mk[v] = mkn[v];
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j) {

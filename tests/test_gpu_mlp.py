@@ -254,3 +254,25 @@ def test_tc_shapes_teacher_forced(oracle, dims, B, P, K):
     lg = g.round(want_loss=True)       # and a full round on top: finite, graph path
     assert np.isfinite(lg) and torch.isfinite(g.w).all()
     g.close()
+
+
+def test_training_converges_and_block_momentum_accelerates():
+    # end-to-end sanity on the CIFAR-shaped data: the training loss falls over the rounds, and
+    # with the same number of rounds M-AVG (mu = 0.7) is ahead of K-AVG (mu = 0), the paper's
+    # central claim (qualitative: no number of the paper is reproduced here)
+    m = _mavg()
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(dims=[3072, 256, 256, 10], P=12, K=8, B=64, S=20000)
+    x, y = m.workloads.make_dataset(cfg, S=cfg["S"])
+    w1 = m.workloads.mlp_init(cfg["dims"])
+    final = {}
+    for mu in (0.0, 0.7):
+        g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=0.02, mu=mu, B=cfg["B"],
+                   seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1,
+                   x=x, y=y, x_bf16=True)
+        losses = [g.round(want_loss=True) for _ in range(60)]
+        assert np.isfinite(losses).all()
+        assert losses[-1] < 0.8 * losses[0]
+        final[mu] = float(np.mean(losses[-5:]))
+        g.close()
+    assert final[0.7] < final[0.0]

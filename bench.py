@@ -165,9 +165,9 @@ def run_reference(args):
 # stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
 # captured; set an entry to None when its kernel changes.
 NCU_TRAFFIC_C2 = {
-    "wgrad_sgd_gemm": (57.709312e6 + 21.674752e6 + 10.521344e6 + 0.009728e6 + 1.326080e6) / 3,
-    "fwd_gemm": (31.535360e6 + 5.321216e6 + 1.273600e6) / 3,
-    "dgrad_gemm": (1.305088e6 + 6.372608e6) / 2,
+    "wgrad_sgd_gemm": (57.709312e6 + 20.414720e6 + 10.521344e6 + 0.011776e6 + 1.326336e6) / 3,
+    "fwd_gemm": (31.539200e6 + 5.325568e6 + 1.273856e6) / 3,
+    "dgrad_gemm": (1.313280e6 + 6.380800e6) / 2,
 }
 
 

@@ -171,7 +171,7 @@ NCU_TRAFFIC_C2 = {
 }
 
 
-def kernel_rooflines(cfg, prof, steps, peaks, tensor_path):
+def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
@@ -180,15 +180,17 @@ def kernel_rooflines(cfg, prof, steps, peaks, tensor_path):
     rows = P * B
     out = {}
     per_round = {
-        # replicas, w~, v read; v, w~, replicas written
-        "meta_update": dict(bytes=(8 * P + 16) * n, flops=0),
+        # replicas, w~, v read; v, w~ and (unless the copies are deferred) the replicas written
+        "meta_update": dict(bytes=((4 if deferred else 8) * P + 16) * n, flops=0),
         # bf16 weights read once per learner and step; activations in and out
         "fwd_gemm": dict(bytes=K * (2 * P * sum(nW) + 2 * rows * (sum(dims[:-1]) + 2 * sum(dims[1:]))),
                          flops=K * 2 * rows * sum(nW)),
         "dgrad_gemm": dict(bytes=K * (2 * P * sum(nW[1:]) + 2 * rows * (sum(dims[2:]) + 3 * sum(dims[1:-1]))),
                            flops=K * 2 * rows * sum(nW[1:])),
-        # fp32 master read + written, bf16 copy written
-        "wgrad_sgd_gemm": dict(bytes=K * (P * 10 * sum(nW) + 2 * rows * sum(dims)),
+        # fp32 master read + written, bf16 copy written; on the tensor-core path the first step
+        # of a round reads the one copy of w~ instead of P masters
+        "wgrad_sgd_gemm": dict(bytes=K * (P * 10 * sum(nW) + 2 * rows * sum(dims))
+                               - (4 * (P - 1) * sum(nW) if tensor_path else 0),
                                flops=K * 2 * rows * sum(nW)),
     }
     for name, (ms, cnt) in prof.items():
@@ -268,7 +270,7 @@ def run_pseudograd(args, m, torch, peaks, rank):
     out = []
     for K in cfg["K"]:
         g = m.Mavg(w1, P=P, K=K, local_lr=cfg["gamma"], mu=0.9, seed=W.BASE_SEED,
-                   objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"])
+                   objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"], defer_broadcast=not args.no_defer)
         for _ in range(3):
             g.round()
         g.sync()
@@ -278,12 +280,16 @@ def run_pseudograd(args, m, torch, peaks, rank):
         torch.cuda.synchronize()
         loc = statistics.median(a.elapsed_time(b) for a, b, c in ev)
         met = statistics.median(b.elapsed_time(c) for a, b, c in ev)
+        # the local pass reads w~ once (every learner starts from it) and writes P learner models;
+        # the meta-update reads them with w~ and v and writes w~, v and, unless deferred, P copies
+        meta_b = ((8 if args.no_defer else 4) * P + 16) * n
         out.append(dict(K=K, local_ms=loc, meta_ms=met, round_ms=loc + met,
                         learner_steps_per_s=P * K / ((loc + met) * 1e-3),
-                        local_gbs=8 * P * n / loc / 1e6,
+                        local_gbs=(4 * P + 4) * n / loc / 1e6,
                         variates_per_s=P * K * n / (loc * 1e-3),
-                        meta_gbs=(8 * P + 16) * n / met / 1e6,
-                        meta_frac_measured=(8 * P + 16) * n / met / 1e6 / peaks["hbm_gbs"]))
+                        meta_gbs=meta_b / met / 1e6,
+                        meta_frac_measured=meta_b / met / 1e6 / peaks["hbm_gbs"],
+                        defer_broadcast=not args.no_defer))
         g.close()
         del g
         torch.cuda.empty_cache()
@@ -329,7 +335,8 @@ def run_mavg(args):
     mode = args.gemm
     g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"],
                block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
-               dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}")
+               dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}",
+               defer_broadcast=not args.no_defer)
     units = cfg["P"] * cfg["K"] * cfg["B"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
 
@@ -389,7 +396,7 @@ def run_mavg(args):
         g.round()
     prof = g.get_profile(reset=True)
     g.set_profiling(False)
-    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1)
+    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1, deferred=not args.no_defer)
 
     total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=g.device)
 
@@ -429,6 +436,7 @@ def run_mavg(args):
                        "global_batch": cfg["P"] * cfg["B"], "parallelism": "replicas only",
                        "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
                                 0: "CUDA cores fp32"}[mode],
+                       "defer_broadcast": not args.no_defer,
                        "l2": "flushed between steps by a 256 MiB memset outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
@@ -469,6 +477,9 @@ def main():
                     help="run only the meta-update sweep (profiler captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-defer", action="store_true",
+                    help="write the P copies of w~ in the meta-update instead of folding them into "
+                         "the next round's first local step")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "mavg":
         args.warmup = 3

@@ -94,6 +94,14 @@ typedef struct {
   const int32_t *y;  /* DEVICE [n_samples] labels in [0, dims[n_layers]) */
   int64_t n_samples; /* S >= P, < 2^31 */
   void *stream;      /* cudaStream_t (NULL = the legacy default stream) */
+  int32_t defer_broadcast; /* 0: "set w^j = w~" is carried out as P copies by mavg_create,
+                        mavg_meta_update, mavg_set_round and mavg_round_host (the replica array
+                        then equals w~ between rounds).  1: those calls leave the replica array
+                        untouched; the first local step of the next round reads w~ in place of
+                        every w^j and writes each learner's own result, which is the same
+                        assignment with 4P bytes per element less traffic.  Between a meta-update
+                        and the next local step the replica array then holds the previous round's
+                        learner models; mavg_materialize_replicas writes the copies on request. */
 } mavg_config;
 
 /* Caller-owned DEVICE buffers.  Every base pointer must be 16-byte aligned. */
@@ -110,7 +118,8 @@ typedef struct {
  * loss accumulators, the device status word).  Checks the configuration like mavg_create. */
 mavg_status mavg_workspace_bytes(const mavg_config *cfg, size_t *out_bytes);
 
-/* Algorithm 1, the two initialisation lines and the first "set w^j = w~": v <- 0, w^j <- w~_1.
+/* Algorithm 1, the two initialisation lines and the first "set w^j = w~": v <- 0, w^j <- w~_1
+ * (the copies are skipped with defer_broadcast, see there).
  * Validates everything; on failure *out is NULL.  Enqueues the initialisation on the stream. */
 mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_handle *out);
 
@@ -119,8 +128,14 @@ mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_ha
 mavg_status mavg_local_steps(mavg_handle h);
 
 /* Meta level of Algorithm 1 (a, d, v, w~) fused with the re-broadcast w^j <- w~ that opens the
- * next round; advances the round counter. */
+ * next round (folded into the next local step instead with defer_broadcast); advances the round
+ * counter. */
 mavg_status mavg_meta_update(mavg_handle h);
+
+/* With defer_broadcast: writes w^j <- w~ into the replica array now if the handle is at a round
+ * boundary and has not done so yet (a caller that wants to read the P copies).  Otherwise, and
+ * without defer_broadcast, a no-op. */
+mavg_status mavg_materialize_replicas(mavg_handle h);
 
 /* One round = mavg_local_steps then mavg_meta_update.  If mean_loss is not NULL (HOST, one
  * float) the call waits for the stream and stores the mean of the round's P*K minibatch losses

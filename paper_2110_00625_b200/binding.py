@@ -17,7 +17,7 @@ STATUS = {0: "MAVG_OK", 1: "MAVG_ERR_INVALID_ARG", 2: "MAVG_ERR_BAD_BUFFER", 3: 
           4: "MAVG_ERR_UNSUPPORTED", 5: "MAVG_ERR_CUDA", 6: "MAVG_ERR_TIMEOUT"}
 
 EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta_update",
-           "mavg_round", "mavg_round_host", "mavg_set_hparams", "mavg_get_batch_indices",
+           "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
            "mavg_set_profiling", "mavg_get_profile", "mavg_sync", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
@@ -36,6 +36,7 @@ class Config(C.Structure):
         ("pseudo_grad_sigma", C.c_float),
         ("x", C.c_void_p), ("x_dtype", C.c_int32), ("y", C.c_void_p), ("n_samples", C.c_int64),
         ("stream", C.c_void_p),
+        ("defer_broadcast", C.c_int32),
     ]
 
 
@@ -88,6 +89,7 @@ def load_library():
     L.mavg_batch_indices_noalloc.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_int64, C.c_int32, C.c_void_p,
                                              C.c_void_p]
+    L.mavg_materialize_replicas.argtypes = [H]
     L.mavg_sync.argtypes = [H]
     L.mavg_last_error.argtypes = [H]
     L.mavg_last_error.restype = C.c_char_p
@@ -100,7 +102,8 @@ def load_library():
 
 
 def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE, n=0, dims=None,
-                gemm_bf16=0, sigma=0.0, x_ptr=0, x_dtype=X_F32, y_ptr=0, n_samples=0, stream=0):
+                gemm_bf16=0, sigma=0.0, x_ptr=0, x_dtype=X_F32, y_ptr=0, n_samples=0, stream=0,
+                defer_broadcast=False):
     cfg = Config()
     cfg.P, cfg.K, cfg.B = P, K, B
     cfg.local_lr, cfg.block_lr, cfg.mu = local_lr, block_lr, mu
@@ -115,6 +118,7 @@ def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NON
     cfg.pseudo_grad_sigma = sigma
     cfg.x, cfg.x_dtype, cfg.y, cfg.n_samples = x_ptr, x_dtype, y_ptr, n_samples
     cfg.stream = stream
+    cfg.defer_broadcast = 1 if defer_broadcast else 0
     return cfg
 
 
@@ -140,7 +144,7 @@ class Mavg:
 
     def __init__(self, w1, P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE,
                  dims=None, gemm_bf16=0, sigma=0.0, x=None, y=None, x_bf16=False, stride=None,
-                 device="cuda:0", stream=None):
+                 device="cuda:0", stream=None, defer_broadcast=False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -163,7 +167,8 @@ class Mavg:
         self.stream = stream
         sptr = stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream
         self.cfg = make_config(P, K, local_lr, mu, block_lr, B, seed, objective, n, dims, gemm_bf16,
-                               sigma, x_ptr, X_BF16 if x_bf16 else X_F32, y_ptr, n_samples, sptr)
+                               sigma, x_ptr, X_BF16 if x_bf16 else X_F32, y_ptr, n_samples, sptr,
+                               defer_broadcast)
         nbytes = C.c_size_t()
         st = self.lib.mavg_workspace_bytes(C.byref(self.cfg), C.byref(nbytes))
         if st != 0:
@@ -185,6 +190,9 @@ class Mavg:
 
     def meta_update(self):
         self._check(self.lib.mavg_meta_update(self.handle))
+
+    def materialize_replicas(self):
+        self._check(self.lib.mavg_materialize_replicas(self.handle))
 
     def round(self, want_loss=False):
         if want_loss:

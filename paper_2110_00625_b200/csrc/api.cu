@@ -30,6 +30,8 @@ mavg_status validate_config(const mavg_config* cfg, std::string* why) {
   if (!std::isfinite(cfg->block_lr)) return fail(why, MAVG_ERR_INVALID_ARG, "block_lr is not finite");
   if (!(cfg->mu >= 0.f && cfg->mu < 1.f)) return fail(why, MAVG_ERR_INVALID_ARG, "mu must be in [0, 1)");
   if (cfg->n < 1) return fail(why, MAVG_ERR_INVALID_ARG, "n must be >= 1");
+  if (cfg->defer_broadcast != 0 && cfg->defer_broadcast != 1)
+    return fail(why, MAVG_ERR_INVALID_ARG, "defer_broadcast must be 0 or 1");
   switch (cfg->objective) {
     case MAVG_OBJ_NONE:
       break;
@@ -131,10 +133,16 @@ mavg_status do_local_steps(mavg_ctx* c) {
     CU(c, mlp_local_steps(c, round), "MLP local steps");
   }
   c->replicas_equal_global = false;
+  c->replicas_materialized = true;
   return MAVG_OK;
 }
 
 mavg_status do_meta_update(mavg_ctx* c) {
+  // a meta-update with no local step since the last one averages P copies of w~ (d = 0); with
+  // deferred copies they have to be written first.  Without a learner level the caller wrote
+  // the replicas.
+  if (c->cfg.objective != MAVG_OBJ_NONE && c->replicas_equal_global && !c->replicas_materialized)
+    CU(c, launch_broadcast(c, false, /*force_copies=*/true), "re-broadcast");
   CU(c, launch_meta_update(c), "meta-update");
   c->round += 1;
   c->replicas_equal_global = true;
@@ -253,6 +261,13 @@ mavg_status mavg_local_steps(mavg_handle h) {
 mavg_status mavg_meta_update(mavg_handle h) {
   CHECK_HANDLE(h);
   return do_meta_update(h);
+}
+
+mavg_status mavg_materialize_replicas(mavg_handle h) {
+  CHECK_HANDLE(h);
+  if (h->replicas_equal_global && !h->replicas_materialized)
+    CU(h, launch_broadcast(h, false, /*force_copies=*/true), "re-broadcast");
+  return MAVG_OK;
 }
 
 mavg_status mavg_round(mavg_handle h, float* mean_loss) {

@@ -61,7 +61,10 @@ struct mavg_ctx {
   std::string err;
   int sm_count = 148;
   size_t l2_bytes = 0;
-  bool replicas_equal_global = true;  // true between a (re-)broadcast and the next local step
+  bool replicas_equal_global = true;  // every learner's model is w~: true between a (re-)broadcast
+                                      // and the next local step
+  bool replicas_materialized = true;  // the replica array really holds those P copies (false at a
+                                      // round boundary with defer_broadcast)
   mavg::Workspace ws;
   std::vector<mavg::MlpLayer> layers;
   void* mlp = nullptr;        // state of the MLP path (owned by mlp files)
@@ -88,7 +91,8 @@ namespace mavg {
 
 // Every launcher enqueues on ctx->stream, adds to ctx->launches and returns the CUDA status of
 // the launch (cudaGetLastError), nothing else.
-cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v);
+// w^j <- w~ (or, with defer_broadcast, only the book-keeping for it) and optionally v <- 0
+cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v, bool force_copies = false);
 cudaError_t launch_meta_update(mavg_ctx* c);
 cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round);
 

@@ -1,7 +1,7 @@
 // Meta level of Algorithm 1 fused with the next round's "set w^j = w~":
 //   a = (1/P) sum_j w^j;  d = a - w~;  v <- mu v + zeta d;  w~ <- w~ + v;  w^j <- w~  for all j.
 // One pass over HBM: per element 4P + 8 bytes read (4P + 4 when mu = 0: v is not read) and
-// 4P + 8 bytes written.  d is formed as (sum_j (w^j - w~)) / P in ascending j, which is the same
+// 4P + 8 bytes written (8 when the P copies are left to the next round's first local step).  d is formed as (sum_j (w^j - w~)) / P in ascending j, which is the same
 // real number and keeps the fp32 sum small.
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -20,7 +20,7 @@ __device__ __forceinline__ void acc4(float4& a, float4 b) {
 
 __device__ __forceinline__ void meta_scalar(float* rep, int64_t stride, float* w, float* v, int P,
                                             int64_t i, float mu, float zeta, float inv_p,
-                                            bool read_v) {
+                                            bool read_v, bool bcast) {
   float wt = w[i], acc = 0.f;
   for (int j = 0; j < P; ++j) acc += rep[(size_t)j * stride + i] - wt;
   float d = acc * inv_p;
@@ -28,7 +28,8 @@ __device__ __forceinline__ void meta_scalar(float* rep, int64_t stride, float* w
   float wn = wt + vn;
   v[i] = vn;
   w[i] = wn;
-  for (int j = 0; j < P; ++j) rep[(size_t)j * stride + i] = wn;
+  if (bcast)
+    for (int j = 0; j < P; ++j) rep[(size_t)j * stride + i] = wn;
 }
 
 // U replica loads are kept in flight per thread; STREAM_ST selects evict-first stores for the
@@ -37,7 +38,7 @@ template <int U, bool STREAM_ST>
 __global__ void __launch_bounds__(256)
 k_meta_update(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
               float* __restrict__ v, int P, int64_t n, float mu, float zeta, float inv_p,
-              int read_v) {
+              int read_v, int bcast) {
   const int64_t n4 = n >> 2;
   const int64_t stride4 = stride >> 2;
   float4* rep4 = reinterpret_cast<float4*>(rep);
@@ -68,16 +69,19 @@ k_meta_update(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
     if (STREAM_ST) {
       __stcs(v4 + q, vn);
       __stcs(w4 + q, wn);
-      for (int j = 0; j < P; ++j) __stcs(rep4 + (size_t)j * stride4 + q, wn);
+      if (bcast)
+        for (int j = 0; j < P; ++j) __stcs(rep4 + (size_t)j * stride4 + q, wn);
     } else {
       v4[q] = vn;
       w4[q] = wn;
-      for (int j = 0; j < P; ++j) rep4[(size_t)j * stride4 + q] = wn;
+      if (bcast)
+        for (int j = 0; j < P; ++j) rep4[(size_t)j * stride4 + q] = wn;
     }
   }
   // ragged tail (n not a multiple of 4)
   if (blockIdx.x == 0 && threadIdx.x < (n & 3))
-    meta_scalar(rep, stride, w, v, P, (n4 << 2) + threadIdx.x, mu, zeta, inv_p, read_v != 0);
+    meta_scalar(rep, stride, w, v, P, (n4 << 2) + threadIdx.x, mu, zeta, inv_p, read_v != 0,
+                bcast != 0);
 }
 
 // Algorithm 1's "set w^j = w~" on its own (initialisation, resume), optionally with v <- 0.
@@ -136,7 +140,7 @@ template <int T, int G, int STAGES, int THREADS>
 __global__ void __launch_bounds__(THREADS + 32)
 k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
                    float* __restrict__ v, int P, int64_t n_tiles, float mu, float zeta,
-                   float inv_p, int read_v, int* status) {
+                   float inv_p, int read_v, int bcast, int* status) {
   extern __shared__ __align__(128) uint8_t sm[];
   float* st_rep = reinterpret_cast<float*>(sm);            // [STAGES][G][T]
   float* st_wv = st_rep + (size_t)STAGES * G * T;          // [2][2][T]: (w~, v) of two tiles
@@ -242,8 +246,9 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
     if (tid == 0) {
       bulk_store(w + t * T, st_out + (size_t)(b * 2) * T, T * 4);
       bulk_store(v + t * T, st_out + (size_t)(b * 2 + 1) * T, T * 4);
-      for (int j = 0; j < P; ++j)
-        bulk_store(rep + (size_t)j * stride + t * T, st_out + (size_t)(b * 2) * T, T * 4);
+      if (bcast)
+        for (int j = 0; j < P; ++j)
+          bulk_store(rep + (size_t)j * stride + t * T, st_out + (size_t)(b * 2) * T, T * 4);
       bulk_commit();
     }
   }
@@ -252,7 +257,7 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
 
 template <int T, int G, int STAGES, int THREADS>
 cudaError_t launch_bulk(mavg_ctx* c, int64_t n_tiles, float mu, float zeta, float inv_p,
-                        int read_v) {
+                        int read_v, int bcast) {
   const size_t smem = ((size_t)STAGES * G * T + 8 * (size_t)T) * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {
@@ -264,7 +269,7 @@ cudaError_t launch_bulk(mavg_ctx* c, int64_t n_tiles, float mu, float zeta, floa
   const int grid = (int)(n_tiles < c->sm_count ? n_tiles : c->sm_count);
   k_meta_update_bulk<T, G, STAGES, THREADS><<<grid, THREADS + 32, smem, c->stream>>>(
       c->buf.replicas, c->buf.replica_stride, c->buf.global_w, c->buf.momentum, c->cfg.P, n_tiles,
-      mu, zeta, inv_p, read_v, (int*)ws_ptr(c, c->ws.status));
+      mu, zeta, inv_p, read_v, bcast, (int*)ws_ptr(c, c->ws.status));
   return cudaGetLastError();
 }
 
@@ -277,13 +282,16 @@ int grid_for(const mavg_ctx* c, int64_t work_items, int threads, int blocks_per_
 
 }  // namespace
 
-cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v) {
+cudaError_t launch_broadcast(mavg_ctx* c, bool zero_v, bool force_copies) {
   const int64_t n = c->cfg.n;
+  const bool copies = force_copies || !c->cfg.defer_broadcast;
+  c->replicas_materialized = copies;
+  if (!copies && !zero_v) return cudaSuccess;
   int grid = grid_for(c, n >> 2, 256, 8);
   prof_begin(c, MAVG_K_BROADCAST);
   k_broadcast<<<grid, 256, 0, c->stream>>>(c->buf.replicas, c->buf.replica_stride,
-                                           c->buf.global_w, c->buf.momentum, c->cfg.P, n,
-                                           zero_v ? 1 : 0);
+                                           c->buf.global_w, c->buf.momentum, copies ? c->cfg.P : 0,
+                                           n, zero_v ? 1 : 0);
   prof_end(c);
   return cudaGetLastError();
 }
@@ -294,6 +302,8 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
   const float mu = c->cfg.mu, zeta = c->cfg.block_lr;
   const float inv_p = 1.0f / (float)P;
   const int read_v = mu != 0.f ? 1 : 0;
+  const int bcast = c->cfg.defer_broadcast ? 0 : 1;
+  c->replicas_materialized = bcast != 0;
   // A replica set that fits in L2 is about to be re-read by the next round's first local step:
   // it takes the plain-store kernel, which leaves it there.  Larger sets with more than 8
   // replicas go through the bulk-copy kernel tile by tile (measured faster from P = 16 up; with
@@ -306,7 +316,7 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
   cudaError_t e = cudaSuccess;
   if (big && P > 8 && n >= (int64_t)4096 * c->sm_count * 4) {
     done = n / 4096 * 4096;
-    e = launch_bulk<4096, 2, 3, 512>(c, n / 4096, mu, zeta, inv_p, read_v);
+    e = launch_bulk<4096, 2, 3, 512>(c, n / 4096, mu, zeta, inv_p, read_v, bcast);
   }
   if (e == cudaSuccess && done < n) {
     const int64_t rest = n - done;
@@ -316,10 +326,10 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
     float* v = c->buf.momentum + done;
     if (big)
       k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
-                                                          rest, mu, zeta, inv_p, read_v);
+                                                          rest, mu, zeta, inv_p, read_v, bcast);
     else
       k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
-                                                           rest, mu, zeta, inv_p, read_v);
+                                                           rest, mu, zeta, inv_p, read_v, bcast);
     e = cudaGetLastError();
     if (done > 0) c->launches++;
   }

@@ -57,6 +57,11 @@ namespace {
 __global__ void k_set_round(int64_t* dst, int64_t round) { *dst = round; }
 
 cudaError_t run_steps(mavg_ctx* c, int64_t round) {
+  // the CUDA-core path reads every learner's own copy from the first step on
+  if (!use_tensor_cores(&c->cfg) && c->replicas_equal_global && !c->replicas_materialized) {
+    cudaError_t e = launch_broadcast(c, false, /*force_copies=*/true);
+    if (e != cudaSuccess) return e;
+  }
   for (int k = 1; k <= c->cfg.K; ++k) {
     cudaError_t e = use_tensor_cores(&c->cfg) ? tc_step(c, round, k) : simt_step(c, round, k);
     if (e != cudaSuccess) return e;

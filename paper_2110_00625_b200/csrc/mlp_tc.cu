@@ -54,6 +54,8 @@ struct TcArgs {
   int* counters;            // one per (p, m_tile); zero between launches
   float* bias_rep;          // fp32 masters; the bias this kernel reads (forward) or steps (dgrad,
   int64_t bias_off;         // last layer) is at bias_rep[p*rep_stride + bias_off + m]
+  const float* bias_in;     // where the bias is read: bias_in[p*bias_in_stride + bias_off + m], the
+  int64_t bias_in_stride;   // same place, or w~ (stride 0) at the first step of a round
   __nv_bfloat16* out_bm;    // [P, B, M]  relu(z) (forward) or dZ (dgrad)
   __nv_bfloat16* out_mb;    // [P, M, B]  the same, transposed
   const __nv_bfloat16* mask_mb;  // dgrad: forward activation [P, M, B] whose sign gates dZ
@@ -211,8 +213,9 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     // is still running: the bias (read by the forward tails, stepped by the dgrad tail), the
     // first mask chunk (dgrad) and the label of this thread's batch row (last layer).
     float* bias = g.bias_rep + (size_t)p * g.rep_stride + g.bias_off;
+    const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride + g.bias_off;
     const bool m_ok_pre = m0 + row < g.M;
-    const float bias_pre = (m_ok_pre && (EPI != EPI_DGRAD || half == 0)) ? bias[m0 + row] : 0.f;
+    const float bias_pre = (m_ok_pre && (EPI != EPI_DGRAD || half == 0)) ? bias_in[m0 + row] : 0.f;
     uint4 mk[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
                    make_uint4(0, 0, 0, 0)};
     auto load_mask = [&](int c0, uint4 (&dst)[4]) {
@@ -402,7 +405,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               for (int b = lane; b < g.N; b += 32) sb += dzs[b * C + c];
 #pragma unroll
               for (int o = 16; o > 0; o >>= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
-              if (lane == 0) bias[c] = fmaf(-g.gamma, sb, bias[c]);
+              if (lane == 0) bias[c] = fmaf(-g.gamma, sb, bias_in[c]);
             }
           }
           epilogue_barrier();
@@ -556,6 +559,7 @@ struct TcState {
   CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
   CUtensorMap w_mn[MAVG_MAX_LAYERS + 1], wg_mn[MAVG_MAX_LAYERS + 1];  // [out, in] copies, 64 x 64 boxes
   CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
+  CUtensorMap w32g[MAVG_MAX_LAYERS + 1];      // the same view of w~ (one copy): first-step loads
   CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
@@ -700,6 +704,10 @@ mavg_status tc_setup(mavg_ctx* c) {
                           c->buf.replicas + c->layers[l - 1].w_off, in, out, P, in,
                           c->buf.replica_stride, kWgradTileCols, kWgradTileRows,
                           CU_TENSOR_MAP_SWIZZLE_128B, &why);
+    ok = ok && encode_any(st, &st->w32g[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                          c->buf.global_w + c->layers[l - 1].w_off, in, out, 1, in,
+                          c->buf.replica_stride, kWgradTileCols, kWgradTileRows,
+                          CU_TENSOR_MAP_SWIZZLE_128B, &why);
     ok = ok && encode_any(st, &st->w16_st[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w16, in, out, P,
                           in, t.n16, kWgradTileCols, kWgradTileRows, CU_TENSOR_MAP_SWIZZLE_64B,
                           &why);
@@ -816,6 +824,8 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     g.a_batched = shared_w ? 0 : 1; g.b_batched = 1;
     g.part = part; g.counters = counters;
     g.bias_rep = c->buf.replicas; g.bias_off = ly.b_off;
+    g.bias_in = shared_w ? c->buf.global_w : c->buf.replicas;
+    g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
     const CUtensorMap& wm = shared_w ? st->wg[l] : st->w[l];
     const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
     if (l < L) {
@@ -849,6 +859,8 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.a_batched = shared_w ? 0 : 1; g.b_batched = 1;
       g.part = part; g.counters = counters;
       g.bias_rep = c->buf.replicas; g.bias_off = below.b_off;
+      g.bias_in = shared_w ? c->buf.global_w : c->buf.replicas;
+      g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
       g.out_bm = bfp(t.dz[l - 1]); g.out_mb = bfp(t.dz_t[l - 1]);
       g.mask_mb = bfp(t.act_t[l - 1]);
       g.a_mn = 1;
@@ -860,11 +872,13 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
       c->stream = st->s_wgrad;
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l]));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
+                                 shared_w ? &st->w32g[l] : nullptr));
       c->stream = main_s;
       side_used = true;
     } else {
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l]));
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
+                                 shared_w ? &st->w32g[l] : nullptr));
     }
   }
   if (overlap) {

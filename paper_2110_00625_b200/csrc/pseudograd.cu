@@ -3,7 +3,8 @@
 // g an Irwin-Hall(4) variate of standard deviation sigma built from one SplitMix64 stream value
 // (see mavg.h).  The K steps are applied in order to a value held in registers, so one pass over
 // the replicas (8 bytes per element and learner) serves the whole round; the per-step rounding is
-// the same as K separate passes.
+// the same as K separate passes.  The first pass after a (re-)broadcast reads w~ in place of
+// every w^j ("set w^j = w~"), so the P copies need not exist before it.
 #include "common.cuh"
 
 namespace mavg {
@@ -17,8 +18,8 @@ __device__ __forceinline__ float ih4(uint64_t h, float c) {
 
 // grid = (x, P); dynamic shared memory holds the K step keys of learner blockIdx.y.
 __global__ void __launch_bounds__(256)
-k_pseudograd_steps(float* __restrict__ rep, int64_t stride, int64_t n, int K, uint64_t seed,
-                   int64_t round, int k_first, float c, float gamma) {
+k_pseudograd_steps(float* rep, int64_t stride, const float* src, int64_t src_stride, int64_t n,
+                   int K, uint64_t seed, int64_t round, int k_first, float c, float gamma) {
   extern __shared__ uint64_t keys[];
   const int j = blockIdx.y;
   const uint64_t lk = learner_key(seed, kTagPseudoGrad, (uint64_t)round, (uint64_t)j);
@@ -26,11 +27,13 @@ k_pseudograd_steps(float* __restrict__ rep, int64_t stride, int64_t n, int K, ui
   __syncthreads();
   float* row = rep + (size_t)j * stride;
   float4* row4 = reinterpret_cast<float4*>(row);
+  const float* in = src + (size_t)j * src_stride;
+  const float4* in4 = reinterpret_cast<const float4*>(in);
   const int64_t n4 = n >> 2;
   const int64_t step = (int64_t)gridDim.x * blockDim.x;
   const float ng = -gamma;
   for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += step) {
-    float4 w = __ldcs(row4 + q);
+    float4 w = src_stride ? __ldcs(in4 + q) : __ldg(in4 + q);
     const uint64_t c0 = (uint64_t)(4 * q + 1) * kGamma;  // element i uses (i+1) G
     for (int k = 0; k < K; ++k) {
       const uint64_t key = keys[k];
@@ -43,7 +46,7 @@ k_pseudograd_steps(float* __restrict__ rep, int64_t stride, int64_t n, int K, ui
   }
   if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {
     const int64_t i = (n4 << 2) + threadIdx.x;
-    float w = row[i];
+    float w = in[i];
     for (int k = 0; k < K; ++k) w = fmaf(ng, ih4(fold(keys[k], (uint64_t)i), c), w);
     row[i] = w;
   }
@@ -64,11 +67,15 @@ cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round) {
   for (int k0 = 0; k0 < K; k0 += kMaxFused) {
     int kc = K - k0 < kMaxFused ? K - k0 : kMaxFused;
     dim3 grid((unsigned)blocks_x, (unsigned)P);
+    const bool from_global = c->replicas_equal_global;
     prof_begin(c, MAVG_K_PSEUDOGRAD);
     k_pseudograd_steps<<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
-        c->buf.replicas, c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
+        c->buf.replicas, c->buf.replica_stride, from_global ? c->buf.global_w : c->buf.replicas,
+        from_global ? 0 : c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
         c->cfg.local_lr);
     prof_end(c);
+    c->replicas_equal_global = false;
+    c->replicas_materialized = true;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -52,6 +52,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 }
 
 struct WgradArgs {
+  int w32_in_batched;      // 0: every learner loads the one shared master array (w~)
   int nkb;                 // 64-wide slabs of the batch (contraction)
   int m_tiles, n_tiles;    // 128-row tiles of out, 32-column tiles of in
   int chunk;               // column tiles per work item
@@ -66,7 +67,10 @@ struct WgradArgs {
 __global__ void __launch_bounds__(kThreads)
 k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out, B]  load
                    const __grid_constant__ CUtensorMap tm_at,    // bf16 [P, in, B]   load
-                   const __grid_constant__ CUtensorMap tm_w32,   // fp32 [P, out, in] load + store
+                   const __grid_constant__ CUtensorMap tm_w32,   // fp32 [P, out, in] store
+                   const __grid_constant__ CUtensorMap tm_w32_in,  // fp32 masters to load: the same
+                                                                   // array, or w~ [1, out, in] at
+                                                                   // the first step of a round
                    const __grid_constant__ CUtensorMap tm_w16,   // bf16 [P, out, in] store
                    const WgradArgs g) {
   extern __shared__ uint8_t smem_raw[];
@@ -90,6 +94,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     tma_prefetch_desc(&tm_dzt);
     tma_prefetch_desc(&tm_at);
     tma_prefetch_desc(&tm_w32);
+    tma_prefetch_desc(&tm_w32_in);
     tma_prefetch_desc(&tm_w16);
     for (int s = 0; s < g.slots; ++s) {
       mbar_init(&slot_full[s], 1);
@@ -152,7 +157,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
           mbar_arrive_expect_tx(&slot_full[s], (uint32_t)(kW32Bytes + b_bytes));
-          tma_load_3d(sl, &tm_w32, &slot_full[s], i0, m0, p);
+          tma_load_3d(sl, &tm_w32_in, &slot_full[s], i0, m0, g.w32_in_batched ? p : 0);
           for (int kb = 0; kb < g.nkb; ++kb)
             tma_load_3d(sl + kW32Bytes + kW16Bytes + (size_t)kb * (kBN * kBK * 2),
                         &tm_at, &slot_full[s], kb * kBK, i0, p);
@@ -327,8 +332,9 @@ cudaError_t wgrad_stream_prepare() {
 
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16) {
+                                const CUtensorMap& w16, const CUtensorMap* w32_shared) {
   WgradArgs g{};
+  g.w32_in_batched = w32_shared ? 0 : 1;
   g.nkb = w.nkb;
   g.m_tiles = w.m_tiles;
   g.n_tiles = w.n_tiles;
@@ -350,7 +356,8 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   lc.attrs = at_;
   lc.numAttrs = 1;
   prof_begin(c, MAVG_K_WGRAD_SGD);
-  cudaError_t e = cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream, dzt, at, w32, w16, g);
+  cudaError_t e = cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream, dzt, at, w32,
+                                     w32_shared ? *w32_shared : w32, w16, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -18,9 +18,11 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count);
 cudaError_t wgrad_stream_prepare();
 // dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
 // w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128
-// (64B swizzle).
+// (64B swizzle).  w32_shared, if given, is an fp32 [1, out, in] view of w~ with the same box: the
+// masters are then loaded from it for every learner (first step of a round, all w^j = w~) and
+// stored to w32 as always.
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16);
+                                const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr);
 
 }  // namespace mavg

@@ -198,6 +198,17 @@ inline void sgd_step(float* w, const float* g, int64_t n, float gamma) {
   for (int64_t i = 0; i < n; ++i) w[i] = (float)((double)w[i] - (double)gamma * (double)g[i]);
 }
 
+// Learner-level momentum (the variant named after Eq. 2 and in the conclusion: momentum SGD in
+// place of plain SGD inside each learner), written in the form Eq. 2 uses at the meta level:
+//   u <- beta u - gamma g;  w <- w + u.
+inline void msgd_step(float* w, float* u, const float* g, int64_t n, float gamma, float beta) {
+  for (int64_t i = 0; i < n; ++i) {
+    const float un = (float)((double)beta * (double)u[i] - (double)gamma * (double)g[i]);
+    u[i] = un;
+    w[i] = (float)((double)w[i] + (double)un);
+  }
+}
+
 }  // namespace
 
 extern "C" {
@@ -224,6 +235,10 @@ struct orc_problem {
   // quadratic F(w) = 1/2 sum_i a_i w_i^2, exact gradient (used only to pin the round loop)
   const float* quad_a;
   int32_t threads;  // OpenMP threads over the independent learners (<= 0: library default)
+  // learner-level momentum (0 = plain SGD, Algorithm 1 as printed)
+  float beta;
+  int32_t reset_u;  // 1: u^j <- 0 at the start of every round; 0: u^j carried over the rounds
+  float* u;         // [P, stride] learner momentum buffers; required when beta != 0
 };
 
 uint64_t orc_mix64(uint64_t z) { return mix64(z); }
@@ -277,6 +292,9 @@ void orc_local_steps(const orc_problem* pb, int64_t round, float* replicas, doub
 #endif
   for (int j = 0; j < P; ++j) {
     float* w = replicas + (size_t)j * pb->stride;
+    float* u = pb->beta != 0.f ? pb->u + (size_t)j * pb->stride : nullptr;
+    if (u && pb->reset_u)
+      for (int64_t i = 0; i < n; ++i) u[i] = 0.f;
     std::vector<float> g((size_t)n);
     std::vector<float> X;
     std::vector<int32_t> idx, yb;
@@ -301,7 +319,10 @@ void orc_local_steps(const orc_problem* pb, int64_t round, float* replicas, doub
       }
       if (G)
         for (int64_t i = 0; i < n; ++i) Gj[j][i] += (double)g[i];
-      sgd_step(w, g.data(), n, pb->gamma);
+      if (u)
+        msgd_step(w, u, g.data(), n, pb->gamma, pb->beta);
+      else
+        sgd_step(w, g.data(), n, pb->gamma);
       if (losses) losses[(size_t)j * K + (k - 1)] = loss;
     }
   }

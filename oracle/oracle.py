@@ -42,6 +42,7 @@ class _Problem(C.Structure):
         ("sigma", C.c_float),
         ("quad_a", C.c_void_p),
         ("threads", C.c_int32),
+        ("beta", C.c_float), ("reset_u", C.c_int32), ("u", C.c_void_p),
     ]
 
 
@@ -155,7 +156,7 @@ class Mavg:
 
     def __init__(self, w1, P, K, gamma, mu, zeta=1.0, B=1, seed=0, objective=OBJ_PSEUDOGRAD,
                  dims=None, bf16=False, x=None, y=None, sigma=0.0, quad_a=None, stride=None,
-                 threads=0):
+                 threads=0, beta=0.0, reset_u=False):
         self.w = _f32(w1).copy()
         n = self.w.size
         self.stride = int(stride) if stride else n
@@ -186,6 +187,9 @@ class Mavg:
             pb.quad_a = a.ctypes.data
         pb.sigma = sigma
         pb.threads = threads
+        # learner-level momentum buffers u^j (all zero at the start, like v)
+        self.u = np.zeros((P, self.stride), dtype=np.float32)
+        pb.beta, pb.reset_u, pb.u = beta, int(bool(reset_u)), self.u.ctypes.data
         self.pb = pb
         self.round = 0
         lib().orc_init(P, n, self.stride, _ptr(self.replicas), _ptr(self.w), _ptr(self.v))

@@ -403,3 +403,83 @@ def test_learner_order_does_not_matter(oracle):
         m.meta_update()
         outs.append(m.w.copy())
     assert np.abs(outs[0] - outs[1]).max() < 1e-6
+
+
+# -------------------------------------------------------------------- learner-level momentum
+def test_beta_zero_is_algorithm_1_as_printed(oracle):
+    n, P, K = 500, 3, 4
+    w1 = np.random.default_rng(12).standard_normal(n).astype(np.float32)
+    kw = dict(P=P, K=K, gamma=0.05, mu=0.7, seed=5, objective=oracle.OBJ_PSEUDOGRAD, sigma=0.2)
+    a = oracle.Mavg(w1, **kw)
+    b = oracle.Mavg(w1, beta=0.0, reset_u=True, **kw)
+    for _ in range(3):
+        a.run_round(); b.run_round()
+    assert np.array_equal(a.w, b.w) and np.array_equal(a.v, b.v)
+    assert not b.u.any()
+
+
+@pytest.mark.parametrize("beta", [0.5, 0.9])
+def test_learner_momentum_unrolled_sum(oracle, beta):
+    # u_k = -gamma sum_{i<k} beta^i g_{k-i}  and  w_K = w_0 + sum_k u_k, by brute force in fp64
+    n, K, gamma, sigma = 300, 6, 0.05, 0.3
+    w1 = np.random.default_rng(13).standard_normal(n).astype(np.float32)
+    m = oracle.Mavg(w1, P=2, K=K, gamma=gamma, mu=0.0, seed=17, objective=oracle.OBJ_PSEUDOGRAD,
+                    sigma=sigma, beta=beta)
+    m.local_steps()
+    g32, b32 = np.float64(np.float32(gamma)), np.float64(np.float32(beta))
+    for j in range(2):
+        g = [oracle.pseudograd(17, 1, j, k, 0, n, sigma).astype(np.float64) for k in range(1, K + 1)]
+        us = [-g32 * sum(b32 ** i * g[k - 1 - i] for i in range(k)) for k in range(1, K + 1)]
+        assert np.abs(m.u[j, :n] - us[-1]).max() < 1e-6
+        assert np.abs(m.replicas[j, :n] - (w1.astype(np.float64) + sum(us))).max() < 2e-6
+
+
+@pytest.mark.parametrize("beta,gamma", [(0.5, 0.1), (0.9, 0.3)])
+def test_learner_momentum_heavy_ball_closed_form(oracle, beta, gamma):
+    # on F = 1/2 a w^2 the steps are the two-term recurrence w_{k+1} = (1 + beta - gamma a) w_k
+    # - beta w_{k-1}, w_1 = (1 - gamma a) w_0, whose solution is c1 r1^k + c2 r2^k with r1, r2 the
+    # (possibly complex) roots of r^2 - (1 + beta - gamma a) r + beta = 0
+    n, K = 7, 9
+    r = np.random.default_rng(14)
+    a = r.uniform(0.3, 2.5, n).astype(np.float32)
+    w0 = r.standard_normal(n).astype(np.float32)
+    m = oracle.Mavg(w0, P=1, K=K, gamma=gamma, mu=0.0, objective=oracle.OBJ_QUADRATIC, quad_a=a,
+                    beta=beta)
+    m.local_steps()
+    g32, b32 = np.float64(np.float32(gamma)), np.float64(np.float32(beta))
+    t = (1 + b32 - g32 * a.astype(np.float64)).astype(np.complex128)
+    disc = np.sqrt(t * t - 4 * b32)
+    r1, r2 = (t + disc) / 2, (t - disc) / 2
+    w_0 = w0.astype(np.complex128)
+    w_1 = (1 - g32 * a.astype(np.float64)) * w_0
+    c1 = (w_1 - r2 * w_0) / (r1 - r2)
+    c2 = w_0 - c1
+    want = (c1 * r1 ** K + c2 * r2 ** K).real
+    assert np.abs(m.replicas[0, :n] - want).max() < 5e-6 * max(1.0, np.abs(want).max())
+
+
+@pytest.mark.parametrize("reset", [False, True])
+def test_learner_momentum_against_torch_sgd(oracle, reset):
+    # P = 1, mu = 0, zeta = 1: the global model follows the single learner, so the rounds are one
+    # run of momentum SGD -- torch's optimizer (buf <- beta buf + g, p <- p - lr buf, the same
+    # sequence as u = -lr buf) with its buffer kept over the rounds, or re-made every round
+    dims, B, S, K, beta, lr = [8, 6, 3], 4, 40, 3, 0.8, 0.1
+    r = np.random.default_rng(15)
+    x = r.standard_normal((S, dims[0])).astype(np.float32)
+    y = r.integers(0, 3, S).astype(np.int32)
+    w1 = (0.4 * r.standard_normal(oracle.mlp_param_count(dims))).astype(np.float32)
+    m = oracle.Mavg(w1, P=1, K=K, gamma=lr, mu=0.0, B=B, seed=23, objective=oracle.OBJ_MLP,
+                    dims=dims, x=x, y=y, beta=beta, reset_u=reset)
+    w = torch.tensor(w1, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([w], lr=float(np.float32(lr)), momentum=float(np.float32(beta)))
+    for n in range(1, 4):
+        if reset:
+            opt = torch.optim.SGD([w], lr=float(np.float32(lr)), momentum=float(np.float32(beta)))
+        for k in range(1, K + 1):
+            idx = oracle.batch_indices(23, n, 1, 0, k, S, B)
+            opt.zero_grad()
+            _torch_mlp_loss(dims, w, torch.tensor(x[idx], dtype=torch.float64),
+                            torch.tensor(y[idx], dtype=torch.long)).backward()
+            opt.step()
+        m.run_round()
+        assert np.abs(m.w - w.detach().numpy()).max() < 2e-5

@@ -102,6 +102,16 @@ typedef struct {
                         assignment with 4P bytes per element less traffic.  Between a meta-update
                         and the next local step the replica array then holds the previous round's
                         learner models; mavg_materialize_replicas writes the copies on request. */
+  /* Learner-level momentum (the variant the paper names after Eq. 2 and in its conclusion:
+   * momentum SGD inside each learner, under the block momentum of the meta level).  With
+   * beta = learner_momentum != 0 the local step of Algorithm 1 becomes, in the form Eq. 2 uses,
+   *     u^j <- beta u^j - gamma g;   w^j <- w^j + u^j
+   * with one buffer u^j per learner (mavg_buffers.learner_u).  beta = 0 is Algorithm 1 as printed.
+   * The paper does not say what happens to u^j when a round ends; learner_momentum_reset picks:
+   * 0: u^j is kept over the rounds (zero only before the first round); 1: u^j <- 0 whenever the
+   * learners restart from w~ (the first local step after a (re-)broadcast). */
+  float learner_momentum;         /* beta, 0 <= beta < 1 */
+  int32_t learner_momentum_reset; /* 0 or 1 */
 } mavg_config;
 
 /* Caller-owned DEVICE buffers.  Every base pointer must be 16-byte aligned. */
@@ -112,6 +122,9 @@ typedef struct {
   float *momentum;        /* [n] v */
   void *workspace;        /* scratch, at least mavg_workspace_bytes() bytes */
   size_t workspace_bytes;
+  float *learner_u;       /* [P, replica_stride] fp32 learner momentum buffers u^j, same layout as
+                             replicas; required iff learner_momentum != 0 (else ignored, may be
+                             NULL).  mavg_create zeroes it. */
 } mavg_buffers;
 
 /* Bytes of scratch the configuration needs (activations, bf16 operand copies, batch indices,
@@ -149,6 +162,10 @@ mavg_status mavg_round_host(mavg_handle h, float *w_host, float *v_host, float *
 
 /* Per-round schedules (Algorithm 1 lets gamma_n and B_n vary with n; B stays fixed here). */
 mavg_status mavg_set_hparams(mavg_handle h, int32_t K, float local_lr, float block_lr, float mu);
+
+/* Changes the learner-level momentum between rounds (see mavg_config).  beta != 0 needs the
+ * learner_u buffer given at mavg_create; the buffer's contents are left as they are. */
+mavg_status mavg_set_learner_momentum(mavg_handle h, float beta, int32_t reset);
 
 /* Runs the device index generator for (round, learner, step) and copies the B indices to
  * out (HOST, B int32); waits for the stream.  MLP objective only. */

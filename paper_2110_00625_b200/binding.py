@@ -17,7 +17,8 @@ STATUS = {0: "MAVG_OK", 1: "MAVG_ERR_INVALID_ARG", 2: "MAVG_ERR_BAD_BUFFER", 3: 
           4: "MAVG_ERR_UNSUPPORTED", 5: "MAVG_ERR_CUDA", 6: "MAVG_ERR_TIMEOUT"}
 
 EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta_update",
-           "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams", "mavg_get_batch_indices",
+           "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams",
+           "mavg_set_learner_momentum", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
            "mavg_set_profiling", "mavg_get_profile", "mavg_sync", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
@@ -37,6 +38,7 @@ class Config(C.Structure):
         ("x", C.c_void_p), ("x_dtype", C.c_int32), ("y", C.c_void_p), ("n_samples", C.c_int64),
         ("stream", C.c_void_p),
         ("defer_broadcast", C.c_int32),
+        ("learner_momentum", C.c_float), ("learner_momentum_reset", C.c_int32),
     ]
 
 
@@ -45,6 +47,7 @@ class Buffers(C.Structure):
         ("replicas", C.c_void_p), ("replica_stride", C.c_int64),
         ("global_w", C.c_void_p), ("momentum", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("learner_u", C.c_void_p),
     ]
 
 
@@ -79,6 +82,7 @@ def load_library():
     L.mavg_round.argtypes = [H, C.POINTER(C.c_float)]
     L.mavg_round_host.argtypes = [H, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
     L.mavg_set_hparams.argtypes = [H, C.c_int32, C.c_float, C.c_float, C.c_float]
+    L.mavg_set_learner_momentum.argtypes = [H, C.c_float, C.c_int32]
     L.mavg_get_batch_indices.argtypes = [H, C.c_int64, C.c_int32, C.c_int32, C.c_void_p]
     L.mavg_get_losses.argtypes = [H, C.c_void_p]
     L.mavg_get_round.argtypes = [H, C.POINTER(C.c_int64)]
@@ -103,7 +107,7 @@ def load_library():
 
 def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE, n=0, dims=None,
                 gemm_bf16=0, sigma=0.0, x_ptr=0, x_dtype=X_F32, y_ptr=0, n_samples=0, stream=0,
-                defer_broadcast=False):
+                defer_broadcast=False, learner_momentum=0.0, learner_momentum_reset=False):
     cfg = Config()
     cfg.P, cfg.K, cfg.B = P, K, B
     cfg.local_lr, cfg.block_lr, cfg.mu = local_lr, block_lr, mu
@@ -119,6 +123,8 @@ def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NON
     cfg.x, cfg.x_dtype, cfg.y, cfg.n_samples = x_ptr, x_dtype, y_ptr, n_samples
     cfg.stream = stream
     cfg.defer_broadcast = 1 if defer_broadcast else 0
+    cfg.learner_momentum = learner_momentum
+    cfg.learner_momentum_reset = 1 if learner_momentum_reset else 0
     return cfg
 
 
@@ -144,7 +150,8 @@ class Mavg:
 
     def __init__(self, w1, P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE,
                  dims=None, gemm_bf16=0, sigma=0.0, x=None, y=None, x_bf16=False, stride=None,
-                 device="cuda:0", stream=None, defer_broadcast=False):
+                 device="cuda:0", stream=None, defer_broadcast=False, learner_momentum=0.0,
+                 learner_momentum_reset=False, with_learner_u=None):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -168,14 +175,21 @@ class Mavg:
         sptr = stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream
         self.cfg = make_config(P, K, local_lr, mu, block_lr, B, seed, objective, n, dims, gemm_bf16,
                                sigma, x_ptr, X_BF16 if x_bf16 else X_F32, y_ptr, n_samples, sptr,
-                               defer_broadcast)
+                               defer_broadcast, learner_momentum, learner_momentum_reset)
+        # learner momentum buffers u^j [P, stride]: allocated when beta != 0 or on request (a
+        # handle that switches the momentum on later with set_learner_momentum)
+        if with_learner_u is None:
+            with_learner_u = learner_momentum != 0.0
+        self.u = (torch.empty((P, self.stride), dtype=torch.float32, device=self.device)
+                  if with_learner_u else None)
         nbytes = C.c_size_t()
         st = self.lib.mavg_workspace_bytes(C.byref(self.cfg), C.byref(nbytes))
         if st != 0:
             raise MavgError(st, self.lib.mavg_last_error(None).decode())
         self.workspace = torch.empty(max(nbytes.value, 256), dtype=torch.uint8, device=self.device)
         self.buf = Buffers(self.replicas.data_ptr(), self.stride, self.w.data_ptr(),
-                           self.v.data_ptr(), self.workspace.data_ptr(), self.workspace.numel())
+                           self.v.data_ptr(), self.workspace.data_ptr(), self.workspace.numel(),
+                           self.u.data_ptr() if self.u is not None else None)
         self.handle = C.c_void_p()
         st = self.lib.mavg_create(C.byref(self.cfg), C.byref(self.buf), C.byref(self.handle))
         if st != 0:
@@ -212,6 +226,9 @@ class Mavg:
     def set_hparams(self, K, local_lr, block_lr, mu):
         self._check(self.lib.mavg_set_hparams(self.handle, K, local_lr, block_lr, mu))
         self.K = K
+
+    def set_learner_momentum(self, beta, reset=False):
+        self._check(self.lib.mavg_set_learner_momentum(self.handle, beta, int(bool(reset))))
 
     def get_batch_indices(self, round_, learner, step):
         import numpy as np

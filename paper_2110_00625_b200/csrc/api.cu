@@ -32,6 +32,12 @@ mavg_status validate_config(const mavg_config* cfg, std::string* why) {
   if (cfg->n < 1) return fail(why, MAVG_ERR_INVALID_ARG, "n must be >= 1");
   if (cfg->defer_broadcast != 0 && cfg->defer_broadcast != 1)
     return fail(why, MAVG_ERR_INVALID_ARG, "defer_broadcast must be 0 or 1");
+  if (!(cfg->learner_momentum >= 0.f && cfg->learner_momentum < 1.f))
+    return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum must be in [0, 1)");
+  if (cfg->learner_momentum_reset != 0 && cfg->learner_momentum_reset != 1)
+    return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum_reset must be 0 or 1");
+  if (cfg->learner_momentum != 0.f && cfg->objective == MAVG_OBJ_NONE)
+    return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum needs a learner level (objective)");
   switch (cfg->objective) {
     case MAVG_OBJ_NONE:
       break;
@@ -203,6 +209,10 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
   if (buf->replica_stride < cfg->n || buf->replica_stride % 4)
     return fail(&g_create_error, MAVG_ERR_BAD_BUFFER,
                 "replica_stride must be >= n and a multiple of 4");
+  if (cfg->learner_momentum != 0.f && !buf->learner_u)
+    return fail(&g_create_error, MAVG_ERR_BAD_BUFFER, "learner_momentum != 0 needs the learner_u buffer");
+  if ((uintptr_t)buf->learner_u % 16)
+    return fail(&g_create_error, MAVG_ERR_BAD_BUFFER, "learner_u must be 16-byte aligned");
   Workspace ws;
   carve_workspace(cfg, &ws);
   if (buf->workspace_bytes < ws.total)
@@ -230,6 +240,9 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
   e = cudaMemsetAsync(ws_ptr(c, c->ws.status), 0, 256, c->stream);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ws_ptr(c, c->ws.losses), 0, (size_t)cfg->P * cfg->K * sizeof(float), c->stream);
+  if (e == cudaSuccess && buf->learner_u && cfg->objective != MAVG_OBJ_NONE)
+    e = cudaMemsetAsync(buf->learner_u, 0,
+                        ((size_t)(cfg->P - 1) * buf->replica_stride + cfg->n) * sizeof(float), c->stream);
   if (e == cudaSuccess) e = launch_broadcast(c, /*zero_v=*/true);
   if (e != cudaSuccess) {
     g_create_error = std::string("initialisation: ") + cudaGetErrorString(e);
@@ -319,6 +332,18 @@ mavg_status mavg_set_hparams(mavg_handle h, int32_t K, float local_lr, float blo
   h->cfg.local_lr = local_lr;
   h->cfg.block_lr = block_lr;
   h->cfg.mu = mu;
+  return MAVG_OK;
+}
+
+mavg_status mavg_set_learner_momentum(mavg_handle h, float beta, int32_t reset) {
+  CHECK_HANDLE(h);
+  if (!(beta >= 0.f && beta < 1.f))
+    return set_err(h, MAVG_ERR_INVALID_ARG, "learner momentum must be in [0, 1)");
+  if (reset != 0 && reset != 1) return set_err(h, MAVG_ERR_INVALID_ARG, "reset must be 0 or 1");
+  if (beta != 0.f && (!h->buf.learner_u || h->cfg.objective == MAVG_OBJ_NONE))
+    return set_err(h, MAVG_ERR_STATE, "this handle was created without the learner_u buffer");
+  h->cfg.learner_momentum = beta;
+  h->cfg.learner_momentum_reset = reset;
   return MAVG_OK;
 }
 

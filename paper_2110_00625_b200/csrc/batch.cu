@@ -123,7 +123,7 @@ k_softmax_ce(const float* __restrict__ logits, int ldz, const int32_t* __restric
              int C, float* __restrict__ loss_out, int loss_stride, float* __restrict__ dz_f32,
              int ld32, __nv_bfloat16* __restrict__ dz_bf, int ldbf,
              __nv_bfloat16* __restrict__ dz_bft, int ldbft, float* __restrict__ rep,
-             int64_t rep_stride, int64_t bias_off, float gamma) {
+             int64_t rep_stride, int64_t bias_off, float gamma, const MomArgs mom) {
   extern __shared__ float part[];     // [blockDim.x] loss partials
   const int p = blockIdx.x;
   const float inv_b = 1.0f / (float)B;
@@ -156,10 +156,11 @@ k_softmax_ce(const float* __restrict__ logits, int ldz, const int32_t* __restric
   }
   if (rep) {
     float* bias = rep + (size_t)p * rep_stride + bias_off;
+    float* ub = mom.u ? mom.u + (size_t)p * mom.u_stride + bias_off : nullptr;
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
       float s = 0.f;
       for (int b = 0; b < B; ++b) s += dz_f32[((size_t)p * B + b) * ld32 + c];
-      bias[c] = fmaf(-gamma, s, bias[c]);
+      local_update(bias + c, bias[c], ub ? ub + c : nullptr, mom.read_u, s, gamma, mom.beta);
     }
   }
 }
@@ -213,7 +214,7 @@ cudaError_t launch_gather(mavg_ctx* c, const int32_t* idx, int quant, float* out
 cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const int32_t* labels,
                               float* loss_out, int loss_stride, float* dz_f32, int ld32,
                               __nv_bfloat16* dz_bf, int ldbf, __nv_bfloat16* dz_bft, int ldbft,
-                              bool update_bias) {
+                              bool update_bias, const MomArgs& mom) {
   const int P = c->cfg.P, B = c->cfg.B, C = c->cfg.dims[c->cfg.n_layers];
   int threads = 32;
   while (threads < B && threads < 256) threads <<= 1;
@@ -223,7 +224,7 @@ cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const i
   k_softmax_ce<<<P, threads, smem, c->stream>>>(
       logits, ldz, labels, B, C, loss_out, loss_stride, dz_f32, ld32, dz_bf, ldbf, dz_bft, ldbft,
       update_bias ? c->buf.replicas : nullptr, c->buf.replica_stride, last.b_off,
-      c->cfg.local_lr);
+      c->cfg.local_lr, mom);
   prof_end(c);
   return cudaGetLastError();
 }

@@ -33,6 +33,34 @@ __host__ __device__ __forceinline__ uint64_t learner_key(uint64_t seed, uint64_t
   return fold(fold(fold(seed, tag), n), j);
 }
 
+// --------------------------------------------------------------------- learner-level update
+// Algorithm 1's local step  w <- w - gamma g,  or with learner-level momentum (u != nullptr)
+//   u <- beta u - gamma g;  w <- w + u
+// on the buffers u^j, laid out like the replicas.  read_u == 0: the stored u counts as zero (the
+// learners restart from w~ and the momentum is reset there), so it is written but not read.
+struct MomArgs {
+  float beta = 0.f;
+  float* u = nullptr;
+  int64_t u_stride = 0;
+  int read_u = 0;
+};
+__device__ __forceinline__ void msgd(float& w, float& u, float grad, float gamma, float beta) {
+  u = fmaf(-gamma, grad, beta * u);
+  w += u;
+}
+// One scalar parameter at *wp (read from w_in), its momentum slot at *up (may be null).
+__device__ __forceinline__ void local_update(float* wp, float w_in, float* up, int read_u,
+                                             float grad, float gamma, float beta) {
+  if (up) {
+    float u = read_u ? *up : 0.f;
+    msgd(w_in, u, grad, gamma, beta);
+    *up = u;
+    *wp = w_in;
+  } else {
+    *wp = fmaf(-gamma, grad, w_in);
+  }
+}
+
 // ------------------------------------------------------------------------------------- context
 struct MlpLayer {
   int in, out;
@@ -84,10 +112,24 @@ struct mavg_ctx {
   cudaStream_t cap_stream = nullptr;
   int graph_K = 0;
   float graph_lr = 0.f;
+  float graph_beta = 0.f;
+  int graph_reset = 0;
   int64_t graph_nodes = 0;
 };
 
 namespace mavg {
+
+// Momentum arguments of a local step; from_broadcast: the step starts from w^j = w~.
+inline MomArgs mom_args(const mavg_ctx* c, bool from_broadcast) {
+  MomArgs m;
+  if (c->cfg.learner_momentum != 0.f) {
+    m.beta = c->cfg.learner_momentum;
+    m.u = c->buf.learner_u;
+    m.u_stride = c->buf.replica_stride;
+    m.read_u = (from_broadcast && c->cfg.learner_momentum_reset) ? 0 : 1;
+  }
+  return m;
+}
 
 // Every launcher enqueues on ctx->stream, adds to ctx->launches and returns the CUDA status of
 // the launch (cudaGetLastError), nothing else.

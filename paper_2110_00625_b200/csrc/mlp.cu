@@ -110,6 +110,8 @@ cudaError_t build_graph(mavg_ctx* c, int64_t round) {
   }
   c->graph_K = c->cfg.K;
   c->graph_lr = c->cfg.local_lr;
+  c->graph_beta = c->cfg.learner_momentum;
+  c->graph_reset = c->cfg.learner_momentum_reset;
   return cudaSuccess;
 }
 
@@ -127,7 +129,8 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
   // capture failed once take the launch-by-launch path.
   const bool want_graph = !c->profiling && !c->graph_disabled && c->replicas_equal_global;
   if (!want_graph) return run_steps(c, round);
-  if (!c->graph_exec || c->graph_K != c->cfg.K || c->graph_lr != c->cfg.local_lr) {
+  if (!c->graph_exec || c->graph_K != c->cfg.K || c->graph_lr != c->cfg.local_lr ||
+      c->graph_beta != c->cfg.learner_momentum || c->graph_reset != c->cfg.learner_momentum_reset) {
     cudaError_t e = build_graph(c, round);
     if (e != cudaSuccess) {
       cudaGetLastError();

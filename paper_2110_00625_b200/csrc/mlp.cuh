@@ -15,7 +15,7 @@ cudaError_t launch_sample_gather(mavg_ctx* c, int64_t round, int step, int32_t* 
 cudaError_t launch_softmax_ce(mavg_ctx* c, const float* logits, int ldz, const int32_t* labels,
                               float* loss_out, int loss_stride, float* dz_f32, int ld32,
                               __nv_bfloat16* dz_bf, int ldbf, __nv_bfloat16* dz_bft, int ldbft,
-                              bool update_bias);
+                              bool update_bias, const MomArgs& mom = MomArgs());
 
 // CUDA-core path (mlp_simt.cu): fp32 arithmetic, or bf16-rounded operands with fp32 FMAs.
 size_t simt_workspace_bytes(const mavg_config* cfg, size_t base, size_t* act_off);

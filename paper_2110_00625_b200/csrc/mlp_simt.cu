@@ -31,6 +31,8 @@ struct GemmArgs {
   float* C; int64_t c_batch; int64_t c_m;               // C(m,n) = C[p*c_batch + m*c_m + n]
   const float* aux; int64_t aux_batch; int64_t aux_m;   // bias [n] (fwd) or mask source Z (dgrad)
   float gamma;
+  MomArgs mom;          // EPI_WGRAD_SGD: learner momentum slots at mom.u[p*u_stride + (C's offset)]
+  int64_t u_off;        // offset of C inside a replica (the same inside u^j)
 };
 
 enum Epi { EPI_FWD = 0, EPI_DGRAD = 1, EPI_WGRAD_SGD = 2 };
@@ -88,6 +90,8 @@ __global__ void __launch_bounds__(256) k_simt_gemm(GemmArgs g) {
   }
 
   float* C = g.C + (size_t)p * g.c_batch;
+  float* U = (EPI == EPI_WGRAD_SGD && g.mom.u) ? g.mom.u + (size_t)p * g.mom.u_stride + g.u_off
+                                               : nullptr;
   const float* aux = g.aux ? g.aux + (size_t)p * g.aux_batch : nullptr;
 #pragma unroll
   for (int i = 0; i < TM; ++i) {
@@ -104,7 +108,7 @@ __global__ void __launch_bounds__(256) k_simt_gemm(GemmArgs g) {
       } else if (EPI == EPI_DGRAD) {
         C[ci] = aux[(size_t)gm * g.aux_m + gn] > 0.f ? v : 0.f;   // ReLU'(0) = 0
       } else {
-        C[ci] = fmaf(-g.gamma, v, C[ci]);
+        local_update(C + ci, C[ci], U ? U + ci : nullptr, g.mom.read_u, v, g.gamma, g.mom.beta);
       }
     }
   }
@@ -113,7 +117,8 @@ __global__ void __launch_bounds__(256) k_simt_gemm(GemmArgs g) {
 // b[o] -= gamma * sum_b dZ[b, o], ascending b.  grid (ceil(out/256), P)
 __global__ void __launch_bounds__(256)
 k_simt_bias_sgd(const float* __restrict__ dz, int64_t dz_batch, int B, int out,
-                float* __restrict__ rep, int64_t rep_stride, int64_t b_off, float gamma) {
+                float* __restrict__ rep, int64_t rep_stride, int64_t b_off, float gamma,
+                const MomArgs mom) {
   int o = blockIdx.x * blockDim.x + threadIdx.x;
   if (o >= out) return;
   const int p = blockIdx.y;
@@ -121,7 +126,8 @@ k_simt_bias_sgd(const float* __restrict__ dz, int64_t dz_batch, int B, int out,
   float s = 0.f;
   for (int b = 0; b < B; ++b) s += d[(size_t)b * out + o];
   float* bias = rep + (size_t)p * rep_stride + b_off;
-  bias[o] = fmaf(-gamma, s, bias[o]);
+  float* ub = mom.u ? mom.u + (size_t)p * mom.u_stride + b_off : nullptr;
+  local_update(bias + o, bias[o], ub ? ub + o : nullptr, mom.read_u, s, gamma, mom.beta);
 }
 
 struct SimtBuffers {
@@ -160,6 +166,7 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
   if ((e = launch_gather(c, idx, QUANT ? 1 : 0, sb.xg, nullptr, nullptr)) != cudaSuccess) return e;
   float* rep = c->buf.replicas;
   const int64_t rs = c->buf.replica_stride;
+  const MomArgs mom = mom_args(c, c->replicas_equal_global);
   // forward
   for (int l = 1; l <= L; ++l) {
     const MlpLayer& ly = c->layers[l - 1];
@@ -181,7 +188,7 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
   // loss, dZ_L and the last bias
   const int C = cfg.dims[L];
   if ((e = launch_softmax_ce(c, sb.z[L], C, labels, losses + (step - 1), cfg.K, sb.dz[L], C,
-                             nullptr, 0, nullptr, 0, true)) != cudaSuccess)
+                             nullptr, 0, nullptr, 0, true, mom)) != cudaSuccess)
     return e;
   // backward + SGD, layer L down to 1; dgrad reads W_l before wgrad overwrites it
   for (int l = L; l >= 1; --l) {
@@ -206,6 +213,7 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
       g.M = ly.out; g.N = ly.in; g.K = B;
       g.C = rep + ly.w_off; g.c_batch = rs; g.c_m = ly.in;
       g.gamma = cfg.local_lr;
+      g.mom = mom; g.u_off = ly.w_off;
       dim3 grid((ly.in + BN - 1) / BN, (ly.out + BM - 1) / BM, P);
       prof_begin(c, MAVG_K_WGRAD_SGD);
       if (l == 1)
@@ -219,7 +227,7 @@ cudaError_t step_impl(mavg_ctx* c, int64_t round, int step) {
       dim3 grid((ly.out + 255) / 256, P);
       prof_begin(c, MAVG_K_WGRAD_SGD);
       k_simt_bias_sgd<<<grid, 256, 0, c->stream>>>(sb.dz[l], (int64_t)B * ly.out, B, ly.out, rep,
-                                                   rs, ly.b_off, cfg.local_lr);
+                                                   rs, ly.b_off, cfg.local_lr, mom);
       prof_end(c);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }

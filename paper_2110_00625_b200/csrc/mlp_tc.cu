@@ -68,6 +68,7 @@ struct TcArgs {
   __nv_bfloat16* dz_mb;     // [P, M, B]
   int64_t rep_stride;
   float gamma;
+  MomArgs mom;              // learner momentum of the bias this kernel steps (slots laid out like bias_rep)
   int* status;
 };
 
@@ -364,8 +365,11 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           // share a row add their column sums in a fixed order
           colsum[half][row] = dsum;
           epilogue_barrier();
-          if (half == 0 && m_ok)
-            bias[m] = fmaf(-g.gamma, colsum[0][row] + colsum[1][row], bias_pre);
+          if (half == 0 && m_ok) {
+            float* ub = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride + g.bias_off + m : nullptr;
+            local_update(bias + m, bias_pre, ub, g.mom.read_u, colsum[0][row] + colsum[1][row],
+                         g.gamma, g.mom.beta);
+          }
         }
         if (EPI == EPI_FWD_LAST) {
           // softmax cross-entropy on the block's [N, M] logits: thread t takes batch row t
@@ -405,7 +409,10 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               for (int b = lane; b < g.N; b += 32) sb += dzs[b * C + c];
 #pragma unroll
               for (int o = 16; o > 0; o >>= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
-              if (lane == 0) bias[c] = fmaf(-g.gamma, sb, bias_in[c]);
+              if (lane == 0) {
+                float* ub = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride + g.bias_off + c : nullptr;
+                local_update(bias + c, bias_in[c], ub, g.mom.read_u, sb, g.gamma, g.mom.beta);
+              }
             }
           }
           epilogue_barrier();
@@ -561,6 +568,8 @@ struct TcState {
   CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
   CUtensorMap w32g[MAVG_MAX_LAYERS + 1];      // the same view of w~ (one copy): first-step loads
   CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
+  CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
+  bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap
@@ -678,7 +687,13 @@ mavg_status tc_setup(mavg_ctx* c) {
     const int in = cfg.dims[l - 1], out = cfg.dims[l];
     const int dz_ld = l < L ? out : t.cpad;
     st->fwd[l] = plan_partial(out, B, in, P, kPlanSmCount, l < L);
-    st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count);
+    st->wgrad_mom = c->buf.learner_u != nullptr;
+    st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count, st->wgrad_mom);
+    if (st->wgrad_mom)
+      ok = ok && encode_any(st, &st->u32[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                            c->buf.learner_u + c->layers[l - 1].w_off, in, out, P, in,
+                            c->buf.replica_stride, kWgradTileCols, kWgradTileRows,
+                            CU_TENSOR_MAP_SWIZZLE_128B, &why);
     __nv_bfloat16* w16 = (__nv_bfloat16*)bf(t.w16) + t.sh_off[l - 1];
     __nv_bfloat16* w16g = (__nv_bfloat16*)bf(t.w16g) + t.sh_off[l - 1];
     ok = ok && encode_map(st, &st->w[l], w16, in, out, P, in, t.n16, kBM, &why);
@@ -801,6 +816,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   float* part = (float*)(ws + t.part);
   int* counters = (int*)(ws + t.counters);
   const bool shared_w = c->replicas_equal_global;   // first step after a (re-)broadcast
+  const MomArgs mom = mom_args(c, shared_w);
   const bool overlap = !c->profiling;
   const int xb = step & 1;                          // batch buffer of this step
   cudaStream_t main_s = c->stream;
@@ -834,6 +850,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     } else {
       g.labels = labels_b; g.loss_out = losses + (step - 1); g.loss_stride = K;
       g.dz_bm = bfp(t.dz[L]); g.cpad = t.cpad; g.dz_mb = bfp(t.dz_t[L]);
+      g.mom = mom;
       TC_TRY(launch_gemm<EPI_FWD_LAST>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
     }
   }
@@ -864,6 +881,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.out_bm = bfp(t.dz[l - 1]); g.out_mb = bfp(t.dz_t[l - 1]);
       g.mask_mb = bfp(t.act_t[l - 1]);
       g.a_mn = 1;
+      g.mom = mom;
       TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : st->w_mn[l],
                                     st->dz[l], st->dgrad[l], g));
     }
@@ -873,12 +891,12 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
       c->stream = st->s_wgrad;
       TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
-                                 shared_w ? &st->w32g[l] : nullptr));
+                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
       c->stream = main_s;
       side_used = true;
     } else {
       TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
-                                 shared_w ? &st->w32g[l] : nullptr));
+                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
     }
   }
   if (overlap) {

@@ -17,9 +17,12 @@ __device__ __forceinline__ float ih4(uint64_t h, float c) {
 }
 
 // grid = (x, P); dynamic shared memory holds the K step keys of learner blockIdx.y.
+// MOM: learner-level momentum, u^j read (unless mom.read_u == 0) and written once per pass like w^j.
+template <bool MOM>
 __global__ void __launch_bounds__(256)
 k_pseudograd_steps(float* rep, int64_t stride, const float* src, int64_t src_stride, int64_t n,
-                   int K, uint64_t seed, int64_t round, int k_first, float c, float gamma) {
+                   int K, uint64_t seed, int64_t round, int k_first, float c, float gamma,
+                   const MomArgs mom) {
   extern __shared__ uint64_t keys[];
   const int j = blockIdx.y;
   const uint64_t lk = learner_key(seed, kTagPseudoGrad, (uint64_t)round, (uint64_t)j);
@@ -32,23 +35,44 @@ k_pseudograd_steps(float* rep, int64_t stride, const float* src, int64_t src_str
   const int64_t n4 = n >> 2;
   const int64_t step = (int64_t)gridDim.x * blockDim.x;
   const float ng = -gamma;
+  float* urow = MOM ? mom.u + (size_t)j * mom.u_stride : nullptr;
+  float4* urow4 = reinterpret_cast<float4*>(urow);
   for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += step) {
     float4 w = src_stride ? __ldcs(in4 + q) : __ldg(in4 + q);
+    float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (MOM && mom.read_u) u = __ldcs(urow4 + q);
     const uint64_t c0 = (uint64_t)(4 * q + 1) * kGamma;  // element i uses (i+1) G
     for (int k = 0; k < K; ++k) {
       const uint64_t key = keys[k];
-      w.x = fmaf(ng, ih4(mix64(key + c0), c), w.x);
-      w.y = fmaf(ng, ih4(mix64(key + c0 + kGamma), c), w.y);
-      w.z = fmaf(ng, ih4(mix64(key + c0 + 2 * kGamma), c), w.z);
-      w.w = fmaf(ng, ih4(mix64(key + c0 + 3 * kGamma), c), w.w);
+      const float g0 = ih4(mix64(key + c0), c), g1 = ih4(mix64(key + c0 + kGamma), c);
+      const float g2 = ih4(mix64(key + c0 + 2 * kGamma), c);
+      const float g3 = ih4(mix64(key + c0 + 3 * kGamma), c);
+      if (MOM) {
+        msgd(w.x, u.x, g0, gamma, mom.beta);
+        msgd(w.y, u.y, g1, gamma, mom.beta);
+        msgd(w.z, u.z, g2, gamma, mom.beta);
+        msgd(w.w, u.w, g3, gamma, mom.beta);
+      } else {
+        w.x = fmaf(ng, g0, w.x);
+        w.y = fmaf(ng, g1, w.y);
+        w.z = fmaf(ng, g2, w.z);
+        w.w = fmaf(ng, g3, w.w);
+      }
     }
     __stcs(row4 + q, w);
+    if (MOM) __stcs(urow4 + q, u);
   }
   if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {
     const int64_t i = (n4 << 2) + threadIdx.x;
     float w = in[i];
-    for (int k = 0; k < K; ++k) w = fmaf(ng, ih4(fold(keys[k], (uint64_t)i), c), w);
+    float u = (MOM && mom.read_u) ? urow[i] : 0.f;
+    for (int k = 0; k < K; ++k) {
+      const float gk = ih4(fold(keys[k], (uint64_t)i), c);
+      if (MOM) msgd(w, u, gk, gamma, mom.beta);
+      else w = fmaf(ng, gk, w);
+    }
     row[i] = w;
+    if (MOM) urow[i] = u;
   }
 }
 
@@ -68,11 +92,18 @@ cudaError_t launch_pseudograd_steps(mavg_ctx* c, int64_t round) {
     int kc = K - k0 < kMaxFused ? K - k0 : kMaxFused;
     dim3 grid((unsigned)blocks_x, (unsigned)P);
     const bool from_global = c->replicas_equal_global;
+    const MomArgs mom = mom_args(c, from_global);
     prof_begin(c, MAVG_K_PSEUDOGRAD);
-    k_pseudograd_steps<<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
-        c->buf.replicas, c->buf.replica_stride, from_global ? c->buf.global_w : c->buf.replicas,
-        from_global ? 0 : c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
-        c->cfg.local_lr);
+    if (mom.u)
+      k_pseudograd_steps<true><<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
+          c->buf.replicas, c->buf.replica_stride, from_global ? c->buf.global_w : c->buf.replicas,
+          from_global ? 0 : c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
+          c->cfg.local_lr, mom);
+    else
+      k_pseudograd_steps<false><<<grid, 256, (size_t)kc * sizeof(uint64_t), c->stream>>>(
+          c->buf.replicas, c->buf.replica_stride, from_global ? c->buf.global_w : c->buf.replicas,
+          from_global ? 0 : c->buf.replica_stride, n, kc, c->cfg.seed, round, k0 + 1, scale,
+          c->cfg.local_lr, mom);
     prof_end(c);
     c->replicas_equal_global = false;
     c->replicas_materialized = true;

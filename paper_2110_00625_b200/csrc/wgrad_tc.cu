@@ -13,6 +13,9 @@
 //                   shared memory and write the bf16 tile beside it;
 //   store warp      one thread sends the two finished tiles back with TMA stores and frees the
 //                   slot once they have left shared memory.
+// With learner-level momentum (MOM) the tile of u^j travels with the master tile: loaded into the
+// same slot (unless the momentum is reset at this step), updated in place (u <- beta u - gamma dW;
+// W <- W + u) and stored back, 18 bytes per weight instead of 10.
 // Edge tiles need no predicates: TMA zero-fills loads and clips stores at the tensor bounds.
 #include <cuda.h>
 
@@ -61,9 +64,12 @@ struct WgradArgs {
   int slots;               // ring depth
   int a_bufs;              // 1 or 2 buffers for the dZ^T tile
   float gamma;
+  float beta;              // learner momentum (MOM)
+  int read_u;              // 0: the stored u counts as zero and is not loaded
   int* status;
 };
 
+template <bool MOM>
 __global__ void __launch_bounds__(kThreads)
 k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out, B]  load
                    const __grid_constant__ CUtensorMap tm_at,    // bf16 [P, in, B]   load
@@ -72,6 +78,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
                                                                    // array, or w~ [1, out, in] at
                                                                    // the first step of a round
                    const __grid_constant__ CUtensorMap tm_w16,   // bf16 [P, out, in] store
+                   const __grid_constant__ CUtensorMap tm_u,     // fp32 [P, out, in] u^j, load + store (MOM)
                    const WgradArgs g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
@@ -85,7 +92,9 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
   const int b_bytes = g.nkb * kBN * kBK * 2;         // A^T tile:  nkb slabs of 4 KB
-  const int slot_bytes = kW32Bytes + kW16Bytes + b_bytes;   // multiple of 1024
+  constexpr int kUBytes = MOM ? kW32Bytes : 0;              // the u tile follows the bf16 tile
+  constexpr int kBOff = kW32Bytes + kW16Bytes + kUBytes;    // the A^T slabs come last
+  const int slot_bytes = kBOff + b_bytes;                   // multiple of 1024
   uint8_t* a_base = smem;
   uint8_t* slot_base = smem + (size_t)g.a_bufs * a_bytes;
 
@@ -96,6 +105,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     tma_prefetch_desc(&tm_w32);
     tma_prefetch_desc(&tm_w32_in);
     tma_prefetch_desc(&tm_w16);
+    if (MOM) tma_prefetch_desc(&tm_u);
     for (int s = 0; s < g.slots; ++s) {
       mbar_init(&slot_full[s], 1);
       mbar_init(&slot_empty[s], 1);
@@ -156,10 +166,13 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           }
           uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
-          mbar_arrive_expect_tx(&slot_full[s], (uint32_t)(kW32Bytes + b_bytes));
+          const bool load_u = MOM && g.read_u;
+          mbar_arrive_expect_tx(&slot_full[s],
+                                (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0)));
           tma_load_3d(sl, &tm_w32_in, &slot_full[s], i0, m0, g.w32_in_batched ? p : 0);
+          if (load_u) tma_load_3d(sl + kW32Bytes + kW16Bytes, &tm_u, &slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
-            tma_load_3d(sl + kW32Bytes + kW16Bytes + (size_t)kb * (kBN * kBK * 2),
+            tma_load_3d(sl + kBOff + (size_t)kb * (kBN * kBK * 2),
                         &tm_at, &slot_full[s], kb * kBK, i0, p);
         }
       }
@@ -188,8 +201,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
             break;
           }
           tc_fence_after_sync();
-          const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + kW32Bytes +
-                                           kW16Bytes);
+          const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + kBOff);
           for (int kb = 0; kb < g.nkb; ++kb) {
             const uint64_t adesc = smem_desc_k_sw128(a_addr + kb * (kBM * kBK * 2));
             const uint64_t bdesc = smem_desc_k_sw128(b_addr + kb * (kBN * kBK * 2));
@@ -240,10 +252,22 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
         for (int c = 0; c < 8; ++c) {
           float4* cell = reinterpret_cast<float4*>(w32 + ((c ^ (r & 7)) << 4));
           float4 w = *cell;
-          w.x = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 0]), w.x);
-          w.y = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 1]), w.y);
-          w.z = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 2]), w.z);
-          w.w = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 3]), w.w);
+          if (MOM) {
+            // the u tile has the master tile's shape and swizzle
+            float4* ucell = reinterpret_cast<float4*>(w32 + kW32Bytes + kW16Bytes +
+                                                      ((c ^ (r & 7)) << 4));
+            float4 u = g.read_u ? *ucell : make_float4(0.f, 0.f, 0.f, 0.f);
+            msgd(w.x, u.x, __uint_as_float(acc[4 * c + 0]), g.gamma, g.beta);
+            msgd(w.y, u.y, __uint_as_float(acc[4 * c + 1]), g.gamma, g.beta);
+            msgd(w.z, u.z, __uint_as_float(acc[4 * c + 2]), g.gamma, g.beta);
+            msgd(w.w, u.w, __uint_as_float(acc[4 * c + 3]), g.gamma, g.beta);
+            *ucell = u;
+          } else {
+            w.x = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 0]), w.x);
+            w.y = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 1]), w.y);
+            w.z = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 2]), w.z);
+            w.w = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 3]), w.w);
+          }
           *cell = w;
           __nv_bfloat162 h0 = __floats2bfloat162_rn(w.x, w.y);
           __nv_bfloat162 h1 = __floats2bfloat162_rn(w.z, w.w);
@@ -277,6 +301,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
           const int i0 = (nt0 + j) * kBN;
           tma_store_3d(&tm_w32, sl, i0, m0, p);
           tma_store_3d(&tm_w16, sl + kW32Bytes, i0, m0, p);
+          if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes + kW16Bytes, i0, m0, p);
           tma_store_commit();
           // the slot of the previous tile is free once its stores have read shared memory
           if (tile_ctr > 0) {
@@ -297,7 +322,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
 
 }  // namespace
 
-WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count) {
+WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum) {
   WgradPlan w{};
   w.nkb = (B + kBK - 1) / kBK;
   w.m_tiles = (out + kBM - 1) / kBM;
@@ -311,7 +336,7 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count) {
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
   w.items = P * w.m_tiles * w.n_chunks;
   const int a_bytes = w.nkb * kBM * kBK * 2;
-  const int slot_bytes = kW32Bytes + kW16Bytes + w.nkb * kBN * kBK * 2;
+  const int slot_bytes = kW32Bytes + kW16Bytes + (momentum ? kW32Bytes : 0) + w.nkb * kBN * kBK * 2;
   const int budget = 220 * 1024;
   w.a_bufs = 2;
   w.slots = (budget - 2 * a_bytes) / slot_bytes;
@@ -326,13 +351,17 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count) {
 }
 
 cudaError_t wgrad_stream_prepare() {
-  return cudaFuncSetAttribute(k_wgrad_sgd_stream, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              225 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(k_wgrad_sgd_stream<false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_wgrad_sgd_stream<true>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
 }
 
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16, const CUtensorMap* w32_shared) {
+                                const CUtensorMap& w16, const CUtensorMap* w32_shared,
+                                const CUtensorMap* u32, const MomArgs& mom) {
   WgradArgs g{};
   g.w32_in_batched = w32_shared ? 0 : 1;
   g.nkb = w.nkb;
@@ -344,6 +373,8 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
   g.gamma = c->cfg.local_lr;
+  g.beta = mom.beta;
+  g.read_u = mom.read_u;
   g.status = (int*)ws_ptr(c, c->ws.status);
   cudaLaunchConfig_t lc{};
   lc.gridDim = dim3((unsigned)w.grid);
@@ -356,8 +387,11 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   lc.attrs = at_;
   lc.numAttrs = 1;
   prof_begin(c, MAVG_K_WGRAD_SGD);
-  cudaError_t e = cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream, dzt, at, w32,
-                                     w32_shared ? *w32_shared : w32, w16, g);
+  cudaError_t e = (mom.u && u32)
+      ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<true>, dzt, at, w32,
+                           w32_shared ? *w32_shared : w32, w16, *u32, g)
+      : cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<false>, dzt, at, w32,
+                           w32_shared ? *w32_shared : w32, w16, w32, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
 }

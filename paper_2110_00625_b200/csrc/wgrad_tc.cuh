@@ -14,15 +14,17 @@ struct WgradPlan {
 constexpr int kWgradTileRows = 128;   // rows of out per tile (box rows of the dZ^T and master maps)
 constexpr int kWgradTileCols = 32;    // columns of in per tile
 
-WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count);
+WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum = false);
 cudaError_t wgrad_stream_prepare();
 // dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
 // w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128
 // (64B swizzle).  w32_shared, if given, is an fp32 [1, out, in] view of w~ with the same box: the
 // masters are then loaded from it for every learner (first step of a round, all w^j = w~) and
-// stored to w32 as always.
+// stored to w32 as always.  With learner-level momentum (mom.u set; the plan made with
+// momentum = true) u32 is the fp32 [P, out, in] view of the buffers u^j with w32's box.
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
-                                const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr);
+                                const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr,
+                                const CUtensorMap* u32 = nullptr, const MomArgs& mom = MomArgs());
 
 }  // namespace mavg

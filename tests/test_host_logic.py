@@ -45,6 +45,8 @@ def _cfg(**kw):
     (dict(P=0), 1), (dict(K=0), 1), (dict(mu=1.0), 1), (dict(mu=-0.1), 1),
     (dict(mu=float("nan")), 1), (dict(local_lr=float("inf")), 1), (dict(block_lr=float("nan")), 1),
     (dict(n=0), 1), (dict(objective=7), 1),
+    (dict(objective=1, learner_momentum=1.0), 1), (dict(objective=1, learner_momentum=-0.5), 1),
+    (dict(learner_momentum=0.5), 1),      # no learner level to apply it to
     (dict(objective=1, sigma=-1.0), 1),
     (dict(objective=2, dims=[4, 3], n=15, B=0, x_ptr=256, y_ptr=256, n_samples=10), 1),
     (dict(objective=2, dims=[4, 3], n=14, B=2, x_ptr=256, y_ptr=256, n_samples=10), 1),
@@ -79,10 +81,17 @@ def test_workspace_size_and_buffer_checks(lib):
         (Buffers(256, 96, 256, 256, 256, 1 << 20), 2),
         (Buffers(256, 100, 256, 256, 256, 16), 2),
         (Buffers(264, 100, 256, 256, 256, 1 << 20), 2),
+        (Buffers(256, 100, 256, 256, 256, 1 << 20, 264), 2),   # misaligned learner_u
     ]:
         assert lib.mavg_create(C.byref(cfg), C.byref(buf), C.byref(h)) == st
         assert h.value is None
         h = C.c_void_p(1)
+    # learner momentum without its buffer
+    cfg_m = _cfg(objective=1, learner_momentum=0.5)
+    assert lib.mavg_create(C.byref(cfg_m), C.byref(Buffers(256, 100, 256, 256, 256, 1 << 20)),
+                           C.byref(h)) == 2
+    assert b"learner_u" in lib.mavg_last_error(None)
+    h = C.c_void_p(1)
     assert lib.mavg_create(C.byref(cfg), None, C.byref(h)) == 1
     assert lib.mavg_create(C.byref(cfg), C.byref(Buffers(256, 100, 256, 256, 256, 1 << 20)), None) == 1
     # NULL handles

@@ -171,7 +171,7 @@ NCU_TRAFFIC_C2 = {
 }
 
 
-def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False):
+def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
@@ -189,7 +189,8 @@ def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False):
                            flops=K * 2 * rows * sum(nW[1:])),
         # fp32 master read + written, bf16 copy written; on the tensor-core path the first step
         # of a round reads the one copy of w~ instead of P masters
-        "wgrad_sgd_gemm": dict(bytes=K * (P * 10 * sum(nW) + 2 * rows * sum(dims))
+        # (learner momentum: the fp32 u tile read and written as well)
+        "wgrad_sgd_gemm": dict(bytes=K * (P * (18 if momentum else 10) * sum(nW) + 2 * rows * sum(dims))
                                - (4 * (P - 1) * sum(nW) if tensor_path else 0),
                                flops=K * 2 * rows * sum(nW)),
     }
@@ -270,7 +271,8 @@ def run_pseudograd(args, m, torch, peaks, rank):
     out = []
     for K in cfg["K"]:
         g = m.Mavg(w1, P=P, K=K, local_lr=cfg["gamma"], mu=0.9, seed=W.BASE_SEED,
-                   objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"], defer_broadcast=not args.no_defer)
+                   objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"], defer_broadcast=not args.no_defer,
+                   learner_momentum=args.beta)
         for _ in range(3):
             g.round()
         g.sync()
@@ -285,7 +287,8 @@ def run_pseudograd(args, m, torch, peaks, rank):
         meta_b = ((8 if args.no_defer else 4) * P + 16) * n
         out.append(dict(K=K, local_ms=loc, meta_ms=met, round_ms=loc + met,
                         learner_steps_per_s=P * K / ((loc + met) * 1e-3),
-                        local_gbs=(4 * P + 4) * n / loc / 1e6,
+                        local_gbs=((12 if args.beta else 4) * P + 4) * n / loc / 1e6,
+                        learner_momentum=args.beta,
                         variates_per_s=P * K * n / (loc * 1e-3),
                         meta_gbs=meta_b / met / 1e6,
                         meta_frac_measured=meta_b / met / 1e6 / peaks["hbm_gbs"],
@@ -336,7 +339,7 @@ def run_mavg(args):
     g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"],
                block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
                dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}",
-               defer_broadcast=not args.no_defer)
+               defer_broadcast=not args.no_defer, learner_momentum=args.beta)
     units = cfg["P"] * cfg["K"] * cfg["B"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
 
@@ -396,7 +399,8 @@ def run_mavg(args):
         g.round()
     prof = g.get_profile(reset=True)
     g.set_profiling(False)
-    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1, deferred=not args.no_defer)
+    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1, deferred=not args.no_defer,
+                            momentum=args.beta != 0.0)
 
     total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=g.device)
 
@@ -421,7 +425,7 @@ def run_mavg(args):
                         "unit": "GB/s", "frac": e["frac_hbm"], "traffic": None}
             roof["kernel"] = dom
             roof["peak_source"] = peaks["source"]
-            if args.workload == "C2" and mode == 1 and not args.learners:
+            if args.workload == "C2" and mode == 1 and not args.learners and not args.beta:
                 roof["traffic"] = NCU_TRAFFIC_C2.get(dom)
         sweep = meta_update_sweep(m, torch, peaks) if world == 1 and not args.no_sweep else None
         n = g.n
@@ -436,7 +440,7 @@ def run_mavg(args):
                        "global_batch": cfg["P"] * cfg["B"], "parallelism": "replicas only",
                        "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
                                 0: "CUDA cores fp32"}[mode],
-                       "defer_broadcast": not args.no_defer,
+                       "defer_broadcast": not args.no_defer, "learner_momentum": args.beta,
                        "l2": "flushed between steps by a 256 MiB memset outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
@@ -475,6 +479,8 @@ def main():
                     help="override P (for small profiler captures; not a benchmark setting)")
     ap.add_argument("--sweep-only", action="store_true",
                     help="run only the meta-update sweep (profiler captures)")
+    ap.add_argument("--beta", type=float, default=0.0,
+                    help="learner-level momentum (0 = Algorithm 1 as printed, the benchmark setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-defer", action="store_true",

@@ -201,6 +201,14 @@ typedef enum {
   MAVG_K_COUNT = 9
 } mavg_kernel_class;
 mavg_status mavg_set_profiling(mavg_handle h, int32_t on);
+/* Schedule of the tensor-core MLP learner level (the paper has no counterpart).  on = 0, the
+ * default: one launch per matrix product, the K steps of a round replayed from a CUDA graph.
+ * on = 1: where the shapes allow it (2 to 5 layers, no product that splits its contraction over
+ * blocks, no learner-level momentum), the K local steps of a round run as ONE persistent kernel
+ * whose blocks hand work to each other through counters in the workspace; other shapes keep the
+ * graph.  Both schedules run the same tiles and compute the same bits; profiled rounds
+ * (mavg_set_profiling) always take the per-launch schedule. */
+mavg_status mavg_set_round_kernel(mavg_handle h, int32_t on);
 mavg_status mavg_get_profile(mavg_handle h, float *ms, int64_t *launches, int32_t reset);
 
 /* Waits for the stream; reports CUDA errors and a tripped device-side wait limit. */

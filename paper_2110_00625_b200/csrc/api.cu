@@ -402,6 +402,12 @@ mavg_status mavg_set_profiling(mavg_handle h, int32_t on) {
   return MAVG_OK;
 }
 
+mavg_status mavg_set_round_kernel(mavg_handle h, int32_t on) {
+  CHECK_HANDLE(h);
+  h->round_kernel = on != 0;
+  return MAVG_OK;
+}
+
 mavg_status mavg_get_profile(mavg_handle h, float* ms, int64_t* launches, int32_t reset) {
   CHECK_HANDLE(h);
   if (!ms || !launches) return set_err(h, MAVG_ERR_INVALID_ARG, "ms or launches is NULL");

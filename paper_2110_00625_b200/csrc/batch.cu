@@ -8,16 +8,6 @@
 namespace mavg {
 namespace {
 
-// idx = lo_j + floor(u * len_j / 2^32), u = top 32 bits of the stream value (see mavg.h).
-__device__ __forceinline__ int32_t sample_index(uint64_t seed, int64_t round, int j, int step,
-                                                int s, int P, int64_t S) {
-  int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
-  int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
-  uint64_t key = fold(learner_key(seed, kTagBatch, (uint64_t)round, (uint64_t)j), (uint64_t)step);
-  uint64_t u = fold(key, (uint64_t)s) >> 32;
-  return (int32_t)(lo + (int64_t)((u * (uint64_t)(hi - lo)) >> 32));
-}
-
 // One thread per (learner, slot).  Also fetches the label.
 __global__ void k_batch_indices(int32_t* __restrict__ idx, int32_t* __restrict__ labels,
                                 const int32_t* __restrict__ y, uint64_t seed, int64_t round,

@@ -106,6 +106,7 @@ struct mavg_ctx {
   int cls_open = 0;
   // CUDA graph of one round's K local steps (MLP objective): captured once on a private stream,
   // replayed on the caller's stream; rebuilt when K or the local learning rate change
+  bool round_kernel = false;  // MLP tensor-core path: run a round's K steps as one kernel where covered
   bool capturing = false;
   bool graph_disabled = false;
   cudaGraphExec_t graph_exec = nullptr;

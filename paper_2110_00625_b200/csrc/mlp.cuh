@@ -5,6 +5,16 @@
 
 namespace mavg {
 
+// idx = lo_j + floor(u * len_j / 2^32), u = top 32 bits of the stream value (see mavg.h).
+__device__ __forceinline__ int32_t sample_index(uint64_t seed, int64_t round, int j, int step,
+                                                int s, int P, int64_t S) {
+  int64_t lo = (int64_t)(((unsigned __int128)j * (unsigned __int128)S) / (unsigned)P);
+  int64_t hi = (int64_t)(((unsigned __int128)(j + 1) * (unsigned __int128)S) / (unsigned)P);
+  uint64_t key = fold(learner_key(seed, kTagBatch, (uint64_t)round, (uint64_t)j), (uint64_t)step);
+  uint64_t u = fold(key, (uint64_t)s) >> 32;
+  return (int32_t)(lo + (int64_t)((u * (uint64_t)(hi - lo)) >> 32));
+}
+
 // batch.cu
 cudaError_t launch_batch_indices(mavg_ctx* c, int64_t round, int step, int j_first, int j_count,
                                  int32_t* idx, int32_t* labels);
@@ -28,6 +38,10 @@ mavg_status tc_setup(mavg_ctx* c);
 void tc_teardown(mavg_ctx* c);
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c);
 cudaError_t tc_step(mavg_ctx* c, int64_t round, int step);
+
+// Whole-round kernel (round_tc.cu): all K local steps of a round in one launch.
+bool tc_round_supported(mavg_ctx* c);
+cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
 
 inline bool use_tensor_cores(const mavg_config* cfg) { return cfg->gemm_bf16 == 1; }
 

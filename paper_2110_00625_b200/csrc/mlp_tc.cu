@@ -23,8 +23,10 @@
 
 #include <algorithm>
 
+#include "gemm_unit.cuh"
 #include "mlp.cuh"
 #include "tc_ptx.cuh"
+#include "tc_state.cuh"
 #include "wgrad_tc.cuh"
 
 namespace mavg {
@@ -32,68 +34,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kBM = 128;        // MMA M (rows of operand A per tile)
-constexpr int kBK = 64;         // contraction elements per pipeline stage (128 bytes of bf16)
 constexpr int kThreads = 320;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
-constexpr int kMaxStages = 8;
-constexpr int kATileBytes = kBM * kBK * 2;
-
-enum { EPI_FWD_HIDDEN = 0, EPI_FWD_LAST = 1, EPI_DGRAD = 2 };
-enum { ERR_PRODUCER = 11, ERR_MMA = 12, ERR_EPILOGUE = 13 };
-
-struct TcArgs {
-  int M, N;                 // valid rows of A and of B
-  int BN;                   // N tile: multiple of 16, <= 256
-  int m_tiles, n_tiles, splits, kb_per_split, nkb, stages;
-  int a_batched, b_batched; // 0: the operand is shared by all learners
-  int a_mn;                 // 1: A is read MN-major from a [K rows, M contiguous] array (dgrad: W itself)
-  int P;
-  uint32_t tmem_cols;
-  // forward / dgrad: A rows are features m (M of them), B rows the batch (N = B of them)
-  float* part;              // split partials, part[((split*P + p)*N + n)*M + m]
-  int* counters;            // one per (p, m_tile); zero between launches
-  float* bias_rep;          // fp32 masters; the bias this kernel reads (forward) or steps (dgrad,
-  int64_t bias_off;         // last layer) is at bias_rep[p*rep_stride + bias_off + m]
-  const float* bias_in;     // where the bias is read: bias_in[p*bias_in_stride + bias_off + m], the
-  int64_t bias_in_stride;   // same place, or w~ (stride 0) at the first step of a round
-  __nv_bfloat16* out_bm;    // [P, B, M]  relu(z) (forward) or dZ (dgrad)
-  __nv_bfloat16* out_mb;    // [P, M, B]  the same, transposed
-  const __nv_bfloat16* mask_mb;  // dgrad: forward activation [P, M, B] whose sign gates dZ
-  // last layer (M = classes <= 32): loss, dZ_L and the bias step
-  const int32_t* labels;    // [P*B]
-  float* loss_out;          // loss_out[p*loss_stride]
-  int loss_stride;
-  __nv_bfloat16* dz_bm;     // [P, B, cpad]
-  int cpad;
-  __nv_bfloat16* dz_mb;     // [P, M, B]
-  int64_t rep_stride;
-  float gamma;
-  MomArgs mom;              // learner momentum of the bias this kernel steps (slots laid out like bias_rep)
-  int* status;
-};
-
-// Synchronises the 8 epilogue warps (256 threads) without the producer and MMA warps.
-__device__ __forceinline__ void epilogue_barrier() {
-  asm volatile("bar.sync 1, 256;" ::: "memory");
-}
-
-// 32 accumulator columns starting at c0 for this warp's 32 lanes (16 when the tile ends there;
-// the rest reads as zero).  Returns the number of valid columns.  Warp-collective.
-__device__ __forceinline__ int load_acc_chunk(uint32_t lane_addr, int c0, int BN, float (&z)[32]) {
-  uint32_t r[32];
-  if (c0 + 32 <= BN) {
-    tmem_ld_32x32(lane_addr + (uint32_t)c0, r);
-  } else {                                   // BN is a multiple of 16
-    uint32_t h[16];
-    tmem_ld_16cols(lane_addr + (uint32_t)c0, h);
-#pragma unroll
-    for (int j = 0; j < 16; ++j) { r[j] = h[j]; r[16 + j] = 0u; }
-  }
-  tmem_ld_wait();
-#pragma unroll
-  for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(r[j]);
-  return min(32, BN - c0);
-}
+using namespace gemm;
 
 // MINB = 2 caps the registers so that two blocks fit an SM (used when a launch has more blocks
 // than SMs; costs a few spills in the tail), MINB = 1 leaves the compiler free.
@@ -102,330 +44,35 @@ __global__ void __launch_bounds__(kThreads, MINB)
 k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
           const TcArgs g) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[kMaxStages];
-  __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-  __shared__ __align__(8) uint64_t acc_bar;
-  __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag;
-  __shared__ int last_flag;
-  __shared__ float colsum[2][kBM];
+  __shared__ __align__(8) GemmShared sh;
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~(uintptr_t)1023);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int stage_bytes = kATileBytes + g.BN * kBK * 2;
-  const int stages = g.stages;
-
-  const int split = blockIdx.x % g.splits;
-  const int tile = blockIdx.x / g.splits;
-  const int n_tile = tile % g.n_tiles, m_tile = tile / g.n_tiles;
-  const int p = blockIdx.y;
-  const int m0 = m_tile * kBM, n0 = n_tile * g.BN;
-  const int kb0 = split * g.kb_per_split;
-  const int kb1 = min(g.nkb, kb0 + g.kb_per_split);
-  const int count = kb1 - kb0;
+  const int warp = threadIdx.x >> 5;
 
   grid_launch_dependents();   // the next kernel may begin its own set-up early
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], 1);
-    }
-    mbar_init(&acc_bar, 1);
-    abort_flag = 0;
+    gemm_init_barriers(sh, g.stages);
+    sh.abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
   if (warp == 1) {
-    tmem_alloc(&tmem_slot, g.tmem_cols);
+    tmem_alloc(&sh.tmem_slot, g.tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_base = sh.tmem_slot;
   // Everything above touched only this block's own shared and tensor memory.  When the launch
   // allowed it, that much ran while the previous kernel of the stream was still finishing; from
   // here on its results are read, so wait for it to complete (returns at once otherwise).
   grid_dependency_wait();
-  volatile int* abortp = &abort_flag;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      int issued = 0;
-      for (int i = 0; i < count; ++i) {
-        const int s = i % stages, u = i / stages;
-        if (!mbar_wait(&empty_bar[s], (u & 1) ^ 1, abortp, g.status, ERR_PRODUCER)) break;
-        uint8_t* sa = smem + (size_t)s * stage_bytes;
-        mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
-        if (g.a_mn) {     // two 64-wide halves of the M range, each 64 K-rows of 128 bytes
-          tma_load_3d(sa, &tmA, &full_bar[s], m0, (kb0 + i) * kBK, g.a_batched ? p : 0);
-          tma_load_3d(sa + kATileBytes / 2, &tmA, &full_bar[s], m0 + 64, (kb0 + i) * kBK,
-                      g.a_batched ? p : 0);
-        } else {
-          tma_load_3d(sa, &tmA, &full_bar[s], (kb0 + i) * kBK, m0, g.a_batched ? p : 0);
-        }
-        tma_load_3d(sa + kATileBytes, &tmB, &full_bar[s], (kb0 + i) * kBK, n0,
-                    g.b_batched ? p : 0);
-        issued = i + 1;
-      }
-      if (*abortp) {
-        // give the copies already issued a bounded chance to land before the block retires
-        for (int i = max(0, issued - stages); i < issued; ++i) {
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(&full_bar[i % stages], (i / stages) & 1))
-            if (global_timer_ns() - t0 > kWaitLimitNs) break;
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    if (lane == 0) {
-      const uint32_t idesc = idesc_bf16_f32(kBM, g.BN, g.a_mn);
-      bool ok = true;
-      for (int i = 0; i < count; ++i) {
-        const int s = i % stages, u = i / stages;
-        if (!mbar_wait(&full_bar[s], u & 1, abortp, g.status, ERR_MMA)) { ok = false; break; }
-        tc_fence_after_sync();
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t adesc = g.a_mn ? smem_desc_mn_sw128(sa) : smem_desc_k_sw128(sa);
-        const uint64_t bdesc = smem_desc_k_sw128(sa + kATileBytes);
-        // per MMA (16 K-elements) a K-major tile advances 32 bytes inside its 128-byte rows, an
-        // MN-major tile 16 rows of 128 bytes; descriptor addresses count 16-byte units
-        const uint32_t a_step = g.a_mn ? (16 * 128) >> 4 : 2;
-#pragma unroll
-        for (int k = 0; k < kBK / 16; ++k)
-          umma_bf16(tmem_base, adesc + a_step * k, bdesc + 2 * k, idesc, (uint32_t)((i | k) != 0));
-        umma_commit(&empty_bar[s]);
-      }
-      if (ok) umma_commit(&acc_bar);
-    }
-    __syncwarp();
-  } else {
-    // 8 epilogue warps: warp (q, half) owns TMEM lanes [32q, 32q+32) -- the only lanes a warp
-    // with (warp index mod 4) == q may read -- and every second 32-column chunk.
-    const int ew = warp - 2;
-    const int q = warp & 3;
-    const int half = ew >> 2;
-    const int row = q * 32 + lane;
-    // Operands of the tail that do not depend on the accumulator are fetched while the main loop
-    // is still running: the bias (read by the forward tails, stepped by the dgrad tail), the
-    // first mask chunk (dgrad) and the label of this thread's batch row (last layer).
-    float* bias = g.bias_rep + (size_t)p * g.rep_stride + g.bias_off;
-    const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride + g.bias_off;
-    const bool m_ok_pre = m0 + row < g.M;
-    const float bias_pre = (m_ok_pre && (EPI != EPI_DGRAD || half == 0)) ? bias_in[m0 + row] : 0.f;
-    uint4 mk[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
-                   make_uint4(0, 0, 0, 0)};
-    auto load_mask = [&](int c0, uint4 (&dst)[4]) {
-      if (!m_ok_pre || c0 >= g.BN) return;
-      const uint4* msrc = reinterpret_cast<const uint4*>(
-          g.mask_mb + ((size_t)p * g.M + m0 + row) * g.N + n0 + c0);
-      if (n0 + c0 + 32 <= g.N) {               // whole chunk inside the batch: 4 loads in flight
-#pragma unroll
-        for (int v = 0; v < 4; ++v) dst[v] = msrc[v];
-      } else {
-#pragma unroll
-        for (int v = 0; v < 4; ++v)
-          dst[v] = n0 + c0 + v * 8 < g.N ? msrc[v] : make_uint4(0, 0, 0, 0);
-      }
-    };
-    // (only in the one-block-per-SM build: the register-capped build has no room to hold it)
-    if (EPI == EPI_DGRAD) load_mask(half * 32, mk);
-    int label_pre = 0;
-    if (EPI == EPI_FWD_LAST && ew * 32 + lane < g.N)
-      label_pre = g.labels[(size_t)p * g.N + ew * 32 + lane];
-    const bool ok = mbar_wait(&acc_bar, 0, abortp, g.status, ERR_EPILOGUE);
-    tc_fence_after_sync();
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    {
-      // forward / dgrad: feature m per lane, the batch along the columns (the dgrad and last-layer
-      // tails need the whole batch in one tile: n_tiles == 1 there)
-      const int m = m0 + row;
-      const bool m_ok = m < g.M;
-      bool finisher = ok;
-      if (MINB == 1 && g.splits > 1) {   // the register-capped build is never used with a split
-        if (ok) {
-          float* dst = g.part + ((size_t)(split * g.P + p) * g.N) * g.M + m;
-          for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
-            float z[32];
-            const int ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
-            if (m_ok) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols && n0 + c0 + j < g.N) dst[(size_t)(n0 + c0 + j) * g.M] = z[j];
-            }
-          }
-        }
-        // the block that publishes the last of the `splits` partials of this tile finishes it
-        __threadfence();
-        epilogue_barrier();
-        if (ew == 0 && lane == 0) {
-          int* ctr = g.counters + (p * g.m_tiles + m_tile) * g.n_tiles + n_tile;
-          const int old = ok ? atomicAdd(ctr, 1) : -1;
-          const int last = old == g.splits - 1;
-          if (last) *ctr = 0;
-          __threadfence();
-          last_flag = last;
-        }
-        epilogue_barrier();
-        finisher = last_flag != 0;
-      }
-      if (finisher) {
-        const float my_bias = EPI != EPI_DGRAD ? bias_pre : 0.f;
-        float dsum = 0.f;
-        float* lg = reinterpret_cast<float*>(smem);          // last layer: logits [N][M]
-        for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
-          float z[32];
-          int ncols;
-          if (MINB != 1 || g.splits == 1) {
-            ncols = load_acc_chunk(lane_addr, c0, g.BN, z);
-          } else {
-            ncols = min(32, g.BN - c0);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) z[j] = 0.f;
-            if (m_ok) {
-              const int nvalid = min(ncols, g.N - n0 - c0);
-#pragma unroll 2
-              for (int sp = 0; sp < g.splits; ++sp) {        // ascending split order
-                const float* src = g.part + ((size_t)(sp * g.P + p) * g.N + n0 + c0) * g.M + m;
-                float t[32];
-                if (nvalid == 32) {                          // all loads in flight together
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * g.M);
-                } else {
-#pragma unroll
-                  for (int j = 0; j < 32; ++j)
-                    t[j] = __ldcg(src + (size_t)min(j, max(nvalid - 1, 0)) * g.M);
-                }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) z[j] += j < nvalid ? t[j] : 0.f;
-              }
-            }
-          }
-          if (EPI == EPI_FWD_LAST) {
-            if (m_ok) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols && n0 + c0 + j < g.N) lg[(n0 + c0 + j) * g.M + m] = z[j] + my_bias;
-            }
-          } else {
-            uint32_t hp[16];                                  // 32 bf16 results, packed
-            if (EPI == EPI_DGRAD) {
-              uint4 mkn[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
-                              make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-              load_mask(c0 + 64, mkn);                        // next chunk, used one iteration on
-              const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(mk);
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const bool live = j < ncols && n0 + c0 + j < g.N && __bfloat162float(mh[j]) > 0.f;
-                z[j] = live ? z[j] : 0.f;                     // ReLU'(0) = 0
-                dsum += z[j];
-              }
-#pragma unroll
-              for (int v = 0; v < 4; ++v) mk[v] = mkn[v];
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float a = z[j] + my_bias;
-                z[j] = a > 0.f ? a : 0.f;
-              }
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(z[2 * j], z[2 * j + 1]);
-              hp[j] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            if (m_ok) {
-              const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
-              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + c0) * g.M + m;
-              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + c0);
-              if (ncols == 32 && n0 + c0 + 32 <= g.N) {
-#pragma unroll
-                for (int v = 0; v < 4; ++v)
-                  dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) dbm[(size_t)j * g.M] = hh[j];
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                  if (j < ncols && n0 + c0 + j < g.N) dbm[(size_t)j * g.M] = hh[j];
-#pragma unroll
-                for (int v = 0; v < 4; ++v)
-                  if (v * 8 < ncols && n0 + c0 + v * 8 < g.N)
-                    dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
-              }
-            }
-          }
-        }
-        if (EPI == EPI_DGRAD) {
-          // bias step of the layer below: b[m] -= gamma * sum_b dZ[b, m]; the two warps that
-          // share a row add their column sums in a fixed order
-          colsum[half][row] = dsum;
-          epilogue_barrier();
-          if (half == 0 && m_ok) {
-            float* ub = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride + g.bias_off + m : nullptr;
-            local_update(bias + m, bias_pre, ub, g.mom.read_u, colsum[0][row] + colsum[1][row],
-                         g.gamma, g.mom.beta);
-          }
-        }
-        if (EPI == EPI_FWD_LAST) {
-          // softmax cross-entropy on the block's [N, M] logits: thread t takes batch row t
-          float* dzs = lg + g.N * g.M;
-          float* lossp = dzs + g.N * g.M;
-          epilogue_barrier();
-          const int t = ew * 32 + lane;
-          const int C = g.M;
-          if (t < g.N) {
-            const float* zr = lg + t * C;
-            float mx = zr[0];
-            for (int c = 1; c < C; ++c) mx = fmaxf(mx, zr[c]);
-            float se = 0.f;
-            for (int c = 0; c < C; ++c) se += expf(zr[c] - mx);
-            const float lse = mx + logf(se);
-            const int yb = label_pre;
-            lossp[t] = lse - zr[yb];
-            const float inv_b = 1.0f / (float)g.N;
-            for (int c = 0; c < C; ++c) {
-              const float gr = (expf(zr[c] - lse) - (c == yb ? 1.f : 0.f)) * inv_b;
-              dzs[t * C + c] = gr;
-              const __nv_bfloat16 gq = __float2bfloat16_rn(gr);
-              g.dz_bm[((size_t)p * g.N + t) * g.cpad + c] = gq;
-              g.dz_mb[((size_t)p * C + c) * g.N + t] = gq;
-            }
-          }
-          epilogue_barrier();
-          // loss: every warp adds its 32 rows, thread 0 the warps' sums; bias gradient of class c:
-          // a warp adds the rows lane, lane + 32, ... and then its lanes, in a fixed order
-          {
-            float sl = t < g.N ? lossp[t] : 0.f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sl += __shfl_xor_sync(0xffffffffu, sl, o);
-            if (lane == 0) colsum[0][ew] = sl;
-            for (int c = ew; c < C; c += 8) {
-              float sb = 0.f;
-              for (int b = lane; b < g.N; b += 32) sb += dzs[b * C + c];
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
-              if (lane == 0) {
-                float* ub = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride + g.bias_off + c : nullptr;
-                local_update(bias + c, bias_in[c], ub, g.mom.read_u, sb, g.gamma, g.mom.beta);
-              }
-            }
-          }
-          epilogue_barrier();
-          if (t == 0) {
-            float sl = 0.f;
-            const int nw = (g.N + 31) / 32;
-            for (int w = 0; w < nw; ++w) sl += colsum[0][w];
-            g.loss_out[(size_t)p * g.loss_stride] = sl / (float)g.N;
-          }
-        }
-      }
-    }
-  }
+  // the split path is compiled out of the register-capped build, which is never used with a split
+  gemm_tile<EPI, MINB == 1>(tmA, tmB, g, (int)blockIdx.x, (int)blockIdx.y, smem, sh, tmem_base);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, g.tmem_cols);
@@ -443,22 +90,6 @@ k_shadow_from_global(const float* __restrict__ w, int64_t w_off, int64_t total,
 
 // ---------------------------------------------------------------------------------- host side
 size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-struct TcLayout {
-  int L;
-  int cpad;                                  // last layer's dZ row length (multiple of 8)
-  int64_t n16;                               // elements per bf16 copy row
-  int64_t sh_off[MAVG_MAX_LAYERS];
-  size_t xg[2], xt[2];                       // gathered batch, two buffers used by alternate steps
-  size_t act[MAVG_MAX_LAYERS + 1], act_t[MAVG_MAX_LAYERS + 1];
-  size_t dz[MAVG_MAX_LAYERS + 1], dz_t[MAVG_MAX_LAYERS + 1];
-  size_t part, part_bytes;
-  size_t counters, counters_bytes;
-  size_t w16, w16g;
-  size_t end;
-};
-
-struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages, two_per_sm; uint32_t tmem_cols; };
 
 // Forward / dgrad plan.  To fill the GPU the batch may be cut into column tiles (`tile_n`: only
 // the hidden-layer forward can, its tail needs no sum over the batch) and, if blocks are still
@@ -541,6 +172,8 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.counters = take(t.counters_bytes);
   t.w16 = take((size_t)P * t.n16 * 2);
   t.w16g = take((size_t)t.n16 * 2);
+  t.round_ctr_bytes = (size_t)4 * (MAVG_MAX_LAYERS + 1) * P * sizeof(int);
+  t.round_ctr = take(t.round_ctr_bytes);
   t.end = off;
   return t;
 }
@@ -548,35 +181,6 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
 // SM count the plans (and with them the size of the partial buffer) are made for, so that the
 // workspace size does not depend on the device that later runs the problem.
 constexpr int kPlanSmCount = 148;
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-struct TcState {
-  TcLayout lay;
-  EncodeTiledFn encode = nullptr;
-  // per layer l = 1..L (index l)
-  CUtensorMap w[MAVG_MAX_LAYERS + 1], wg[MAVG_MAX_LAYERS + 1];       // [out, in] copies
-  CUtensorMap act_in[MAVG_MAX_LAYERS + 1];    // [B, d_{l-1}] input activations of layer l >= 2
-  CUtensorMap act_in_t[MAVG_MAX_LAYERS + 1];  // [d_{l-1}, B]
-  CUtensorMap x_in[2], x_in_t[2];             // layer 1's input: the two gather buffers
-  CUtensorMap dz[MAVG_MAX_LAYERS + 1];        // [B, d_l]
-  CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
-  CUtensorMap w_mn[MAVG_MAX_LAYERS + 1], wg_mn[MAVG_MAX_LAYERS + 1];  // [out, in] copies, 64 x 64 boxes
-  CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
-  CUtensorMap w32g[MAVG_MAX_LAYERS + 1];      // the same view of w~ (one copy): first-step loads
-  CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
-  CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
-  bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
-  GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
-  WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
-  // side streams and events for the branches of a step that may overlap
-  cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,
-              ev_x_free[2] = {nullptr, nullptr};
-};
 
 // Tensor [batch, rows, inner] with the given strides (in elements) and box inner x box_rows.
 bool encode_any(TcState* st, CUtensorMap* m, CUtensorMapDataType dt, int esize, void* ptr,
@@ -746,6 +350,7 @@ mavg_status tc_setup(mavg_ctx* c) {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
   if (e == cudaSuccess) e = wgrad_stream_prepare();
+  if (e == cudaSuccess) e = tc_round_prepare(c);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);
   cudaEvent_t* evs[] = {&st->ev_fork, &st->ev_wgrad_done, &st->ev_gather_done, &st->ev_x_free[0],

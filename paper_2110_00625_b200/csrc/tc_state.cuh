@@ -1,0 +1,67 @@
+// Host-side state of the tensor-core MLP path: workspace layout, launch plans and tensor maps.
+// Built by mlp_tc.cu, also read by the whole-round kernel's launcher (round_tc.cu).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "wgrad_tc.cuh"
+
+namespace mavg {
+
+struct TcLayout {
+  int L;
+  int cpad;                                  // last layer's dZ row length (multiple of 8)
+  int64_t n16;                               // elements per bf16 copy row
+  int64_t sh_off[MAVG_MAX_LAYERS];
+  size_t xg[2], xt[2];                       // gathered batch, two buffers used by alternate steps
+  size_t act[MAVG_MAX_LAYERS + 1], act_t[MAVG_MAX_LAYERS + 1];
+  size_t dz[MAVG_MAX_LAYERS + 1], dz_t[MAVG_MAX_LAYERS + 1];
+  size_t part, part_bytes;
+  size_t counters, counters_bytes;
+  size_t w16, w16g;
+  size_t round_ctr, round_ctr_bytes;         // completion counters of the whole-round kernel
+  size_t end;
+};
+
+struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages, two_per_sm; uint32_t tmem_cols; };
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  TcLayout lay;
+  EncodeTiledFn encode = nullptr;
+  // per layer l = 1..L (index l)
+  CUtensorMap w[MAVG_MAX_LAYERS + 1], wg[MAVG_MAX_LAYERS + 1];       // [out, in] copies
+  CUtensorMap act_in[MAVG_MAX_LAYERS + 1];    // [B, d_{l-1}] input activations of layer l >= 2
+  CUtensorMap act_in_t[MAVG_MAX_LAYERS + 1];  // [d_{l-1}, B]
+  CUtensorMap x_in[2], x_in_t[2];             // layer 1's input: the two gather buffers
+  CUtensorMap dz[MAVG_MAX_LAYERS + 1];        // [B, d_l]
+  CUtensorMap dz_t[MAVG_MAX_LAYERS + 1];      // [d_l, B]
+  CUtensorMap w_mn[MAVG_MAX_LAYERS + 1], wg_mn[MAVG_MAX_LAYERS + 1];  // [out, in] copies, 64 x 64 boxes
+  CUtensorMap w32[MAVG_MAX_LAYERS + 1];       // fp32 masters [out, in]: wgrad loads and stores
+  CUtensorMap w32g[MAVG_MAX_LAYERS + 1];      // the same view of w~ (one copy): first-step loads
+  CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
+  CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
+  bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
+  // whole-round kernel (round_tc.cu)
+  bool round_ok = false;
+  int round_stages = 0, round_grid = 0;
+  size_t round_smem = 0;
+  GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
+  WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
+  // side streams and events for the branches of a step that may overlap
+  cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,
+              ev_x_free[2] = {nullptr, nullptr};
+};
+
+
+// round_tc.cu: all K local steps of a round in one persistent kernel.
+bool tc_round_supported(mavg_ctx* c);
+cudaError_t tc_round_prepare(mavg_ctx* c);
+cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
+
+}  // namespace mavg

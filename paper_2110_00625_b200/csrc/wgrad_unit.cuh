@@ -1,0 +1,340 @@
+// Roles of the streaming weight-gradient + SGD block (see wgrad_tc.cu for the scheme): shared by
+// the stand-alone kernel and by the whole-round kernel of round_tc.cu.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace mavg {
+namespace wgrad {
+
+using namespace tc;
+
+constexpr int kBM = 128, kBN = 32, kBK = 64;
+constexpr int kThreads = 352;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores
+constexpr int kMaxSlots = 6;
+constexpr int kW32Bytes = kBM * kBN * 4;  // 16 KB, rows of 128 bytes, 128-byte swizzle
+constexpr int kW16Bytes = kBM * kBN * 2;  //  8 KB, rows of  64 bytes,  64-byte swizzle
+enum { ERR_WG_PRODUCER = 21, ERR_WG_MMA = 22, ERR_WG_EPILOGUE = 23, ERR_WG_STORE = 24 };
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* src, int c0, int c1,
+                                             int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Waits until at most `N` of this thread's store groups still have shared memory left to read.
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+struct WgradArgs {
+  int w32_in_batched;      // 0: every learner loads the one shared master array (w~)
+  int nkb;                 // 64-wide slabs of the batch (contraction)
+  int m_tiles, n_tiles;    // 128-row tiles of out, 32-column tiles of in
+  int chunk;               // column tiles per work item
+  int n_chunks;            // ceil(n_tiles / chunk)
+  int items;               // P * m_tiles * n_chunks
+  int slots;               // ring depth
+  int a_bufs;              // 1 or 2 buffers for the dZ^T tile
+  float gamma;
+  float beta;              // learner momentum (MOM)
+  int read_u;              // 0: the stored u counts as zero and is not loaded
+  int* status;
+};
+
+
+// Waits until all but the last N store groups of this thread have been written to global memory.
+constexpr int kStoreLag = 4;
+template <int N>
+__device__ __forceinline__ void tma_store_wait_pending() {
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+// Waits until every store group of this thread has been written to global memory.
+__device__ __forceinline__ void tma_store_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+struct WgradShared {
+  uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
+  uint64_t tmem_full[2], tmem_empty[2];
+  uint64_t a_full[2], a_empty[2];
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+
+__device__ __forceinline__ void wgrad_init_barriers(WgradShared& sh, int slots) {
+  for (int s = 0; s < slots; ++s) {
+    mbar_init(&sh.slot_full[s], 1);
+    mbar_init(&sh.slot_empty[s], 1);
+    mbar_init(&sh.out_full[s], 4);
+  }
+  for (int b = 0; b < 2; ++b) {
+    mbar_init(&sh.tmem_full[b], 1);
+    mbar_init(&sh.tmem_empty[b], 4);
+    mbar_init(&sh.a_full[b], 1);
+    mbar_init(&sh.a_empty[b], 1);
+  }
+}
+
+// Tiles and items of the run (vblock, vgrid) of the launch g: what a later run of the same block
+// adds to tile_base and item_base.
+__device__ __forceinline__ void wgrad_run_totals(const WgradArgs& g, int vblock, int vgrid,
+                                                 uint32_t& tiles, uint32_t& items) {
+  for (int item = vblock; item < g.items; item += vgrid) {
+    const int nt0 = (item % g.n_chunks) * g.chunk;
+    tiles += (uint32_t)min(g.chunk, g.n_tiles - nt0);
+    items += 1;
+  }
+}
+
+// Dependency hooks of a run: the producer thread calls inputs_ready(p) before it loads anything
+// of an item of learner p; with kSignals the store thread calls item_done(p) once the item's
+// tiles have reached global memory.  A stand-alone launch needs neither.
+struct NoDeps {
+  static constexpr bool kSignals = false;
+  __device__ __forceinline__ bool inputs_ready(int, volatile int*) const { return true; }
+  __device__ __forceinline__ void item_done(int) const {}
+};
+
+// Work items vblock, vblock + vgrid, ... of the launch described by g.  Barriers initialised
+// (phase 0) and a block-wide barrier passed before; 64 columns of tensor memory at tmem_base.
+// A block that makes several runs keeps using the same barriers (g.slots and g.a_bufs must not
+// change): tile_base and item_base are the tiles and items of its earlier runs, see
+// wgrad_run_totals.
+template <bool MOM, typename Dep>
+__device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUtensorMap& tm_at,
+                                          const CUtensorMap& tm_w32, const CUtensorMap& tm_w32_in,
+                                          const CUtensorMap& tm_w16, const CUtensorMap& tm_u,
+                                          const WgradArgs& g, int vblock, int vgrid, uint8_t* smem,
+                                          WgradShared& sh, uint32_t tmem_base, const Dep& dep,
+                                          uint32_t tile_base = 0, uint32_t item_base = 0) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
+  const int b_bytes = g.nkb * kBN * kBK * 2;         // A^T tile:  nkb slabs of 4 KB
+  constexpr int kUBytes = MOM ? kW32Bytes : 0;              // the u tile follows the bf16 tile
+  constexpr int kBOff = kW32Bytes + kW16Bytes + kUBytes;    // the A^T slabs come last
+  const int slot_bytes = kBOff + b_bytes;                   // multiple of 1024
+  uint8_t* a_base = smem;
+  uint8_t* slot_base = smem + (size_t)g.a_bufs * a_bytes;
+  volatile int* abortp = &sh.abort_flag;
+
+  // work item -> (learner p, row tile, first column tile, number of column tiles)
+  auto decode = [&](int item, int& p, int& m0, int& nt0, int& nt) {
+    const int nc = item % g.n_chunks;
+    const int rest = item / g.n_chunks;
+    const int mt = rest % g.m_tiles;
+    p = rest / g.m_tiles;
+    m0 = mt * kBM;
+    nt0 = nc * g.chunk;
+    nt = min(g.chunk, g.n_tiles - nt0);
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t tile_ctr = tile_base, item_ctr = item_base;
+      bool ok = true;
+      for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
+        int p, m0, nt0, nt;
+        decode(item, p, m0, nt0, nt);
+        const int ab = item_ctr % g.a_bufs;
+        const uint32_t a_use = item_ctr / g.a_bufs;
+        if (!dep.inputs_ready(p, abortp)) break;
+        if (!mbar_wait(&sh.a_empty[ab], (a_use & 1) ^ 1, abortp, g.status, ERR_WG_PRODUCER)) break;
+        mbar_arrive_expect_tx(&sh.a_full[ab], (uint32_t)a_bytes);
+        for (int kb = 0; kb < g.nkb; ++kb)
+          tma_load_3d(a_base + (size_t)ab * a_bytes + (size_t)kb * (kBM * kBK * 2), &tm_dzt,
+                      &sh.a_full[ab], kb * kBK, m0, p);
+        for (int j = 0; j < nt; ++j, ++tile_ctr) {
+          const int s = tile_ctr % g.slots;
+          const uint32_t use = tile_ctr / g.slots;
+          if (!mbar_wait(&sh.slot_empty[s], (use & 1) ^ 1, abortp, g.status, ERR_WG_PRODUCER)) {
+            ok = false;
+            break;
+          }
+          uint8_t* sl = slot_base + (size_t)s * slot_bytes;
+          const int i0 = (nt0 + j) * kBN;
+          const bool load_u = MOM && g.read_u;
+          mbar_arrive_expect_tx(&sh.slot_full[s],
+                                (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0)));
+          tma_load_3d(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0);
+          if (load_u) tma_load_3d(sl + kW32Bytes + kW16Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
+          for (int kb = 0; kb < g.nkb; ++kb)
+            tma_load_3d(sl + kBOff + (size_t)kb * (kBN * kBK * 2),
+                        &tm_at, &sh.slot_full[s], kb * kBK, i0, p);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_f32(kBM, kBN);
+      uint32_t tile_ctr = tile_base, item_ctr = item_base;
+      bool ok = true;
+      for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
+        int p, m0, nt0, nt;
+        decode(item, p, m0, nt0, nt);
+        const int ab = item_ctr % g.a_bufs;
+        const uint32_t a_use = item_ctr / g.a_bufs;
+        if (!mbar_wait(&sh.a_full[ab], a_use & 1, abortp, g.status, ERR_WG_MMA)) break;
+        const uint32_t a_addr = smem_u32(a_base + (size_t)ab * a_bytes);
+        for (int j = 0; j < nt; ++j, ++tile_ctr) {
+          const int s = tile_ctr % g.slots;
+          const uint32_t use = tile_ctr / g.slots;
+          const int tb = tile_ctr & 1;
+          const uint32_t tuse = tile_ctr >> 1;
+          if (!mbar_wait(&sh.slot_full[s], use & 1, abortp, g.status, ERR_WG_MMA) ||
+              !mbar_wait(&sh.tmem_empty[tb], (tuse & 1) ^ 1, abortp, g.status, ERR_WG_MMA)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + kBOff);
+          for (int kb = 0; kb < g.nkb; ++kb) {
+            const uint64_t adesc = smem_desc_k_sw128(a_addr + kb * (kBM * kBK * 2));
+            const uint64_t bdesc = smem_desc_k_sw128(b_addr + kb * (kBN * kBK * 2));
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              umma_bf16(tmem_base + tb * kBN, adesc + 2 * k, bdesc + 2 * k, idesc,
+                        (uint32_t)((kb | k) != 0));
+          }
+          umma_commit(&sh.tmem_full[tb]);
+        }
+        if (ok) umma_commit(&sh.a_empty[ab]);     // all MMAs that read this dZ^T tile have finished
+      }
+    }
+    __syncwarp();
+  } else if (warp < 10) {
+    const int grp = (warp - 2) >> 2;           // epilogue group = TMEM buffer = tile parity
+    const int q = warp & 3;                    // TMEM lane quarter this warp may read
+    const int r = q * 32 + lane;               // weight row inside the tile
+    uint32_t tile_ctr = tile_base;
+    bool ok = true;
+    for (int item = vblock; item < g.items && ok; item += vgrid) {
+      int p, m0, nt0, nt;
+      decode(item, p, m0, nt0, nt);
+      for (int j = 0; j < nt; ++j, ++tile_ctr) {
+        if ((int)(tile_ctr & 1) != grp) continue;
+        const int s = tile_ctr % g.slots;
+        const uint32_t use = tile_ctr / g.slots;
+        const uint32_t tuse = tile_ctr >> 1;
+        // the master tile landed with the same barrier the MMA waited on; the accumulator next
+        if (!mbar_wait(&sh.slot_full[s], use & 1, abortp, g.status, ERR_WG_EPILOGUE) ||
+            !mbar_wait(&sh.tmem_full[grp], tuse & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        uint32_t acc[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(grp * kBN), acc);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.tmem_empty[grp]);    // this warp is done with the buffer
+
+        uint8_t* sl = slot_base + (size_t)s * slot_bytes;
+        uint8_t* w32 = sl + (size_t)r * 128;             // 8 chunks of 16 B, chunk c at c ^ (r & 7)
+        uint8_t* w16 = sl + kW32Bytes + (size_t)r * 64;  // 4 chunks, chunk c at c ^ ((r >> 1) & 3)
+        uint32_t hp[16];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float4* cell = reinterpret_cast<float4*>(w32 + ((c ^ (r & 7)) << 4));
+          float4 w = *cell;
+          if (MOM) {
+            // the u tile has the master tile's shape and swizzle
+            float4* ucell = reinterpret_cast<float4*>(w32 + kW32Bytes + kW16Bytes +
+                                                      ((c ^ (r & 7)) << 4));
+            float4 u = g.read_u ? *ucell : make_float4(0.f, 0.f, 0.f, 0.f);
+            msgd(w.x, u.x, __uint_as_float(acc[4 * c + 0]), g.gamma, g.beta);
+            msgd(w.y, u.y, __uint_as_float(acc[4 * c + 1]), g.gamma, g.beta);
+            msgd(w.z, u.z, __uint_as_float(acc[4 * c + 2]), g.gamma, g.beta);
+            msgd(w.w, u.w, __uint_as_float(acc[4 * c + 3]), g.gamma, g.beta);
+            *ucell = u;
+          } else {
+            w.x = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 0]), w.x);
+            w.y = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 1]), w.y);
+            w.z = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 2]), w.z);
+            w.w = fmaf(-g.gamma, __uint_as_float(acc[4 * c + 3]), w.w);
+          }
+          *cell = w;
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(w.x, w.y);
+          __nv_bfloat162 h1 = __floats2bfloat162_rn(w.z, w.w);
+          hp[2 * c] = *reinterpret_cast<uint32_t*>(&h0);
+          hp[2 * c + 1] = *reinterpret_cast<uint32_t*>(&h1);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          *reinterpret_cast<uint4*>(w16 + ((c ^ ((r >> 1) & 3)) << 4)) =
+              make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
+        fence_proxy_async();                   // generic-proxy writes -> visible to the TMA stores
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.out_full[s]);
+      }
+    }
+  } else {
+    if (lane == 0) {
+      uint32_t tile_ctr = tile_base;
+      bool ok = true;
+      // items whose tiles have all been handed to the TMA unit but may not have reached global
+      // memory yet: (index after the item's last tile, learner); signalled kStoreLag tiles later
+      uint32_t pend_end[8];
+      int pend_p[8];
+      uint32_t ph = 0, pt = 0;
+      for (int item = vblock; item < g.items && ok; item += vgrid) {
+        int p, m0, nt0, nt;
+        decode(item, p, m0, nt0, nt);
+        for (int j = 0; j < nt; ++j, ++tile_ctr) {
+          const int s = tile_ctr % g.slots;
+          const uint32_t use = tile_ctr / g.slots;
+          if (!mbar_wait(&sh.out_full[s], use & 1, abortp, g.status, ERR_WG_STORE)) {
+            ok = false;
+            break;
+          }
+          uint8_t* sl = slot_base + (size_t)s * slot_bytes;
+          const int i0 = (nt0 + j) * kBN;
+          tma_store_3d(&tm_w32, sl, i0, m0, p);
+          tma_store_3d(&tm_w16, sl + kW32Bytes, i0, m0, p);
+          if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes + kW16Bytes, i0, m0, p);
+          tma_store_commit();
+          // the slot of the previous tile is free once its stores have read shared memory
+          if (tile_ctr > tile_base) {
+            tma_store_wait_read<1>();
+            mbar_arrive(&sh.slot_empty[(tile_ctr - 1) % g.slots]);
+          }
+          if (Dep::kSignals) {
+            // all but the last kStoreLag store groups are in global memory
+            tma_store_wait_pending<kStoreLag>();
+            while (ph != pt && pend_end[ph & 7] + kStoreLag <= tile_ctr + 1) {
+              dep.item_done(pend_p[ph & 7]);
+              ++ph;
+            }
+          }
+        }
+        if (Dep::kSignals && ok) {
+          pend_end[pt & 7] = tile_ctr;
+          pend_p[pt & 7] = p;
+          ++pt;
+        }
+      }
+      tma_store_wait_read<0>();
+      if (tile_ctr > tile_base && ok) mbar_arrive(&sh.slot_empty[(tile_ctr - 1) % g.slots]);
+      if (Dep::kSignals && ok) {
+        tma_store_wait_all();
+        for (; ph != pt; ++ph) dep.item_done(pend_p[ph & 7]);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+}  // namespace wgrad
+}  // namespace mavg

@@ -340,8 +340,7 @@ def run_mavg(args):
                block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
                dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}",
                defer_broadcast=not args.no_defer, learner_momentum=args.beta)
-    if args.round_kernel:
-        g.set_round_kernel(True)
+    g.set_schedule(args.schedule)
     units = cfg["P"] * cfg["K"] * cfg["B"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
 
@@ -443,8 +442,9 @@ def run_mavg(args):
                        "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
                                 0: "CUDA cores fp32"}[mode],
                        "defer_broadcast": not args.no_defer, "learner_momentum": args.beta,
-                       "schedule": ("one persistent kernel per round" if args.round_kernel
-                                    else "CUDA graph of per-product launches"),
+                       "schedule": ["CUDA graph of per-product launches, fused last layer",
+                                    "one persistent kernel per round",
+                                    "CUDA graph of per-product launches, all on tensor cores"][args.schedule],
                        "l2": "flushed between steps by a 256 MiB memset outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
@@ -485,9 +485,10 @@ def main():
                     help="run only the meta-update sweep (profiler captures)")
     ap.add_argument("--beta", type=float, default=0.0,
                     help="learner-level momentum (0 = Algorithm 1 as printed, the benchmark setting)")
-    ap.add_argument("--round-kernel", action="store_true",
-                    help="run the K local steps of a round as one persistent kernel instead of the "
-                         "graph of per-product launches (same results; for comparison)")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
+                    help="0: CUDA graph with the fused last-layer kernel (default); 1: the K local "
+                         "steps of a round as one persistent kernel; 2: CUDA graph with every "
+                         "product on tensor cores (1 and 2 for comparison)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-defer", action="store_true",

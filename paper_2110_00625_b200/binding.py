@@ -10,6 +10,7 @@ import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 OBJ_NONE, OBJ_PSEUDOGRAD, OBJ_MLP = 0, 1, 2
+SCHED_GRAPH, SCHED_ROUND_KERNEL, SCHED_GRAPH_TC = 0, 1, 2
 X_F32, X_BF16 = 0, 1
 MAX_LAYERS = 8
 
@@ -20,7 +21,7 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams",
            "mavg_set_learner_momentum", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
-           "mavg_set_profiling", "mavg_set_round_kernel", "mavg_get_profile", "mavg_sync", "mavg_last_error",
+           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
@@ -89,7 +90,7 @@ def load_library():
     L.mavg_set_round.argtypes = [H, C.c_int64]
     L.mavg_get_launch_count.argtypes = [H, C.POINTER(C.c_int64)]
     L.mavg_set_profiling.argtypes = [H, C.c_int32]
-    L.mavg_set_round_kernel.argtypes = [H, C.c_int32]
+    L.mavg_set_schedule.argtypes = [H, C.c_int32]
     L.mavg_get_profile.argtypes = [H, C.c_void_p, C.c_void_p, C.c_int32]
     L.mavg_batch_indices_noalloc.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_int64, C.c_int32, C.c_void_p,
@@ -260,8 +261,10 @@ class Mavg:
     def set_profiling(self, on):
         self._check(self.lib.mavg_set_profiling(self.handle, int(bool(on))))
 
-    def set_round_kernel(self, on):
-        self._check(self.lib.mavg_set_round_kernel(self.handle, int(bool(on))))
+    def set_schedule(self, mode):
+        """0: CUDA graph with the fused last layer (default); 1: one persistent kernel per round;
+        2: CUDA graph with every product on tensor cores."""
+        self._check(self.lib.mavg_set_schedule(self.handle, int(mode)))
 
     def get_profile(self, reset=True):
         """{kernel class: (milliseconds, launches)} since the last reset."""

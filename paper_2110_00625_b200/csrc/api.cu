@@ -402,9 +402,10 @@ mavg_status mavg_set_profiling(mavg_handle h, int32_t on) {
   return MAVG_OK;
 }
 
-mavg_status mavg_set_round_kernel(mavg_handle h, int32_t on) {
+mavg_status mavg_set_schedule(mavg_handle h, int32_t mode) {
   CHECK_HANDLE(h);
-  h->round_kernel = on != 0;
+  if (mode < 0 || mode > 2) return set_err(h, MAVG_ERR_INVALID_ARG, "schedule must be 0, 1 or 2");
+  h->schedule = mode;
   return MAVG_OK;
 }
 

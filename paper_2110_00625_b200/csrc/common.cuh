@@ -106,7 +106,7 @@ struct mavg_ctx {
   int cls_open = 0;
   // CUDA graph of one round's K local steps (MLP objective): captured once on a private stream,
   // replayed on the caller's stream; rebuilt when K or the local learning rate change
-  bool round_kernel = false;  // MLP tensor-core path: run a round's K steps as one kernel where covered
+  int schedule = 0;           // MLP tensor-core path, see mavg_set_schedule
   bool capturing = false;
   bool graph_disabled = false;
   cudaGraphExec_t graph_exec = nullptr;
@@ -115,6 +115,7 @@ struct mavg_ctx {
   float graph_lr = 0.f;
   float graph_beta = 0.f;
   int graph_reset = 0;
+  int graph_schedule = 0;
   int64_t graph_nodes = 0;
 };
 

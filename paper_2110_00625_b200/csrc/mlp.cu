@@ -112,6 +112,7 @@ cudaError_t build_graph(mavg_ctx* c, int64_t round) {
   c->graph_lr = c->cfg.local_lr;
   c->graph_beta = c->cfg.learner_momentum;
   c->graph_reset = c->cfg.learner_momentum_reset;
+  c->graph_schedule = c->schedule;
   return cudaSuccess;
 }
 
@@ -128,7 +129,7 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
   // start elsewhere (local steps called twice in a row), profiled rounds and handles whose
   // capture failed once take the launch-by-launch path.
   // Where the whole-round kernel covers the problem, the K steps are one launch of it.
-  if (use_tensor_cores(&c->cfg) && !c->profiling && c->round_kernel && tc_round_supported(c)) {
+  if (use_tensor_cores(&c->cfg) && !c->profiling && c->schedule == 1 && tc_round_supported(c)) {
     cudaError_t e = tc_round_launch(c, round);
     if (e != cudaSuccess) return e;
     c->replicas_equal_global = false;
@@ -137,7 +138,8 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
   const bool want_graph = !c->profiling && !c->graph_disabled && c->replicas_equal_global;
   if (!want_graph) return run_steps(c, round);
   if (!c->graph_exec || c->graph_K != c->cfg.K || c->graph_lr != c->cfg.local_lr ||
-      c->graph_beta != c->cfg.learner_momentum || c->graph_reset != c->cfg.learner_momentum_reset) {
+      c->graph_beta != c->cfg.learner_momentum || c->graph_reset != c->cfg.learner_momentum_reset ||
+      c->graph_schedule != c->schedule) {
     cudaError_t e = build_graph(c, round);
     if (e != cudaSuccess) {
       cudaGetLastError();

@@ -39,6 +39,28 @@ void tc_teardown(mavg_ctx* c);
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c);
 cudaError_t tc_step(mavg_ctx* c, int64_t round, int step);
 
+// Fused last layer on CUDA cores (tail_fused.cu): forward, loss, dZ_L, dgrad through the layer
+// and the bias steps of the last two layers, for the tensor-core path's bf16 operands.
+struct TailLaunch {
+  const __nv_bfloat16* a_bm;     // A_{L-1} [P, B, in]
+  const __nv_bfloat16* w16;      // bf16 W_L of learner 0
+  int64_t w16_stride;            // elements between learners' copies (0: shared copy)
+  bool shared_w;                 // biases are read from w~ (first step of a round)
+  const int32_t* labels;
+  float* loss_out;
+  int loss_stride;
+  __nv_bfloat16* dz_t;           // out: dZ_L^T [P, C, B]
+  __nv_bfloat16* dzp_bm;         // out: dZ_{L-1} [P, B, in] and its transpose [P, in, B]
+  __nv_bfloat16* dzp_mb;
+  float* part;                   // scratch of tail_fused_part_bytes()
+  int* counters;                 // [P] ints, zero between launches
+  MomArgs mom;
+};
+bool tail_fused_supported(const mavg_config* cfg);
+size_t tail_fused_part_bytes(const mavg_config* cfg);
+cudaError_t tail_fused_prepare();
+cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t);
+
 // Whole-round kernel (round_tc.cu): all K local steps of a round in one launch.
 bool tc_round_supported(mavg_ctx* c);
 cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);

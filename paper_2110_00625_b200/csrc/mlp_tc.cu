@@ -174,6 +174,7 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.w16g = take((size_t)t.n16 * 2);
   t.round_ctr_bytes = (size_t)4 * (MAVG_MAX_LAYERS + 1) * P * sizeof(int);
   t.round_ctr = take(t.round_ctr_bytes);
+  t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
   t.end = off;
   return t;
 }
@@ -351,6 +352,8 @@ mavg_status tc_setup(mavg_ctx* c) {
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
   if (e == cudaSuccess) e = wgrad_stream_prepare();
   if (e == cudaSuccess) e = tc_round_prepare(c);
+  st->tail_ok = tail_fused_supported(&cfg);
+  if (e == cudaSuccess && st->tail_ok) e = tail_fused_prepare();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);
   cudaEvent_t* evs[] = {&st->ev_fork, &st->ev_wgrad_done, &st->ev_gather_done, &st->ev_x_free[0],
@@ -422,6 +425,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   int* counters = (int*)(ws + t.counters);
   const bool shared_w = c->replicas_equal_global;   // first step after a (re-)broadcast
   const MomArgs mom = mom_args(c, shared_w);
+  const bool fused_tail = st->tail_ok && c->schedule == 0;
   const bool overlap = !c->profiling;
   const int xb = step & 1;                          // batch buffer of this step
   cudaStream_t main_s = c->stream;
@@ -452,6 +456,20 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     if (l < L) {
       g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
       TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
+    } else if (fused_tail) {
+      // last layer forward, loss, dZ_L and dgrad_L in one CUDA-core kernel
+      TailLaunch tl{};
+      tl.a_bm = L >= 2 ? bfp(t.act[L - 1]) : bfp(t.xg[xb]);
+      tl.w16 = (shared_w ? bfp(t.w16g) : bfp(t.w16)) + t.sh_off[L - 1];
+      tl.w16_stride = shared_w ? 0 : t.n16;
+      tl.shared_w = shared_w;
+      tl.labels = labels_b; tl.loss_out = losses + (step - 1); tl.loss_stride = K;
+      tl.dz_t = bfp(t.dz_t[L]);
+      if (L >= 2) { tl.dzp_bm = bfp(t.dz[L - 1]); tl.dzp_mb = bfp(t.dz_t[L - 1]); }
+      tl.part = (float*)(ws + t.tail_part);
+      tl.counters = counters;
+      tl.mom = mom;
+      TC_TRY(launch_tail_fused(c, tl));
     } else {
       g.labels = labels_b; g.loss_out = losses + (step - 1); g.loss_stride = K;
       g.dz_bm = bfp(t.dz[L]); g.cpad = t.cpad; g.dz_mb = bfp(t.dz_t[L]);
@@ -474,7 +492,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   bool side_used = false;
   for (int l = L; l >= 1; --l) {
     const MlpLayer& ly = c->layers[l - 1];
-    if (l > 1) {
+    if (l > 1 && !(fused_tail && l == L)) {
       const MlpLayer& below = c->layers[l - 2];
       TcArgs g{};
       g.M = ly.in; g.N = B;

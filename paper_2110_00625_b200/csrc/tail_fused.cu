@@ -1,0 +1,257 @@
+// Last layer of the MLP learner step in one CUDA-core kernel: forward product, softmax
+// cross-entropy loss, dZ_L, the data gradient through the layer (with the ReLU mask of the layer
+// below) and the two bias steps that hang on them.  With at most 32 classes these products are a
+// few hundred thousand multiply-adds per learner -- far too small for a tensor-core tile each to
+// pay for its launch and its tail -- so one block takes 16 batch rows of one learner through the
+// whole sequence with the operands in shared memory:
+//   z[b, c]      = sum_k A[b, k] W[c, k] + bias[c]                  (bf16 operands, fp32 sums)
+//   loss_b       = logsumexp(z_b) - z_b[y_b];   dZ[b, c] = (softmax(z_b)[c] - [c == y_b]) / B
+//   dA[b, k]     = sum_c bf16(dZ[b, c]) W[c, k];   dZprev[b, k] = A[b, k] > 0 ? dA[b, k] : 0
+// and writes bf16(dZ) transposed (the weight-gradient kernel's operand), bf16(dZprev) in both
+// orientations, and per-block partial sums of the loss and of the two bias gradients (from the
+// unrounded dZ values).  The block of a learner that finishes last adds the partials in ascending
+// block order and takes the bias steps of Algorithm 1's local update, so the result does not
+// depend on the order in which blocks run.
+#include "mlp.cuh"
+
+namespace mavg {
+namespace {
+
+constexpr int kRows = 16;        // batch rows per block
+constexpr int kThreads = 256;
+constexpr int kMaxC = 32;
+
+struct TailArgs {
+  const __nv_bfloat16* a_bm;     // A_{L-1} [P, B, in]
+  const __nv_bfloat16* w16;      // W_L as bf16 [C, in]: w16 + p * w16_stride
+  int64_t w16_stride;            // 0: one copy shared by all learners
+  const float* bias_in;          // biases are read at bias_in[p * bias_in_stride + offset + i]
+  int64_t bias_in_stride;        //   (the masters, or w~ with stride 0 at a round's first step)
+  float* rep;                    // masters [P, rep_stride]: where the stepped biases are written
+  int64_t rep_stride;
+  int64_t b_off, bprev_off;      // offsets of b_L and b_{L-1} inside a replica
+  const int32_t* labels;         // [P*B]
+  float* loss_out;               // loss_out[p * loss_stride]
+  int loss_stride;
+  __nv_bfloat16* dz_t;           // dZ_L transposed [P, C, B]
+  __nv_bfloat16* dzp_bm;         // dZ_{L-1} [P, B, in]     (null for a one-layer model)
+  __nv_bfloat16* dzp_mb;         // dZ_{L-1} transposed [P, in, B]
+  float* part;                   // [P, blocks, in + C + 1] partial sums
+  int* counters;                 // [P], zero between launches
+  int B, in, C;
+  float gamma;
+  MomArgs mom;
+};
+
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+// grid (B / 16, P), 256 threads.  Dynamic shared memory: W [C, in] bf16, A [16, in] bf16.
+__global__ void __launch_bounds__(kThreads)
+k_last_layer_fused(const TailArgs g) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  __shared__ float z[kRows][kMaxC + 1];     // logits, then unrounded dZ
+  __shared__ float zq[kRows][kMaxC + 1];    // dZ rounded to bf16 values
+  __shared__ float row_loss[kRows];
+  __shared__ int is_last;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int p = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
+  const int r0 = blk * kRows;
+  const int in = g.in, C = g.C, B = g.B;
+  __nv_bfloat16* Ws = reinterpret_cast<__nv_bfloat16*>(smem_raw);
+  __nv_bfloat16* As = Ws + (size_t)C * in;
+
+  // operands into shared memory, 16 bytes per load (in is a multiple of 8)
+  {
+    const uint4* wsrc = reinterpret_cast<const uint4*>(g.w16 + (size_t)p * g.w16_stride);
+    uint4* wdst = reinterpret_cast<uint4*>(Ws);
+    for (int i = tid; i < C * in / 8; i += kThreads) wdst[i] = wsrc[i];
+    const uint4* asrc = reinterpret_cast<const uint4*>(g.a_bm + ((size_t)p * B + r0) * in);
+    uint4* adst = reinterpret_cast<uint4*>(As);
+    for (int i = tid; i < kRows * in / 8; i += kThreads) adst[i] = asrc[i];
+  }
+  __syncthreads();
+
+  // forward: warp w takes rows 2w and 2w + 1; lanes split the contraction, two elements at a time
+  const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride;
+  for (int rr = 0; rr < 2; ++rr) {
+    const int r = 2 * warp + rr;
+    const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)r * in);
+    for (int c = 0; c < C; ++c) {
+      const uint32_t* wrow = reinterpret_cast<const uint32_t*>(Ws + (size_t)c * in);
+      float acc = 0.f;
+      for (int k2 = lane; k2 < in / 2; k2 += 32) {
+        const uint32_t a = arow[k2], w = wrow[k2];
+        acc = fmaf(bf_lo(a), bf_lo(w), acc);
+        acc = fmaf(bf_hi(a), bf_hi(w), acc);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) z[r][c] = acc + bias_in[g.b_off + c];
+    }
+  }
+  __syncthreads();
+
+  // softmax cross-entropy, one thread per row
+  if (tid < kRows) {
+    const int r = tid;
+    const int yb = g.labels[(size_t)p * B + r0 + r];
+    float mx = z[r][0];
+    for (int c = 1; c < C; ++c) mx = fmaxf(mx, z[r][c]);
+    float se = 0.f;
+    for (int c = 0; c < C; ++c) se += __expf(z[r][c] - mx);
+    const float lse = mx + __logf(se);
+    row_loss[r] = lse - z[r][yb];
+    const float inv_b = 1.0f / (float)B;
+    for (int c = 0; c < C; ++c) {
+      const float gr = (__expf(z[r][c] - lse) - (c == yb ? 1.f : 0.f)) * inv_b;
+      z[r][c] = gr;
+      zq[r][c] = __bfloat162float(__float2bfloat16_rn(gr));
+    }
+  }
+  __syncthreads();
+
+  float* part = g.part + ((size_t)p * nblk + blk) * (in + C + 1);
+  // dZ_L transposed: class c, this block's 16 rows (32 contiguous bytes); partial bias gradient
+  if (tid < C) {
+    const int c = tid;
+    uint32_t w[8];
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(z[2 * j][c], z[2 * j + 1][c]);
+      w[j] = *reinterpret_cast<uint32_t*>(&h2);
+      s += z[2 * j][c];
+      s += z[2 * j + 1][c];
+    }
+    uint4* dst = reinterpret_cast<uint4*>(g.dz_t + ((size_t)p * C + c) * B + r0);
+    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    part[in + c] = s;
+  }
+  if (tid == kThreads - 1) {
+    float s = 0.f;
+    for (int r = 0; r < kRows; ++r) s += row_loss[r];
+    part[in + C] = s;
+  }
+
+  // data gradient through the layer, masked by the activation below; thread per input column
+  if (g.dzp_bm) {
+    for (int k = tid; k < in; k += kThreads) {
+      float acc[kRows];
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) acc[r] = 0.f;
+      for (int c = 0; c < C; ++c) {
+        const float wv = __bfloat162float(Ws[(size_t)c * in + k]);
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) acc[r] = fmaf(zq[r][c], wv, acc[r]);
+      }
+      float colsum = 0.f;
+      uint32_t w[8];
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) {
+        const bool live = __bfloat162float(As[(size_t)r * in + k]) > 0.f;     // ReLU'(0) = 0
+        acc[r] = live ? acc[r] : 0.f;
+        colsum += acc[r];
+        g.dzp_bm[((size_t)p * B + r0 + r) * in + k] = __float2bfloat16_rn(acc[r]);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t*>(&h2);
+      }
+      uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + k) * B + r0);
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      part[k] = colsum;
+    }
+  }
+
+  // the learner's last block adds the partials (ascending block order) and steps the biases
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(g.counters + p, 1);
+    const int last = old == nblk - 1;
+    if (last) g.counters[p] = 0;
+    __threadfence();
+    is_last = last;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  const float* pp = g.part + (size_t)p * nblk * (in + C + 1);
+  float* rep = g.rep + (size_t)p * g.rep_stride;
+  float* urow = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride : nullptr;
+  const int n_sum = (g.dzp_bm ? in : 0);
+  for (int i = tid; i < in + C + 1; i += kThreads) {
+    if (i < in && i >= n_sum) continue;
+    float s = 0.f;
+    for (int b = 0; b < nblk; ++b) s += __ldcg(pp + (size_t)b * (in + C + 1) + i);
+    if (i < in) {
+      const int64_t o = g.bprev_off + i;
+      local_update(rep + o, bias_in[o], urow ? urow + o : nullptr, g.mom.read_u, s, g.gamma, g.mom.beta);
+    } else if (i < in + C) {
+      const int64_t o = g.b_off + (i - in);
+      local_update(rep + o, bias_in[o], urow ? urow + o : nullptr, g.mom.read_u, s, g.gamma, g.mom.beta);
+    } else {
+      g.loss_out[(size_t)p * g.loss_stride] = s / (float)B;
+    }
+  }
+}
+
+size_t tail_smem_bytes(int in, int C) { return ((size_t)C * in + (size_t)kRows * in) * 2; }
+
+}  // namespace
+
+bool tail_fused_supported(const mavg_config* cfg) {
+  const int L = cfg->n_layers;
+  const int in = cfg->dims[L - 1], C = cfg->dims[L];
+  if (cfg->B % kRows != 0 || in % 8 != 0 || C > kMaxC) return false;
+  return tail_smem_bytes(in, C) <= 160 * 1024;
+}
+
+size_t tail_fused_part_bytes(const mavg_config* cfg) {
+  const int L = cfg->n_layers;
+  return (size_t)cfg->P * (cfg->B / kRows) * (cfg->dims[L - 1] + cfg->dims[L] + 1) * sizeof(float);
+}
+
+cudaError_t tail_fused_prepare() {
+  return cudaFuncSetAttribute(k_last_layer_fused, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              160 * 1024);
+}
+
+cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t) {
+  const mavg_config& cfg = c->cfg;
+  const int L = cfg.n_layers;
+  const MlpLayer& ly = c->layers[L - 1];
+  TailArgs g{};
+  g.a_bm = t.a_bm;
+  g.w16 = t.w16;
+  g.w16_stride = t.w16_stride;
+  g.bias_in = t.shared_w ? c->buf.global_w : c->buf.replicas;
+  g.bias_in_stride = t.shared_w ? 0 : c->buf.replica_stride;
+  g.rep = c->buf.replicas;
+  g.rep_stride = c->buf.replica_stride;
+  g.b_off = ly.b_off;
+  g.bprev_off = L >= 2 ? c->layers[L - 2].b_off : 0;
+  g.labels = t.labels;
+  g.loss_out = t.loss_out;
+  g.loss_stride = t.loss_stride;
+  g.dz_t = t.dz_t;
+  g.dzp_bm = L >= 2 ? t.dzp_bm : nullptr;
+  g.dzp_mb = L >= 2 ? t.dzp_mb : nullptr;
+  g.part = t.part;
+  g.counters = t.counters;
+  g.B = cfg.B;
+  g.in = ly.in;
+  g.C = ly.out;
+  g.gamma = cfg.local_lr;
+  g.mom = t.mom;
+  dim3 grid((unsigned)(cfg.B / kRows), (unsigned)cfg.P);
+  prof_begin(c, MAVG_K_FWD);
+  k_last_layer_fused<<<grid, kThreads, tail_smem_bytes(ly.in, ly.out), c->stream>>>(g);
+  prof_end(c);
+  return cudaGetLastError();
+}
+
+}  // namespace mavg

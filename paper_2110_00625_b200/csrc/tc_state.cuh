@@ -20,6 +20,7 @@ struct TcLayout {
   size_t counters, counters_bytes;
   size_t w16, w16g;
   size_t round_ctr, round_ctr_bytes;         // completion counters of the whole-round kernel
+  size_t tail_part;                          // partial sums of the fused last-layer kernel
   size_t end;
 };
 
@@ -46,6 +47,7 @@ struct TcState {
   CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
   CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
   bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
+  bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   // whole-round kernel (round_tc.cu)
   bool round_ok = false;
   int round_stages = 0, round_grid = 0;

@@ -24,7 +24,7 @@ def _make(cfg, round_kernel, defer=False):
     g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
                seed=SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1, x=x, y=y,
                x_bf16=cfg.get("x_bf16", False), defer_broadcast=defer)
-    g.set_round_kernel(round_kernel)
+    g.set_schedule(1 if round_kernel else 2)
     return g, x, y, w1
 
 

@@ -352,7 +352,11 @@ mavg_status tc_setup(mavg_ctx* c) {
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
   if (e == cudaSuccess) e = wgrad_stream_prepare();
   if (e == cudaSuccess) e = tc_round_prepare(c);
-  st->tail_ok = tail_fused_supported(&cfg);
+  // The fused CUDA-core last layer pays where the tensor-core products of that layer would leave
+  // most of the GPU idle (few learners, narrow layer below); with many tiles the tensor-core
+  // kernels are the faster ones.
+  st->tail_ok = tail_fused_supported(&cfg) &&
+                P * ((cfg.dims[L - 1] + kBM - 1) / kBM) <= c->sm_count / 2;
   if (e == cudaSuccess && st->tail_ok) e = tail_fused_prepare();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_wgrad, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&st->s_gather, cudaStreamNonBlocking);

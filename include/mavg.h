@@ -194,7 +194,7 @@ typedef enum {
   MAVG_K_PSEUDOGRAD = 2,
   MAVG_K_BATCH = 3,     /* index stream and gather */
   MAVG_K_FWD = 4,       /* forward GEMMs (+bias, ReLU) */
-  MAVG_K_LOSS = 5,      /* softmax cross-entropy, loss reductions */
+  MAVG_K_LOSS = 5,      /* softmax cross-entropy and loss reductions; the fused last-layer kernel */
   MAVG_K_DGRAD = 6,     /* backward-data GEMMs (+ReLU mask, bias step) */
   MAVG_K_WGRAD_SGD = 7, /* backward-weight GEMMs fused with the SGD step */
   MAVG_K_AUX = 8,       /* operand copies (bf16 shadows) */

@@ -355,6 +355,14 @@ mavg_status tc_setup(mavg_ctx* c) {
   // The fused CUDA-core last layer pays where the tensor-core products of that layer would leave
   // most of the GPU idle (few learners, narrow layer below); with many tiles the tensor-core
   // kernels are the faster ones.
+  // Small problems (a few dozen weight tiles per SM in the largest layer): one persistent launch
+  // takes the weight gradients of all layers, instead of one launch per layer on a side stream.
+  {
+    const WgradPlan& w1 = st->wgrad[1];
+    st->wgrad_merged = L >= 2 && (long)P * w1.m_tiles * w1.n_tiles <= 64L * c->sm_count;
+    for (int l = 2; l <= L; ++l)
+      if (st->wgrad[l].slots != w1.slots || st->wgrad[l].a_bufs != w1.a_bufs) st->wgrad_merged = false;
+  }
   st->tail_ok = tail_fused_supported(&cfg) &&
                 P * ((cfg.dims[L - 1] + kBM - 1) / kBM) <= c->sm_count / 2;
   if (e == cudaSuccess && st->tail_ok) e = tail_fused_prepare();
@@ -494,6 +502,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   }
 
   bool side_used = false;
+  const bool merged = st->wgrad_merged && c->schedule == 0;
   for (int l = L; l >= 1; --l) {
     const MlpLayer& ly = c->layers[l - 1];
     if (l > 1 && !(fused_tail && l == L)) {
@@ -513,6 +522,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
                                     st->dz[l], st->dgrad[l], g));
     }
     const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
+    if (merged) continue;        // all layers' weight gradients follow in one launch
     if (overlap && l > 1) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
@@ -525,6 +535,21 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
     }
+  }
+  if (merged) {
+    // largest layer first, so that the small ones fill the ragged end of the launch
+    WgradLayerRef refs[MAVG_MAX_LAYERS];
+    for (int l = 1; l <= L; ++l) {
+      WgradLayerRef& r = refs[l - 1];
+      r.plan = &st->wgrad[l];
+      r.dzt = &st->dz_t[l];
+      r.at = l == 1 ? &st->x_in_t[xb] : &st->act_in_t[l];
+      r.w32 = &st->w32[l];
+      r.w16 = &st->w16_st[l];
+      r.w32_shared = shared_w ? &st->w32g[l] : nullptr;
+      r.u32 = st->wgrad_mom ? &st->u32[l] : nullptr;
+    }
+    TC_TRY(launch_wgrad_multi(c, L, refs, mom));
   }
   if (overlap) {
     TC_TRY(cudaEventRecord(st->ev_x_free[xb], main_s));     // wgrad_1 was the buffer's last reader

@@ -53,6 +53,8 @@ k_last_layer_fused(const TailArgs g) {
   __shared__ float z[kRows][kMaxC + 1];     // logits, then unrounded dZ
   __shared__ float zq[kRows][kMaxC + 1];    // dZ rounded to bf16 values
   __shared__ float row_loss[kRows];
+  __shared__ float bias_s[kMaxC];
+  __shared__ int label_s[kRows];
   __shared__ int is_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
@@ -61,7 +63,11 @@ k_last_layer_fused(const TailArgs g) {
   __nv_bfloat16* Ws = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   __nv_bfloat16* As = Ws + (size_t)C * in;
 
-  // operands into shared memory, 16 bytes per load (in is a multiple of 8)
+  // operands into shared memory, 16 bytes per load (in is a multiple of 8); the layer's bias and
+  // the rows' labels too, so that no later phase waits for a global load of its own
+  const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride;
+  if (tid < C) bias_s[tid] = bias_in[g.b_off + tid];
+  if (tid >= 32 && tid < 32 + kRows) label_s[tid - 32] = g.labels[(size_t)p * B + r0 + tid - 32];
   {
     const uint4* wsrc = reinterpret_cast<const uint4*>(g.w16 + (size_t)p * g.w16_stride);
     uint4* wdst = reinterpret_cast<uint4*>(Ws);
@@ -73,7 +79,6 @@ k_last_layer_fused(const TailArgs g) {
   __syncthreads();
 
   // forward: warp w takes rows 2w and 2w + 1; lanes split the contraction, two elements at a time
-  const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride;
   for (int rr = 0; rr < 2; ++rr) {
     const int r = 2 * warp + rr;
     const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)r * in);
@@ -87,7 +92,7 @@ k_last_layer_fused(const TailArgs g) {
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) z[r][c] = acc + bias_in[g.b_off + c];
+      if (lane == 0) z[r][c] = acc + bias_s[c];
     }
   }
   __syncthreads();
@@ -95,7 +100,7 @@ k_last_layer_fused(const TailArgs g) {
   // softmax cross-entropy, one thread per row
   if (tid < kRows) {
     const int r = tid;
-    const int yb = g.labels[(size_t)p * B + r0 + r];
+    const int yb = label_s[r];
     float mx = z[r][0];
     for (int c = 1; c < C; ++c) mx = fmaxf(mx, z[r][c]);
     float se = 0.f;
@@ -248,7 +253,7 @@ cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t) {
   g.gamma = cfg.local_lr;
   g.mom = t.mom;
   dim3 grid((unsigned)(cfg.B / kRows), (unsigned)cfg.P);
-  prof_begin(c, MAVG_K_FWD);
+  prof_begin(c, MAVG_K_LOSS);
   k_last_layer_fused<<<grid, kThreads, tail_smem_bytes(ly.in, ly.out), c->stream>>>(g);
   prof_end(c);
   return cudaGetLastError();

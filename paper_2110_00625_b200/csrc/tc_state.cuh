@@ -48,6 +48,7 @@ struct TcState {
   CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
   bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
+  bool wgrad_merged = false;                  // all layers' weight gradients in one launch
   // whole-round kernel (round_tc.cu)
   bool round_ok = false;
   int round_stages = 0, round_grid = 0;

@@ -77,6 +77,55 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   if (warp == 1) tmem_dealloc(tmem_base, 64);
 }
 
+// The same for several layers in one launch: every block makes one run per layer, in the order
+// given, with the ring and its barriers carried from run to run (all layers share the batch, so
+// their rings have the same geometry).  For workloads whose single layers are too small to pay
+// for a persistent launch each.
+struct WgradMultiParams {
+  CUtensorMap dzt[MAVG_MAX_LAYERS], at[MAVG_MAX_LAYERS], w32[MAVG_MAX_LAYERS],
+      w32_in[MAVG_MAX_LAYERS], w16[MAVG_MAX_LAYERS], u[MAVG_MAX_LAYERS];
+  WgradArgs g[MAVG_MAX_LAYERS];
+  int rot[MAVG_MAX_LAYERS];    // block b takes the items (b + rot) % grid, + grid, ... of a layer
+  int n;
+};
+
+template <bool MOM>
+__global__ void __launch_bounds__(kThreads)
+k_wgrad_sgd_multi(const __grid_constant__ WgradMultiParams mp) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) WgradShared sh;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5;
+  grid_launch_dependents();
+  if (threadIdx.x == 0) {
+    wgrad_init_barriers(sh, mp.g[0].slots);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sh.tmem_slot, 64);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = sh.tmem_slot;
+  grid_dependency_wait();
+  uint32_t tiles = 0, items = 0;
+  const int grid = (int)gridDim.x;
+  for (int s = 0; s < mp.n; ++s) {
+    const int vb = ((int)blockIdx.x + mp.rot[s]) % grid;
+    wgrad_run<MOM>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.g[s], vb,
+                   grid, smem, sh, tmem_base, NoDeps(), tiles, items);
+    wgrad_run_totals(mp.g[s], vb, grid, tiles, items);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 64);
+}
+
 }  // namespace
 
 WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum) {
@@ -111,8 +160,70 @@ cudaError_t wgrad_stream_prepare() {
   cudaError_t e = cudaFuncSetAttribute(k_wgrad_sgd_stream<false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_wgrad_sgd_stream<true>,
+  e = cudaFuncSetAttribute(k_wgrad_sgd_stream<true>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_wgrad_sgd_multi<false>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_wgrad_sgd_multi<true>,
                               cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+}
+
+namespace {
+WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs& mom) {
+  WgradArgs g{};
+  g.w32_in_batched = shared ? 0 : 1;
+  g.nkb = w.nkb;
+  g.m_tiles = w.m_tiles;
+  g.n_tiles = w.n_tiles;
+  g.chunk = w.chunk;
+  g.n_chunks = w.n_chunks;
+  g.items = w.items;
+  g.slots = w.slots;
+  g.a_bufs = w.a_bufs;
+  g.gamma = c->cfg.local_lr;
+  g.beta = mom.beta;
+  g.read_u = mom.read_u;
+  g.status = (int*)ws_ptr(c, c->ws.status);
+  return g;
+}
+}  // namespace
+
+cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers, const MomArgs& mom) {
+  WgradMultiParams* mp = new WgradMultiParams();
+  mp->n = n;
+  int grid = 1, rot = 0;
+  size_t smem = 0;
+  for (int s = 0; s < n; ++s) grid = layers[s].plan->grid > grid ? layers[s].plan->grid : grid;
+  const bool with_u = mom.u != nullptr;
+  for (int s = 0; s < n; ++s) {
+    const WgradLayerRef& r = layers[s];
+    mp->dzt[s] = *r.dzt; mp->at[s] = *r.at; mp->w32[s] = *r.w32;
+    mp->w32_in[s] = r.w32_shared ? *r.w32_shared : *r.w32;
+    mp->w16[s] = *r.w16;
+    mp->u[s] = (with_u && r.u32) ? *r.u32 : *r.w32;
+    mp->g[s] = make_args(c, *r.plan, r.w32_shared != nullptr, mom);
+    mp->rot[s] = (grid - rot % grid) % grid;   // this layer's item 0 goes to block `rot`
+    rot = (rot + r.plan->items) % grid;
+    smem = r.plan->smem > smem ? r.plan->smem : smem;
+  }
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)grid);
+  lc.blockDim = dim3(kThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = c->stream;
+  cudaLaunchAttribute at_[1];
+  at_[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at_[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at_;
+  lc.numAttrs = 1;
+  prof_begin(c, MAVG_K_WGRAD_SGD);
+  cudaError_t e = with_u ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_multi<true>, *mp)
+                         : cudaLaunchKernelEx(&lc, k_wgrad_sgd_multi<false>, *mp);
+  prof_end(c);
+  delete mp;
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,

@@ -27,4 +27,16 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
                                 const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr,
                                 const CUtensorMap* u32 = nullptr, const MomArgs& mom = MomArgs());
 
+// Several layers' weight-gradient + SGD tiles in one persistent launch (layers listed in the
+// order their tiles should run).  All plans must come from the same batch size and momentum
+// setting, which fixes the ring geometry.
+struct WgradLayerRef {
+  const WgradPlan* plan;
+  const CUtensorMap *dzt, *at, *w32, *w16;
+  const CUtensorMap* w32_shared;   // null: every learner loads its own masters
+  const CUtensorMap* u32;          // learner momentum view (may be null without momentum)
+};
+cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers,
+                               const MomArgs& mom = MomArgs());
+
 }  // namespace mavg

@@ -246,7 +246,66 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
         const float my_bias = EPI != EPI_DGRAD ? bias_pre : 0.f;
         float dsum = 0.f;
         float* lg = reinterpret_cast<float*>(smem);          // last layer: logits [N][M]
-        for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+        // Hidden-layer forward and dgrad tails of an unsplit tile: eight columns at a time in a
+        // loop that is NOT unrolled.  A tile's tail runs once per block, so its cost is largely
+        // the fetch of its instructions; a short body that is reused beats a long one that is not.
+        // Same values in the same order as the general path below.  The batch and the tile width
+        // are multiples of 16, so a group of eight columns is inside the batch or outside it.
+        const bool compact = EPI != EPI_FWD_LAST && (!ALLOW_SPLIT || g.splits == 1);
+        if (compact) {
+          const __nv_bfloat16* mrow = EPI == EPI_DGRAD
+              ? g.mask_mb + ((size_t)p * g.M + m0 + row) * g.N + n0 : nullptr;
+          uint4 mk8 = mk[0];                                  // first group, fetched before the wait
+#pragma unroll 1
+          for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+#pragma unroll 1
+            for (int s8 = 0; s8 < 32; s8 += 8) {
+              const int cc = c0 + s8;
+              if (cc >= g.BN) break;
+              uint32_t r8[8];
+              tmem_ld_8cols(lane_addr + (uint32_t)cc, r8);
+              // mask of the next group of this warp, in flight while this one is finished
+              uint4 mk8n = make_uint4(0, 0, 0, 0);
+              if (EPI == EPI_DGRAD) {
+                const int cn = s8 < 24 ? cc + 8 : c0 + 64;
+                if (m_ok && cn < g.BN && n0 + cn < g.N)
+                  mk8n = *reinterpret_cast<const uint4*>(mrow + cn);
+              }
+              tmem_ld_wait();
+              const bool valid = n0 + cc < g.N;
+              float z8[8];
+              const __nv_bfloat16* mh = reinterpret_cast<const __nv_bfloat16*>(&mk8);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float v = __uint_as_float(r8[j]);
+                if (EPI == EPI_DGRAD) {
+                  v = (valid && __bfloat162float(mh[j]) > 0.f) ? v : 0.f;   // ReLU'(0) = 0
+                  dsum += v;
+                } else {
+                  v += my_bias;
+                  v = v > 0.f ? v : 0.f;
+                }
+                z8[j] = v;
+              }
+              uint32_t h4[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(z8[2 * j], z8[2 * j + 1]);
+                h4[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              if (m_ok && valid) {
+                const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(h4);
+                *reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + cc) =
+                    make_uint4(h4[0], h4[1], h4[2], h4[3]);
+                __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + cc) * g.M + m;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dbm[(size_t)j * g.M] = hh[j];
+              }
+              mk8 = mk8n;
+            }
+          }
+        }
+        for (int c0 = compact ? g.BN : half * 32; c0 < g.BN; c0 += 64) {
           float z[32];
           int ncols;
           if (!ALLOW_SPLIT || g.splits == 1) {

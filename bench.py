@@ -165,9 +165,9 @@ def run_reference(args):
 # stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
 # captured; set an entry to None when its kernel changes.
 NCU_TRAFFIC_C2 = {
-    "wgrad_sgd_gemm": (57.709312e6 + 20.414720e6 + 10.521344e6 + 0.011776e6 + 1.326336e6) / 3,
-    "fwd_gemm": (31.539200e6 + 5.325568e6 + 1.273856e6) / 3,
-    "dgrad_gemm": (1.313280e6 + 6.380800e6) / 2,
+    "wgrad_sgd_gemm": 69.459968e6 + 33.750016e6,                 # one launch for all layers
+    "fwd_gemm": (31.539968e6 + 0.002048e6 + 5.325824e6) / 2,     # hidden layers 1 and 2
+    "dgrad_gemm": 6.381568e6,
 }
 
 
@@ -456,7 +456,8 @@ def run_mavg(args):
             "cpu_baseline": cpu,
             "wall_s_timed_region": t_wall,
             "meta_update_in_round": {"ms": statistics.median(meta_ms),
-                                     "gbs": (8 * cfg["P"] + 16) * n / statistics.median(meta_ms) / 1e6},
+                                     "gbs": ((8 if args.no_defer else 4) * cfg["P"] + 16) * n
+                                            / statistics.median(meta_ms) / 1e6},
             "kernels": kern,
             "meta_update_sweep": sweep,
             "tflops_round": flop_per_sample(cfg["dims"]) * units * args.steps / (total_ms * 1e-3) / 1e12,

@@ -81,6 +81,7 @@ struct GemmShared {
   uint64_t full_bar[kMaxStages];
   uint64_t empty_bar[kMaxStages];
   uint64_t acc_bar;
+  uint64_t recv_bar;          // cluster split: arrivals of the other blocks' partial tiles
   uint32_t tmem_slot;
   int abort_flag;
   int last_flag;
@@ -104,7 +105,15 @@ __device__ __forceinline__ void gemm_init_barriers(GemmShared& sh, int stages) {
 // accumulator columns are reused.  A block that runs several tiles keeps using the same
 // barriers: it0 is the number of pipeline slabs its earlier tiles went through (with the same
 // g.stages) and acc_phase the number of earlier tiles, which fix the barrier phases to wait for.
-template <int EPI, bool ALLOW_SPLIT>
+//
+// CLUSTER (hidden-layer forward only): the g.splits blocks that share an output tile form a
+// thread-block cluster (rank = split index).  Each accumulates the whole 128 x BN tile over its
+// part of the contraction, BN = 32 * g.splits; block r finishes the columns [32 r, 32 r + 32): the
+// others write their partial sums of those columns into its shared memory (`recv`, behind the
+// pipeline buffer: [splits][128 rows][32] fp32, slot = sender's rank) and arrive on its recv_bar,
+// and it adds the partials in ascending rank order.  An SM then takes in 1/splits of the weight
+// tile's bytes instead of all of them for a quarter of the batch.
+template <int EPI, bool ALLOW_SPLIT, bool CLUSTER = false>
 __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensorMap& tmB,
                                           const TcArgs& g, int bx, int p, uint8_t* smem,
                                           GemmShared& sh, uint32_t tmem_base, uint32_t it0 = 0,
@@ -215,7 +224,78 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
       const int m = m0 + row;
       const bool m_ok = m < g.M;
       bool finisher = ok;
-      if (ALLOW_SPLIT && g.splits > 1) {   // the register-capped build is never used with a split
+      if (CLUSTER) {
+        finisher = false;
+        const uint32_t rank = (uint32_t)split;
+        float* recv = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes);
+        if (ok) {
+          // this warp's chunks that belong to other blocks: into their shared memory
+          for (int c0 = half * 32; c0 < g.BN; c0 += 64) {
+            const uint32_t dest = (uint32_t)(c0 >> 5);
+            if (dest == rank) continue;
+            float z[32];
+            load_acc_chunk(lane_addr, c0, g.BN, z);
+            const uint32_t dst = mapa_u32(smem_u32(recv + ((size_t)rank * kBM + row) * 32), dest);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              st_cluster_f4(dst + 16 * v, z[4 * v], z[4 * v + 1], z[4 * v + 2], z[4 * v + 3]);
+            mbar_arrive_cluster(mapa_u32(smem_u32(&sh.recv_bar), dest));
+          }
+        }
+        // the four warps that hold this block's own columns finish them
+        if (ok && half == (int)(rank & 1u)) {
+          bool got = mbar_try_wait_cluster(&sh.recv_bar, 0);
+          if (!got) {
+            const uint64_t t0 = global_timer_ns();
+            while (!(got = mbar_try_wait_cluster(&sh.recv_bar, 0))) {
+              if (*abortp) break;
+              if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abortp = 1;
+                atomicCAS(g.status, 0, (int)ERR_EPILOGUE);
+                break;
+              }
+            }
+          }
+          if (got) {
+            const int c0 = (int)rank * 32;
+            float own[32], z[32];
+            load_acc_chunk(lane_addr, c0, g.BN, own);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = 0.f;
+            for (int sp = 0; sp < g.splits; ++sp) {            // ascending rank order
+              if (sp == (int)rank) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) z[j] += own[j];
+              } else {
+                const float4* src = reinterpret_cast<const float4*>(recv + ((size_t)sp * kBM + row) * 32);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                  const float4 t = src[v];
+                  z[4 * v] += t.x; z[4 * v + 1] += t.y; z[4 * v + 2] += t.z; z[4 * v + 3] += t.w;
+                }
+              }
+            }
+            uint32_t hp[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float a0 = z[2 * j] + bias_pre, a1 = z[2 * j + 1] + bias_pre;
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
+              hp[j] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            if (m_ok) {
+              const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
+              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + c0) * g.M + m;
+              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + c0);
+#pragma unroll
+              for (int v = 0; v < 4; ++v)
+                dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) dbm[(size_t)j * g.M] = hh[j];
+            }
+          }
+        }
+      }
+      if (!CLUSTER && ALLOW_SPLIT && g.splits > 1) {   // the register-capped build is never used with a split
         if (ok) {
           float* dst = g.part + ((size_t)(split * g.P + p) * g.N) * g.M + m;
           for (int c0 = half * 32; c0 < g.BN; c0 += 64) {

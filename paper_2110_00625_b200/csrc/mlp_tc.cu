@@ -78,6 +78,45 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   if (warp == 1) tmem_dealloc(tmem_base, g.tmem_cols);
 }
 
+// Hidden-layer forward tile with its contraction split over the blocks of a cluster (see
+// gemm_tile, CLUSTER): grid.x = row tiles x splits, cluster = the `splits` blocks of a row tile.
+__global__ void __launch_bounds__(kThreads, 1)
+k_tc_gemm_ks(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+             const TcArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) GemmShared sh;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5;
+  grid_launch_dependents();
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    gemm_init_barriers(sh, g.stages);
+    // every lane of the four sending warps of each other block arrives once
+    mbar_init(&sh.recv_bar, (uint32_t)(g.splits - 1) * 128u);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sh.tmem_slot, g.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  cluster_sync_all();           // every block's barriers exist before anyone arrives on them
+  const uint32_t tmem_base = sh.tmem_slot;
+  grid_dependency_wait();
+  gemm_tile<EPI_FWD_HIDDEN, false, true>(tmA, tmB, g, (int)blockIdx.x, (int)blockIdx.y, smem, sh,
+                                         tmem_base);
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();           // nobody leaves while a peer may still write into its shared memory
+  if (warp == 1) tmem_dealloc(tmem_base, g.tmem_cols);
+}
+
 // bf16 copy of the global model w~ (shared by all learners at the first step of a round, when
 // every replica equals w~).  One launch per layer; grid-stride over the layer's weights.
 __global__ void __launch_bounds__(256)
@@ -244,6 +283,69 @@ cudaError_t launch_gemm(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtens
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+// Plan of the cluster-split forward product of a hidden layer, or splits = 1 if it does not apply:
+// the default plan would cut the batch into B / 32 column tiles (so every block would stream the
+// whole weight tile for a quarter or half of the batch), and the contraction is long enough.
+GemmPlan plan_cluster_split(const GemmPlan& f, int M, int B, int K) {
+  GemmPlan ks{};
+  ks.splits = 1;
+  const int S = B / 32;
+  if ((B != 64 && B != 128) || f.splits != 1 || f.n_tiles != S || f.BN != 32) return ks;
+  const int nkb = (K + kBK - 1) / kBK;
+  const int per = (nkb + S - 1) / S;
+  if (nkb < 4 * S || per * (S - 1) >= nkb) return ks;
+  ks.BN = B;
+  ks.m_tiles = (M + kBM - 1) / kBM;
+  ks.n_tiles = 1;
+  ks.nkb = nkb;
+  ks.splits = S;
+  ks.kb_per_split = per;
+  const int stage_bytes = kATileBytes + B * kBK * 2;
+  ks.stages = (216 * 1024 - S * kBM * 32 * 4) / stage_bytes;
+  if (ks.stages > kMaxStages) ks.stages = kMaxStages;
+  if (ks.stages > per) ks.stages = per;
+  if (ks.stages < 2) { ks.splits = 1; return ks; }
+  ks.tmem_cols = 32;
+  while ((int)ks.tmem_cols < B) ks.tmem_cols <<= 1;
+  return ks;
+}
+
+cudaError_t launch_gemm_ks(mavg_ctx* c, const CUtensorMap& a, const CUtensorMap& b,
+                           const GemmPlan& pl, TcArgs g) {
+  g.BN = pl.BN;
+  g.m_tiles = pl.m_tiles;
+  g.n_tiles = 1;
+  g.splits = pl.splits;
+  g.kb_per_split = pl.kb_per_split;
+  g.nkb = pl.nkb;
+  g.stages = pl.stages;
+  g.tmem_cols = pl.tmem_cols;
+  g.P = c->cfg.P;
+  g.rep_stride = c->buf.replica_stride;
+  g.gamma = c->cfg.local_lr;
+  g.status = (int*)ws_ptr(c, c->ws.status);
+  const size_t smem = (size_t)pl.stages * (kATileBytes + pl.BN * kBK * 2) +
+                      (size_t)pl.splits * kBM * 32 * 4 + 1024;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)(pl.m_tiles * pl.splits), (unsigned)c->cfg.P);
+  lc.blockDim = dim3(kThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = (unsigned)pl.splits;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 2;
+  prof_begin(c, MAVG_K_FWD);
+  cudaError_t e = cudaLaunchKernelEx(&lc, k_tc_gemm_ks, a, b, g);
+  prof_end(c);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 }  // namespace
 
 bool tc_shapes_ok(const mavg_config* cfg, std::string* why) {
@@ -292,6 +394,9 @@ mavg_status tc_setup(mavg_ctx* c) {
     const int in = cfg.dims[l - 1], out = cfg.dims[l];
     const int dz_ld = l < L ? out : t.cpad;
     st->fwd[l] = plan_partial(out, B, in, P, kPlanSmCount, l < L);
+    st->fwd_ks[l] = GemmPlan{};
+    st->fwd_ks[l].splits = 1;
+    if (l < L) st->fwd_ks[l] = plan_cluster_split(st->fwd[l], out, B, in);
     st->wgrad_mom = c->buf.learner_u != nullptr;
     st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count, st->wgrad_mom);
     if (st->wgrad_mom)
@@ -311,12 +416,18 @@ mavg_status tc_setup(mavg_ctx* c) {
                               st->fwd[l].BN, &why);
         ok = ok && encode_map(st, &st->x_in_t[i], bf(t.xt[i]), B, in, P, B, (int64_t)B * in,
                               kWgradTileCols, &why);
+        if (st->fwd_ks[l].splits > 1)
+          ok = ok && encode_map(st, &st->x_in_ks[i], bf(t.xg[i]), in, B, P, in, (int64_t)B * in,
+                                B, &why);
       }
     } else {
       ok = ok && encode_map(st, &st->act_in[l], bf(t.act[l - 1]), in, B, P, in, (int64_t)B * in,
                             st->fwd[l].BN, &why);
       ok = ok && encode_map(st, &st->act_in_t[l], bf(t.act_t[l - 1]), B, in, P, B,
                             (int64_t)B * in, kWgradTileCols, &why);
+      if (st->fwd_ks[l].splits > 1)
+        ok = ok && encode_map(st, &st->act_in_ks[l], bf(t.act[l - 1]), in, B, P, in,
+                              (int64_t)B * in, B, &why);
     }
     ok = ok && encode_map(st, &st->dz_t[l], bf(t.dz_t[l]), B, out, P, B, (int64_t)B * out, kBM,
                           &why);
@@ -346,7 +457,8 @@ mavg_status tc_setup(mavg_ctx* c) {
   e = cudaSuccess;
   const void* kernels[] = {(const void*)k_tc_gemm<EPI_FWD_HIDDEN, 1>, (const void*)k_tc_gemm<EPI_FWD_HIDDEN, 2>,
                            (const void*)k_tc_gemm<EPI_FWD_LAST, 1>,   (const void*)k_tc_gemm<EPI_FWD_LAST, 2>,
-                           (const void*)k_tc_gemm<EPI_DGRAD, 1>,      (const void*)k_tc_gemm<EPI_DGRAD, 2>};
+                           (const void*)k_tc_gemm<EPI_DGRAD, 1>,      (const void*)k_tc_gemm<EPI_DGRAD, 2>,
+                           (const void*)k_tc_gemm_ks};
   for (const void* k : kernels)
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
@@ -467,7 +579,10 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
     if (l < L) {
       g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
-      TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
+      if (c->schedule == 0 && st->fwd_ks[l].splits > 1)
+        TC_TRY(launch_gemm_ks(c, wm, l == 1 ? st->x_in_ks[xb] : st->act_in_ks[l], st->fwd_ks[l], g));
+      else
+        TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
     } else if (fused_tail) {
       // last layer forward, loss, dZ_L and dgrad_L in one CUDA-core kernel
       TailLaunch tl{};

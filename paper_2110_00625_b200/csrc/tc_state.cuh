@@ -47,6 +47,10 @@ struct TcState {
   CUtensorMap w16_st[MAVG_MAX_LAYERS + 1];    // store view of the bf16 copy
   CUtensorMap u32[MAVG_MAX_LAYERS + 1];       // learner momentum buffers, the masters' view
   bool wgrad_mom = false;                     // the wgrad plans leave room for the u tile
+  // hidden-layer forward with the contraction split over a thread-block cluster (fwd_ks[l].splits
+  // > 1 where used): plan and the input maps whose box is the whole batch high
+  GemmPlan fwd_ks[MAVG_MAX_LAYERS + 1];
+  CUtensorMap act_in_ks[MAVG_MAX_LAYERS + 1], x_in_ks[2];
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   bool wgrad_merged = false;                  // all layers' weight gradients in one launch
   // whole-round kernel (round_tc.cu)

@@ -1,0 +1,80 @@
+"""Hidden-layer forward products whose contraction is split over a thread-block cluster (the
+blocks of a cluster exchange partial sums through distributed shared memory and add them in rank
+order), against the schedule that computes the same products one tile per block, and against the
+CPU oracle.  The shapes are chosen so that the default plan would otherwise cut the batch into
+32-column tiles (many learners, long contraction), which is when the cluster plan replaces it.
+The two GPU schedules differ in fp32 summation order only."""
+import numpy as np
+import pytest
+
+from tests.util import l2_rel, rel_err
+
+pytestmark = pytest.mark.gpu
+
+SEED = 0x211000625
+
+
+def _mavg():
+    import paper_2110_00625_b200 as m
+    return m
+
+
+def _cfg(**over):
+    m = _mavg()
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(S=4096, gamma=0.05)
+    cfg.update(over)
+    return cfg
+
+
+def _make(cfg, schedule):
+    m = _mavg()
+    x, y = m.workloads.make_dataset(cfg, S=cfg["S"])
+    w1 = m.workloads.mlp_init(cfg["dims"])
+    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+               seed=SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1, x=x, y=y)
+    g.set_schedule(schedule)
+    return g, x, y, w1
+
+
+SHAPES = [
+    dict(dims=[1024, 128, 10], P=64, K=1, B=64),        # clusters of 2, 8 slabs per block
+    dict(dims=[2048, 128, 10], P=32, K=1, B=128),       # clusters of 4
+    dict(dims=[1000, 200, 10], P=32, K=1, B=64),        # ragged contraction and row tiles
+    dict(dims=[3072, 512, 512, 10], P=8, K=1, B=128),   # the benchmark's first layer
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_agrees_with_one_tile_per_block(shape):
+    cfg = _cfg(**shape)
+    a, *_ = _make(cfg, 0)
+    b, *_ = _make(cfg, 2)
+    a.local_steps(); b.local_steps()
+    a.sync(); b.sync()
+    la, lb = a.get_losses(), b.get_losses()
+    # first step: same weights on both sides, only the order of fp32 sums differs; later steps
+    # start from weights that already differ by single bf16 roundings of activations and dZ
+    assert np.abs(la[:, 0] - lb[:, 0]).max() <= 1e-4 * np.abs(lb).max()
+    assert np.abs(la - lb).max() <= 1e-3 * np.abs(lb).max()
+    ra, rb = a.replicas.cpu().numpy()[:, :a.n], b.replicas.cpu().numpy()[:, :b.n]
+    w0 = a.w.cpu().numpy()
+    for j in range(0, cfg["P"], max(1, cfg["P"] // 8)):
+        assert l2_rel(ra[j] - w0, rb[j] - w0) <= 1e-2, j
+        assert rel_err(ra[j], rb[j]) <= 2e-2, j      # single elements feel ReLU branch flips
+    a.close(); b.close()
+
+
+def test_rounds_against_the_oracle(oracle):
+    cfg = _cfg(dims=[1024, 128, 10], P=64, K=2, B=64, S=8192)
+    g, x, y, w1 = _make(cfg, 0)
+    o = oracle.Mavg(w1, P=cfg["P"], K=cfg["K"], gamma=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
+                    seed=SEED, objective=oracle.OBJ_MLP, dims=cfg["dims"], bf16=True, x=x, y=y,
+                    stride=g.stride)
+    for r in range(2):
+        lg = g.round(want_loss=True)
+        lo, _ = o.run_round()
+        assert abs(lg - lo) <= 2e-2 * abs(lo), (r, lg, lo)
+        assert rel_err(g.w.cpu().numpy(), o.w) <= 5e-2, r
+        assert l2_rel(g.v.cpu().numpy(), o.v) <= 5e-2, r
+    g.close()

@@ -257,40 +257,46 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             }
           }
           if (got) {
-            const int c0 = (int)rank * 32;
-            float own[32], z[32];
-            load_acc_chunk(lane_addr, c0, g.BN, own);
+            // eight columns at a time in a loop that is not unrolled (see the note on the compact
+            // tails below); partials added in ascending rank order, this block's own from TMEM
+            const int cbase = (int)rank * 32;
+#pragma unroll 1
+            for (int s8 = 0; s8 < 32; s8 += 8) {
+              uint32_t r8[8];
+              tmem_ld_8cols(lane_addr + (uint32_t)(cbase + s8), r8);
+              tmem_ld_wait();
+              float z8[8];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) z[j] = 0.f;
-            for (int sp = 0; sp < g.splits; ++sp) {            // ascending rank order
-              if (sp == (int)rank) {
+              for (int j = 0; j < 8; ++j) z8[j] = 0.f;
+#pragma unroll 1
+              for (int sp = 0; sp < g.splits; ++sp) {
+                if (sp == (int)rank) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) z[j] += own[j];
-              } else {
-                const float4* src = reinterpret_cast<const float4*>(recv + ((size_t)sp * kBM + row) * 32);
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                  const float4 t = src[v];
-                  z[4 * v] += t.x; z[4 * v + 1] += t.y; z[4 * v + 2] += t.z; z[4 * v + 3] += t.w;
+                  for (int j = 0; j < 8; ++j) z8[j] += __uint_as_float(r8[j]);
+                } else {
+                  const float4* src =
+                      reinterpret_cast<const float4*>(recv + ((size_t)sp * kBM + row) * 32 + s8);
+                  const float4 t0 = src[0], t1 = src[1];
+                  z8[0] += t0.x; z8[1] += t0.y; z8[2] += t0.z; z8[3] += t0.w;
+                  z8[4] += t1.x; z8[5] += t1.y; z8[6] += t1.z; z8[7] += t1.w;
                 }
               }
-            }
-            uint32_t hp[16];
+              uint32_t h4[4];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const float a0 = z[2 * j] + bias_pre, a1 = z[2 * j + 1] + bias_pre;
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
-              hp[j] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            if (m_ok) {
-              const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(hp);
-              __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + c0) * g.M + m;
-              uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + c0);
+              for (int j = 0; j < 4; ++j) {
+                const float a0 = z8[2 * j] + bias_pre, a1 = z8[2 * j + 1] + bias_pre;
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
+                h4[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              if (m_ok) {
+                const int cc = cbase + s8;
+                const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(h4);
+                *reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.M + m) * g.N + n0 + cc) =
+                    make_uint4(h4[0], h4[1], h4[2], h4[3]);
+                __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.N + n0 + cc) * g.M + m;
 #pragma unroll
-              for (int v = 0; v < 4; ++v)
-                dmb[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
-#pragma unroll
-              for (int j = 0; j < 32; ++j) dbm[(size_t)j * g.M] = hh[j];
+                for (int j = 0; j < 8; ++j) dbm[(size_t)j * g.M] = hh[j];
+              }
             }
           }
         }

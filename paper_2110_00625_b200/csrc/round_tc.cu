@@ -61,7 +61,7 @@ struct RoundParams {
   int L, P, B, K, cpad;
   int first_shared;           // 1: every learner starts the round from w~ (step 1 reads w~)
   int stages;                 // pipeline depth of every forward / dgrad tile of this launch
-  int w_slots, w_a_bufs;      // ring geometry of every weight-gradient run
+  int w_slots, w_a_bufs, w_on_b;   // ring geometry of every weight-gradient run
   int g_slot_groups, g_col_splits;
   int64_t round;
   uint64_t seed;
@@ -373,7 +373,7 @@ k_mlp_round(const __grid_constant__ RoundParams rp) {
     g.nkb = y.w_nkb; g.m_tiles = y.w_m_tiles; g.n_tiles = y.w_n_tiles;
     g.chunk = y.w_chunk; g.n_chunks = y.w_n_chunks;
     g.items = P * y.w_m_tiles * y.w_n_chunks;
-    g.slots = rp.w_slots; g.a_bufs = rp.w_a_bufs;
+    g.slots = rp.w_slots; g.a_bufs = rp.w_a_bufs; g.w16_on_b = rp.w_on_b;
     g.gamma = rp.gamma;
     g.status = rp.status;
     if (vb >= g.items) return;             // nothing of this layer falls to this block
@@ -567,6 +567,7 @@ cudaError_t tc_round_launch(mavg_ctx* c, int64_t round) {
   rp->first_shared = c->replicas_equal_global ? 1 : 0;
   rp->stages = st->round_stages;
   rp->w_slots = st->wgrad[1].slots; rp->w_a_bufs = st->wgrad[1].a_bufs;
+  rp->w_on_b = st->wgrad[1].w16_on_b;
   rp->g_slot_groups = (B + 31) / 32;
   rp->g_col_splits = (cfg.dims[0] + kGatherCols - 1) / kGatherCols;
   rp->round = round; rp->seed = cfg.seed; rp->S = cfg.n_samples;

@@ -142,7 +142,9 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
   w.items = P * w.m_tiles * w.n_chunks;
   const int a_bytes = w.nkb * kBM * kBK * 2;
-  const int slot_bytes = kW32Bytes + kW16Bytes + (momentum ? kW32Bytes : 0) + w.nkb * kBN * kBK * 2;
+  const int b_bytes = w.nkb * kBN * kBK * 2;
+  w.w16_on_b = b_bytes >= kW16Bytes ? 1 : 0;   // the bf16 output tile reuses the A^T slabs' space
+  const int slot_bytes = kW32Bytes + (momentum ? kW32Bytes : 0) + (w.w16_on_b ? 0 : kW16Bytes) + b_bytes;
   const int budget = 220 * 1024;
   w.a_bufs = 2;
   w.slots = (budget - 2 * a_bytes) / slot_bytes;
@@ -182,6 +184,7 @@ WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs&
   g.items = w.items;
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
+  g.w16_on_b = w.w16_on_b;
   g.gamma = c->cfg.local_lr;
   g.beta = mom.beta;
   g.read_u = mom.read_u;
@@ -240,6 +243,7 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   g.items = w.items;
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
+  g.w16_on_b = w.w16_on_b;
   g.gamma = c->cfg.local_lr;
   g.beta = mom.beta;
   g.read_u = mom.read_u;

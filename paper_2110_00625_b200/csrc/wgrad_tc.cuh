@@ -7,7 +7,7 @@
 namespace mavg {
 
 struct WgradPlan {
-  int nkb, m_tiles, n_tiles, chunk, n_chunks, items, slots, a_bufs, grid;
+  int nkb, m_tiles, n_tiles, chunk, n_chunks, items, slots, a_bufs, grid, w16_on_b;
   size_t smem;
 };
 

@@ -46,6 +46,7 @@ struct WgradArgs {
   int items;               // P * m_tiles * n_chunks
   int slots;               // ring depth
   int a_bufs;              // 1 or 2 buffers for the dZ^T tile
+  int w16_on_b;            // 1: the bf16 output tile is written over the slot's A^T slabs
   float gamma;
   float beta;              // learner momentum (MOM)
   int read_u;              // 0: the stored u counts as zero and is not loaded
@@ -121,9 +122,14 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
   const int b_bytes = g.nkb * kBN * kBK * 2;         // A^T tile:  nkb slabs of 4 KB
-  constexpr int kUBytes = MOM ? kW32Bytes : 0;              // the u tile follows the bf16 tile
-  constexpr int kBOff = kW32Bytes + kW16Bytes + kUBytes;    // the A^T slabs come last
-  const int slot_bytes = kBOff + b_bytes;                   // multiple of 1024
+  // Slot: [master tile 16 KB][u tile 16 KB (MOM)][bf16 tile 8 KB][A^T slabs], or, when the A^T
+  // slabs are at least as large as the bf16 tile (g.w16_on_b), without a region of its own for the
+  // bf16 tile: the MMA has finished reading A^T when the epilogue writes, so the bf16 tile goes
+  // on top of it and more slots fit.
+  constexpr int kUBytes = MOM ? kW32Bytes : 0;
+  const int w16_off = kW32Bytes + kUBytes;
+  const int b_off = g.w16_on_b ? w16_off : w16_off + kW16Bytes;
+  const int slot_bytes = b_off + b_bytes;                   // multiple of 1024
   uint8_t* a_base = smem;
   uint8_t* slot_base = smem + (size_t)g.a_bufs * a_bytes;
   volatile int* abortp = &sh.abort_flag;
@@ -167,9 +173,9 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           mbar_arrive_expect_tx(&sh.slot_full[s],
                                 (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0)));
           tma_load_3d(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0);
-          if (load_u) tma_load_3d(sl + kW32Bytes + kW16Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
+          if (load_u) tma_load_3d(sl + kW32Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
-            tma_load_3d(sl + kBOff + (size_t)kb * (kBN * kBK * 2),
+            tma_load_3d(sl + b_off + (size_t)kb * (kBN * kBK * 2),
                         &tm_at, &sh.slot_full[s], kb * kBK, i0, p);
         }
       }
@@ -198,7 +204,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
             break;
           }
           tc_fence_after_sync();
-          const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + kBOff);
+          const uint32_t b_addr = smem_u32(slot_base + (size_t)s * slot_bytes + b_off);
           for (int kb = 0; kb < g.nkb; ++kb) {
             const uint64_t adesc = smem_desc_k_sw128(a_addr + kb * (kBM * kBK * 2));
             const uint64_t bdesc = smem_desc_k_sw128(b_addr + kb * (kBN * kBK * 2));
@@ -243,7 +249,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
 
         uint8_t* sl = slot_base + (size_t)s * slot_bytes;
         uint8_t* w32 = sl + (size_t)r * 128;             // 8 chunks of 16 B, chunk c at c ^ (r & 7)
-        uint8_t* w16 = sl + kW32Bytes + (size_t)r * 64;  // 4 chunks, chunk c at c ^ ((r >> 1) & 3)
+        uint8_t* w16 = sl + w16_off + (size_t)r * 64;    // 4 chunks, chunk c at c ^ ((r >> 1) & 3)
         uint32_t hp[16];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -251,8 +257,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           float4 w = *cell;
           if (MOM) {
             // the u tile has the master tile's shape and swizzle
-            float4* ucell = reinterpret_cast<float4*>(w32 + kW32Bytes + kW16Bytes +
-                                                      ((c ^ (r & 7)) << 4));
+            float4* ucell = reinterpret_cast<float4*>(w32 + kW32Bytes + ((c ^ (r & 7)) << 4));
             float4 u = g.read_u ? *ucell : make_float4(0.f, 0.f, 0.f, 0.f);
             msgd(w.x, u.x, __uint_as_float(acc[4 * c + 0]), g.gamma, g.beta);
             msgd(w.y, u.y, __uint_as_float(acc[4 * c + 1]), g.gamma, g.beta);
@@ -286,6 +291,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       bool ok = true;
       // items whose tiles have all been handed to the TMA unit but may not have reached global
       // memory yet: (index after the item's last tile, learner); signalled kStoreLag tiles later
+      int held = -1;          // slot whose stores are committed but not yet known to be read
       uint32_t pend_end[8];
       int pend_p[8];
       uint32_t ph = 0, pt = 0;
@@ -302,13 +308,26 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
           tma_store_3d(&tm_w32, sl, i0, m0, p);
-          tma_store_3d(&tm_w16, sl + kW32Bytes, i0, m0, p);
-          if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes + kW16Bytes, i0, m0, p);
+          tma_store_3d(&tm_w16, sl + w16_off, i0, m0, p);
+          if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes, i0, m0, p);
           tma_store_commit();
-          // the slot of the previous tile is free once its stores have read shared memory
-          if (tile_ctr > tile_base) {
+          // A slot is free once its stores have read shared memory.  If the next tile is already
+          // waiting to be stored, its stores go out first and this slot is handed back behind
+          // them; if not, this thread has nothing else to do, waits for the read here and hands
+          // the slot back a whole tile period earlier.
+          if (held >= 0) {
             tma_store_wait_read<1>();
-            mbar_arrive(&sh.slot_empty[(tile_ctr - 1) % g.slots]);
+            mbar_arrive(&sh.slot_empty[held]);
+            held = -1;
+          }
+          {
+            const uint32_t nx = tile_ctr + 1;
+            if (mbar_try_wait(&sh.out_full[nx % g.slots], (nx / g.slots) & 1)) {
+              held = s;
+            } else {
+              tma_store_wait_read<0>();
+              mbar_arrive(&sh.slot_empty[s]);
+            }
           }
           if (Dep::kSignals) {
             // all but the last kStoreLag store groups are in global memory
@@ -325,8 +344,10 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           ++pt;
         }
       }
-      tma_store_wait_read<0>();
-      if (tile_ctr > tile_base && ok) mbar_arrive(&sh.slot_empty[(tile_ctr - 1) % g.slots]);
+      if (held >= 0) {
+        tma_store_wait_read<0>();
+        mbar_arrive(&sh.slot_empty[held]);
+      }
       if (Dep::kSignals && ok) {
         tma_store_wait_all();
         for (; ph != pt; ++ph) dep.item_done(pend_p[ph & 7]);

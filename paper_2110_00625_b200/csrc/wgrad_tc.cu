@@ -134,7 +134,7 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   w.m_tiles = (out + kBM - 1) / kBM;
   w.n_tiles = (in + kBN - 1) / kBN;
   const long total = (long)P * w.m_tiles * w.n_tiles;
-  long chunk = total / (8L * sm_count);
+  long chunk = total / (5L * sm_count);
   if (chunk < 1) chunk = 1;
   if (chunk > 16) chunk = 16;
   if (chunk > w.n_tiles) chunk = w.n_tiles;

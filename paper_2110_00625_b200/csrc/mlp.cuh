@@ -53,13 +53,13 @@ struct TailLaunch {
   __nv_bfloat16* dzp_bm;         // out: dZ_{L-1} [P, B, in] and its transpose [P, in, B]
   __nv_bfloat16* dzp_mb;
   float* part;                   // scratch of tail_fused_part_bytes()
-  int* counters;                 // [P] ints, zero between launches
   MomArgs mom;
 };
 bool tail_fused_supported(const mavg_config* cfg);
 size_t tail_fused_part_bytes(const mavg_config* cfg);
 cudaError_t tail_fused_prepare();
-cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t);
+cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t);    // the products, dZ, partial sums
+cudaError_t launch_tail_finish(mavg_ctx* c, const TailLaunch& t);   // bias steps and loss from the partials
 
 // Whole-round kernel (round_tc.cu): all K local steps of a round in one launch.
 bool tc_round_supported(mavg_ctx* c);

@@ -550,6 +550,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   const bool shared_w = c->replicas_equal_global;   // first step after a (re-)broadcast
   const MomArgs mom = mom_args(c, shared_w);
   const bool fused_tail = st->tail_ok && c->schedule == 0;
+  bool tail_on_side = false;
   const bool overlap = !c->profiling;
   const int xb = step & 1;                          // batch buffer of this step
   cudaStream_t main_s = c->stream;
@@ -594,9 +595,19 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       tl.dz_t = bfp(t.dz_t[L]);
       if (L >= 2) { tl.dzp_bm = bfp(t.dz[L - 1]); tl.dzp_mb = bfp(t.dz_t[L - 1]); }
       tl.part = (float*)(ws + t.tail_part);
-      tl.counters = counters;
       tl.mom = mom;
       TC_TRY(launch_tail_fused(c, tl));
+      // bias steps and loss: beside the backward pass, joined at the end of the step
+      if (overlap) {
+        TC_TRY(cudaEventRecord(st->ev_fork, main_s));
+        TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
+        c->stream = st->s_wgrad;
+        TC_TRY(launch_tail_finish(c, tl));
+        c->stream = main_s;
+        tail_on_side = true;
+      } else {
+        TC_TRY(launch_tail_finish(c, tl));
+      }
     } else {
       g.labels = labels_b; g.loss_out = losses + (step - 1); g.loss_stride = K;
       g.dz_bm = bfp(t.dz[L]); g.cpad = t.cpad; g.dz_mb = bfp(t.dz_t[L]);
@@ -616,7 +627,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     TC_TRY(cudaEventRecord(st->ev_gather_done, st->s_gather));
   }
 
-  bool side_used = false;
+  bool side_used = tail_on_side;
   const bool merged = st->wgrad_merged && c->schedule == 0;
   for (int l = L; l >= 1; --l) {
     const MlpLayer& ly = c->layers[l - 1];

@@ -9,9 +9,9 @@
 //   dA[b, k]     = sum_c bf16(dZ[b, c]) W[c, k];   dZprev[b, k] = A[b, k] > 0 ? dA[b, k] : 0
 // and writes bf16(dZ) transposed (the weight-gradient kernel's operand), bf16(dZprev) in both
 // orientations, and per-block partial sums of the loss and of the two bias gradients (from the
-// unrounded dZ values).  The block of a learner that finishes last adds the partials in ascending
-// block order and takes the bias steps of Algorithm 1's local update, so the result does not
-// depend on the order in which blocks run.
+// unrounded dZ values).  A second small kernel adds the partials in ascending block order and
+// takes the bias steps of Algorithm 1's local update; it runs beside the rest of the backward
+// pass, which needs dZ_{L-1} but neither the biases nor the loss.
 #include "mlp.cuh"
 
 namespace mavg {
@@ -37,7 +37,6 @@ struct TailArgs {
   __nv_bfloat16* dzp_bm;         // dZ_{L-1} [P, B, in]     (null for a one-layer model)
   __nv_bfloat16* dzp_mb;         // dZ_{L-1} transposed [P, in, B]
   float* part;                   // [P, blocks, in + C + 1] partial sums
-  int* counters;                 // [P], zero between launches
   int B, in, C;
   float gamma;
   MomArgs mom;
@@ -55,7 +54,6 @@ k_last_layer_fused(const TailArgs g) {
   __shared__ float row_loss[kRows];
   __shared__ float bias_s[kMaxC];
   __shared__ int label_s[kRows];
-  __shared__ int is_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
   const int r0 = blk * kRows;
@@ -171,19 +169,16 @@ k_last_layer_fused(const TailArgs g) {
       part[k] = colsum;
     }
   }
+}
 
-  // the learner's last block adds the partials (ascending block order) and steps the biases
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int old = atomicAdd(g.counters + p, 1);
-    const int last = old == nblk - 1;
-    if (last) g.counters[p] = 0;
-    __threadfence();
-    is_last = last;
-  }
-  __syncthreads();
-  if (!is_last) return;
+// Second half, off the step's critical chain (nothing later in the step reads what it writes):
+// block p adds the per-block partials of learner p in ascending block order and takes the bias
+// steps of Algorithm 1's local update for the last two layers; it also writes the minibatch loss.
+__global__ void __launch_bounds__(kThreads)
+k_last_layer_finish(const TailArgs g, int nblk) {
+  const int tid = threadIdx.x, p = blockIdx.x;
+  const int in = g.in, C = g.C, B = g.B;
+  const float* bias_in = g.bias_in + (size_t)p * g.bias_in_stride;
   const float* pp = g.part + (size_t)p * nblk * (in + C + 1);
   float* rep = g.rep + (size_t)p * g.rep_stride;
   float* urow = g.mom.u ? g.mom.u + (size_t)p * g.mom.u_stride : nullptr;
@@ -191,7 +186,8 @@ k_last_layer_fused(const TailArgs g) {
   for (int i = tid; i < in + C + 1; i += kThreads) {
     if (i < in && i >= n_sum) continue;
     float s = 0.f;
-    for (int b = 0; b < nblk; ++b) s += __ldcg(pp + (size_t)b * (in + C + 1) + i);
+#pragma unroll 4
+    for (int b = 0; b < nblk; ++b) s += pp[(size_t)b * (in + C + 1) + i];
     if (i < in) {
       const int64_t o = g.bprev_off + i;
       local_update(rep + o, bias_in[o], urow ? urow + o : nullptr, g.mom.read_u, s, g.gamma, g.mom.beta);
@@ -225,7 +221,8 @@ cudaError_t tail_fused_prepare() {
                               160 * 1024);
 }
 
-cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t) {
+namespace {
+TailArgs tail_args(mavg_ctx* c, const TailLaunch& t) {
   const mavg_config& cfg = c->cfg;
   const int L = cfg.n_layers;
   const MlpLayer& ly = c->layers[L - 1];
@@ -246,15 +243,28 @@ cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t) {
   g.dzp_bm = L >= 2 ? t.dzp_bm : nullptr;
   g.dzp_mb = L >= 2 ? t.dzp_mb : nullptr;
   g.part = t.part;
-  g.counters = t.counters;
   g.B = cfg.B;
   g.in = ly.in;
   g.C = ly.out;
   g.gamma = cfg.local_lr;
   g.mom = t.mom;
-  dim3 grid((unsigned)(cfg.B / kRows), (unsigned)cfg.P);
+  return g;
+}
+}  // namespace
+
+cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t) {
+  const TailArgs g = tail_args(c, t);
+  dim3 grid((unsigned)(c->cfg.B / kRows), (unsigned)c->cfg.P);
   prof_begin(c, MAVG_K_LOSS);
-  k_last_layer_fused<<<grid, kThreads, tail_smem_bytes(ly.in, ly.out), c->stream>>>(g);
+  k_last_layer_fused<<<grid, kThreads, tail_smem_bytes(g.in, g.C), c->stream>>>(g);
+  prof_end(c);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_tail_finish(mavg_ctx* c, const TailLaunch& t) {
+  const TailArgs g = tail_args(c, t);
+  prof_begin(c, MAVG_K_LOSS);
+  k_last_layer_finish<<<c->cfg.P, kThreads, 0, c->stream>>>(g, c->cfg.B / kRows);
   prof_end(c);
   return cudaGetLastError();
 }

@@ -165,9 +165,9 @@ def run_reference(args):
 # stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
 # captured; set an entry to None when its kernel changes.
 NCU_TRAFFIC_C2 = {
-    "wgrad_sgd_gemm": 69.459968e6 + 33.750016e6,                 # one launch for all layers
-    "fwd_gemm": (31.539968e6 + 0.002048e6 + 5.325824e6) / 2,     # hidden layers 1 and 2
-    "dgrad_gemm": 6.381568e6,
+    "wgrad_sgd_gemm": 69.426688e6 + 33.094400e6,                 # one launch for all layers
+    "fwd_gemm": (31.498240e6 + 5.325056e6) / 2,                  # hidden layers 1 and 2
+    "dgrad_gemm": 6.381824e6,
 }
 
 

@@ -116,6 +116,7 @@ struct mavg_ctx {
   float graph_beta = 0.f;
   int graph_reset = 0;
   int graph_schedule = 0;
+  int graph_w16_cur = 0;      // state of the doubled bf16 copy after the recorded steps
   int64_t graph_nodes = 0;
 };
 

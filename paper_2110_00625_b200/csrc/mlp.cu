@@ -113,6 +113,7 @@ cudaError_t build_graph(mavg_ctx* c, int64_t round) {
   c->graph_beta = c->cfg.learner_momentum;
   c->graph_reset = c->cfg.learner_momentum_reset;
   c->graph_schedule = c->schedule;
+  c->graph_w16_cur = use_tensor_cores(&c->cfg) ? tc_get_w16_cur(c) : 0;
   return cudaSuccess;
 }
 
@@ -156,6 +157,7 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
   if (e != cudaSuccess) return e;
   c->launches += c->graph_nodes;
   c->replicas_equal_global = false;
+  if (use_tensor_cores(&c->cfg)) tc_set_w16_cur(c, c->graph_w16_cur);
   return cudaSuccess;
 }
 

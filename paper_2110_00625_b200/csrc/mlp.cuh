@@ -65,6 +65,9 @@ cudaError_t launch_tail_finish(mavg_ctx* c, const TailLaunch& t);   // bias step
 bool tc_round_supported(mavg_ctx* c);
 cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
 
+int tc_get_w16_cur(mavg_ctx* c);            // which bf16 copy of the doubled layer is current
+void tc_set_w16_cur(mavg_ctx* c, int cur);
+
 inline bool use_tensor_cores(const mavg_config* cfg) { return cfg->gemm_bf16 == 1; }
 
 }  // namespace mavg

@@ -214,6 +214,8 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.round_ctr_bytes = (size_t)4 * (MAVG_MAX_LAYERS + 1) * P * sizeof(int);
   t.round_ctr = take(t.round_ctr_bytes);
   t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
+  t.w16b_stride = L >= 3 ? (int64_t)up((size_t)cfg->dims[L - 2] * cfg->dims[L - 1], 64) : 0;
+  t.w16b = take(L >= 3 ? (size_t)P * t.w16b_stride * 2 : 16);
   t.end = off;
   return t;
 }
@@ -409,6 +411,15 @@ mavg_status tc_setup(mavg_ctx* c) {
     ok = ok && encode_map(st, &st->w[l], w16, in, out, P, in, t.n16, kBM, &why);
     ok = ok && encode_map(st, &st->wg[l], w16g, in, out, 1, in, t.n16, kBM, &why);
     ok = ok && encode_map(st, &st->w_mn[l], w16, in, out, P, in, t.n16, 64, &why);
+    if (L >= 3 && l == L - 1) {      // second copy of this layer's bf16 weights
+      st->dbl_layer = l;
+      __nv_bfloat16* wb = (__nv_bfloat16*)bf(t.w16b);
+      ok = ok && encode_map(st, &st->w_b, wb, in, out, P, in, t.w16b_stride, kBM, &why);
+      ok = ok && encode_map(st, &st->w_mn_b, wb, in, out, P, in, t.w16b_stride, 64, &why);
+      ok = ok && encode_any(st, &st->w16_st_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, wb, in, out, P,
+                            in, t.w16b_stride, kWgradTileCols, kWgradTileRows,
+                            CU_TENSOR_MAP_SWIZZLE_64B, &why);
+    }
     ok = ok && encode_map(st, &st->wg_mn[l], w16g, in, out, 1, in, t.n16, 64, &why);
     if (l == 1) {
       for (int i = 0; i < 2 && ok; ++i) {
@@ -508,6 +519,11 @@ void tc_teardown(mavg_ctx* c) {
   c->mlp = nullptr;
 }
 
+int tc_get_w16_cur(mavg_ctx* c) { return c->mlp ? ((TcState*)c->mlp)->w16_cur : 0; }
+void tc_set_w16_cur(mavg_ctx* c, int cur) {
+  if (c->mlp) ((TcState*)c->mlp)->w16_cur = cur;
+}
+
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
   TcState* st = (TcState*)c->mlp;
   const TcLayout& t = st->lay;
@@ -549,11 +565,36 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   int* counters = (int*)(ws + t.counters);
   const bool shared_w = c->replicas_equal_global;   // first step after a (re-)broadcast
   const MomArgs mom = mom_args(c, shared_w);
+  const bool overlap = !c->profiling;
   const bool fused_tail = st->tail_ok && c->schedule == 0;
   bool tail_on_side = false;
-  const bool overlap = !c->profiling;
+  const bool merged = st->wgrad_merged && c->schedule == 0;
+  // Weight gradients of the last two layers beside the remaining dgrad products (their dZ comes
+  // out of the fused last-layer kernel): layer L-1 then writes the other of its two bf16 copies,
+  // because dgrad through it still reads the current one.
+  const bool split_wg = merged && fused_tail && overlap && L >= 3 && st->dbl_layer == L - 1;
+  const int rd = st->w16_cur;                                  // copy read in this step
+  const int wr = split_wg ? (shared_w ? 0 : 1 - rd) : rd;      // copy written in this step
+  auto w_k = [&](int l) -> const CUtensorMap& {
+    return (l == st->dbl_layer && rd == 1) ? st->w_b : st->w[l]; };
+  auto w_mn = [&](int l) -> const CUtensorMap& {
+    return (l == st->dbl_layer && rd == 1) ? st->w_mn_b : st->w_mn[l]; };
+  auto w_st = [&](int l) -> const CUtensorMap* {
+    return (l == st->dbl_layer && wr == 1) ? &st->w16_st_b : &st->w16_st[l]; };
   const int xb = step & 1;                          // batch buffer of this step
   cudaStream_t main_s = c->stream;
+  auto layer_ref = [&](int l) {
+    WgradLayerRef r{};
+    r.plan = &st->wgrad[l];
+    r.dzt = &st->dz_t[l];
+    r.at = l == 1 ? &st->x_in_t[xb] : &st->act_in_t[l];
+    r.w32 = &st->w32[l];
+    r.w16 = w_st(l);
+    r.w32_shared = shared_w ? &st->w32g[l] : nullptr;
+    r.u32 = st->wgrad_mom ? &st->u32[l] : nullptr;
+    return r;
+  };
+
   cudaError_t e;
 #define TC_TRY(call) do { if ((e = (call)) != cudaSuccess) { c->stream = main_s; return e; } } while (0)
 
@@ -576,7 +617,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     g.bias_rep = c->buf.replicas; g.bias_off = ly.b_off;
     g.bias_in = shared_w ? c->buf.global_w : c->buf.replicas;
     g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
-    const CUtensorMap& wm = shared_w ? st->wg[l] : st->w[l];
+    const CUtensorMap& wm = shared_w ? st->wg[l] : w_k(l);
     const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
     if (l < L) {
       g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
@@ -602,6 +643,14 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
         TC_TRY(cudaEventRecord(st->ev_fork, main_s));
         TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
         c->stream = st->s_wgrad;
+        if (split_wg) {
+          // the last two layers' weight gradients first (they are on the way of the next
+          // step), leaving the SMs of the dgrad tiles alone; then the bias steps and the loss
+          WgradLayerRef refs[2] = {layer_ref(L), layer_ref(L - 1)};
+          const int busy = cfg.P * st->dgrad[L - 1].m_tiles;
+          const int cap = c->sm_count - busy >= 32 ? c->sm_count - busy : 0;
+          TC_TRY(launch_wgrad_multi(c, 2, refs, mom, cap));
+        }
         TC_TRY(launch_tail_finish(c, tl));
         c->stream = main_s;
         tail_on_side = true;
@@ -628,7 +677,6 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   }
 
   bool side_used = tail_on_side;
-  const bool merged = st->wgrad_merged && c->schedule == 0;
   for (int l = L; l >= 1; --l) {
     const MlpLayer& ly = c->layers[l - 1];
     if (l > 1 && !(fused_tail && l == L)) {
@@ -644,7 +692,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.mask_mb = bfp(t.act_t[l - 1]);
       g.a_mn = 1;
       g.mom = mom;
-      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : st->w_mn[l],
+      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : w_mn(l),
                                     st->dz[l], st->dgrad[l], g));
     }
     const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
@@ -653,30 +701,23 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
       c->stream = st->s_wgrad;
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
       c->stream = main_s;
       side_used = true;
     } else {
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], st->w16_st[l],
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
     }
   }
   if (merged) {
     // largest layer first, so that the small ones fill the ragged end of the launch
     WgradLayerRef refs[MAVG_MAX_LAYERS];
-    for (int l = 1; l <= L; ++l) {
-      WgradLayerRef& r = refs[l - 1];
-      r.plan = &st->wgrad[l];
-      r.dzt = &st->dz_t[l];
-      r.at = l == 1 ? &st->x_in_t[xb] : &st->act_in_t[l];
-      r.w32 = &st->w32[l];
-      r.w16 = &st->w16_st[l];
-      r.w32_shared = shared_w ? &st->w32g[l] : nullptr;
-      r.u32 = st->wgrad_mom ? &st->u32[l] : nullptr;
-    }
-    TC_TRY(launch_wgrad_multi(c, L, refs, mom));
+    const int top = split_wg ? L - 2 : L;      // the last two layers already run on the side
+    for (int l = 1; l <= top; ++l) refs[l - 1] = layer_ref(l);
+    TC_TRY(launch_wgrad_multi(c, top, refs, mom));
   }
+  st->w16_cur = wr;
   if (overlap) {
     TC_TRY(cudaEventRecord(st->ev_x_free[xb], main_s));     // wgrad_1 was the buffer's last reader
     if (side_used) {

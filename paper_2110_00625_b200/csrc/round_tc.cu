@@ -544,6 +544,9 @@ cudaError_t tc_round_launch(mavg_ctx* c, int64_t round) {
     rp->act_in[l] = st->act_in[l]; rp->act_in_t[l] = st->act_in_t[l];
     rp->dz[l] = st->dz[l]; rp->dz_t[l] = st->dz_t[l];
     rp->w32[l] = st->w32[l]; rp->w32g[l] = st->w32g[l]; rp->w16_st[l] = st->w16_st[l];
+    if (l == st->dbl_layer && st->w16_cur == 1) {   // the copy that holds this layer's weights now
+      rp->w[l] = st->w_b; rp->w_mn[l] = st->w_mn_b; rp->w16_st[l] = st->w16_st_b;
+    }
     RoundLayer& y = rp->ly[l];
     const MlpLayer& ml = c->layers[l - 1];
     y.in = ml.in; y.out = ml.out; y.w_off = ml.w_off; y.b_off = ml.b_off;

@@ -21,6 +21,8 @@ struct TcLayout {
   size_t w16, w16g;
   size_t round_ctr, round_ctr_bytes;         // completion counters of the whole-round kernel
   size_t tail_part;                          // partial sums of the fused last-layer kernel
+  size_t w16b;                               // second bf16 copy of layer L-1's weights [P, w16b_stride]
+  int64_t w16b_stride;
   size_t end;
 };
 
@@ -51,6 +53,12 @@ struct TcState {
   // > 1 where used): plan and the input maps whose box is the whole batch high
   GemmPlan fwd_ks[MAVG_MAX_LAYERS + 1];
   CUtensorMap act_in_ks[MAVG_MAX_LAYERS + 1], x_in_ks[2];
+  // Layer L-1's bf16 weights exist twice (L >= 3): where its weight gradient runs beside the
+  // dgrad product that still reads the old copy, it writes the other one.  w16_cur says which
+  // copy holds the current weights; *_b are the views of copy 1.
+  int dbl_layer = 0;
+  int w16_cur = 0;
+  CUtensorMap w_b, w_mn_b, w16_st_b;
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   bool wgrad_merged = false;                  // all layers' weight gradients in one launch
   // whole-round kernel (round_tc.cu)
@@ -70,5 +78,7 @@ struct TcState {
 bool tc_round_supported(mavg_ctx* c);
 cudaError_t tc_round_prepare(mavg_ctx* c);
 cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
+int tc_get_w16_cur(mavg_ctx* c);
+void tc_set_w16_cur(mavg_ctx* c, int cur);
 
 }  // namespace mavg

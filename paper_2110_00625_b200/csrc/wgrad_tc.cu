@@ -193,12 +193,14 @@ WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs&
 }
 }  // namespace
 
-cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers, const MomArgs& mom) {
+cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers, const MomArgs& mom,
+                               int max_grid) {
   WgradMultiParams* mp = new WgradMultiParams();
   mp->n = n;
   int grid = 1, rot = 0;
   size_t smem = 0;
   for (int s = 0; s < n; ++s) grid = layers[s].plan->grid > grid ? layers[s].plan->grid : grid;
+  if (max_grid > 0 && grid > max_grid) grid = max_grid;
   const bool with_u = mom.u != nullptr;
   for (int s = 0; s < n; ++s) {
     const WgradLayerRef& r = layers[s];

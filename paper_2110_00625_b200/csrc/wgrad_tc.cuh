@@ -36,7 +36,8 @@ struct WgradLayerRef {
   const CUtensorMap* w32_shared;   // null: every learner loads its own masters
   const CUtensorMap* u32;          // learner momentum view (may be null without momentum)
 };
+// max_grid > 0 caps the number of blocks (a launch that shares the GPU with another kernel).
 cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers,
-                               const MomArgs& mom = MomArgs());
+                               const MomArgs& mom = MomArgs(), int max_grid = 0);
 
 }  // namespace mavg

@@ -277,3 +277,28 @@ def test_training_converges_and_block_momentum_accelerates():
         final[mu] = float(np.mean(losses[-5:]))
         g.close()
     assert final[0.7] < final[0.0]
+
+
+def test_tc_mixed_call_sequences_keep_the_same_bits():
+    # The default schedule keeps two bf16 copies of one layer's weights and alternates between
+    # them from step to step, but only in its overlapped (graph) form.  Whatever mixture of graph
+    # rounds, launch-by-launch rounds, repeated local steps, resumes and schedule changes a caller
+    # makes, the result must be that of the same calls issued launch by launch.
+    def run(profiled):
+        g = _tc_handle(K=3)               # odd K: the current copy changes from round to round
+        g.set_profiling(profiled)
+        g.round()
+        g.set_profiling(True); g.round(); g.set_profiling(profiled)
+        g.local_steps(); g.local_steps(); g.meta_update()
+        g.set_schedule(2); g.round(); g.set_schedule(0)
+        g.round()
+        g.set_round(g.get_round())        # resume: re-broadcast, next step starts from w~ again
+        g.set_hparams(2, 0.02, 1.0, 0.9)
+        g.round(); g.round()
+        g.sync()
+        out = (g.w.cpu().numpy(), g.v.cpu().numpy(), g.replicas.cpu().numpy()[:, :g.n])
+        g.close()
+        return out
+    a, b = run(False), run(True)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)

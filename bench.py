@@ -165,9 +165,10 @@ def run_reference(args):
 # stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
 # captured; set an entry to None when its kernel changes.
 NCU_TRAFFIC_C2 = {
-    "wgrad_sgd_gemm": 69.426688e6 + 33.094400e6,                 # one launch for all layers
-    "fwd_gemm": (31.498240e6 + 5.325056e6) / 2,                  # hidden layers 1 and 2
-    "dgrad_gemm": 6.381824e6,
+    # all layers' weight gradients (captured as the graph's two launches, layer 1 and layers 3 + 2)
+    "wgrad_sgd_gemm": 57.702656e6 + 21.394176e6 + 11.806976e6 + 0.007424e6,
+    "fwd_gemm": (31.498240e6 + 0.001536e6 + 5.325824e6) / 2,     # hidden layers 1 and 2
+    "dgrad_gemm": 6.381056e6,
 }
 
 

@@ -118,13 +118,20 @@ k_tc_gemm_ks(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 }
 
 // bf16 copy of the global model w~ (shared by all learners at the first step of a round, when
-// every replica equals w~).  One launch per layer; grid-stride over the layer's weights.
+// every replica equals w~).  One launch for all layers: block row y takes layer y, grid-stride
+// over that layer's weights.
+struct ShadowArgs {
+  int64_t w_off[MAVG_MAX_LAYERS], total[MAVG_MAX_LAYERS], sh_off[MAVG_MAX_LAYERS];
+};
 __global__ void __launch_bounds__(256)
-k_shadow_from_global(const float* __restrict__ w, int64_t w_off, int64_t total,
-                     __nv_bfloat16* __restrict__ w16, int64_t sh_off) {
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+k_shadow_from_global(const float* __restrict__ w, __nv_bfloat16* __restrict__ w16,
+                     const ShadowArgs a) {
+  const int l = blockIdx.y;
+  const float* src = w + a.w_off[l];
+  __nv_bfloat16* dst = w16 + a.sh_off[l];
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < a.total[l];
        t += (int64_t)gridDim.x * blockDim.x)
-    w16[sh_off + t] = __float2bfloat16_rn(w[w_off + t]);
+    dst[t] = __float2bfloat16_rn(src[t]);
 }
 
 // ---------------------------------------------------------------------------------- host side
@@ -528,18 +535,22 @@ cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
   TcState* st = (TcState*)c->mlp;
   const TcLayout& t = st->lay;
   char* ws = (char*)c->buf.workspace;
+  ShadowArgs a{};
+  int64_t most = 0;
   for (int l = 1; l <= c->cfg.n_layers; ++l) {
     const MlpLayer& ly = c->layers[l - 1];
-    const int64_t total = (int64_t)ly.in * ly.out;
-    int grid = (int)std::min<int64_t>((total + 255) / 256, (int64_t)c->sm_count * 8);
-    prof_begin(c, MAVG_K_AUX);
-    k_shadow_from_global<<<grid, 256, 0, c->stream>>>(c->buf.global_w, ly.w_off, total,
-                                                      (__nv_bfloat16*)(ws + t.w16g),
-                                                      t.sh_off[l - 1]);
-    prof_end(c);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    a.w_off[l - 1] = ly.w_off;
+    a.total[l - 1] = (int64_t)ly.in * ly.out;
+    a.sh_off[l - 1] = t.sh_off[l - 1];
+    most = std::max(most, a.total[l - 1]);
   }
+  const int gx = (int)std::min<int64_t>((most + 255) / 256, (int64_t)c->sm_count * 4);
+  prof_begin(c, MAVG_K_AUX);
+  k_shadow_from_global<<<dim3((unsigned)gx, (unsigned)c->cfg.n_layers), 256, 0, c->stream>>>(
+      c->buf.global_w, (__nv_bfloat16*)(ws + t.w16g), a);
+  prof_end(c);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
   return cudaSuccess;
 }
 

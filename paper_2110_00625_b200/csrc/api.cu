@@ -152,8 +152,9 @@ mavg_status do_meta_update(mavg_ctx* c) {
   CU(c, launch_meta_update(c), "meta-update");
   c->round += 1;
   c->replicas_equal_global = true;
-  if (c->cfg.objective == MAVG_OBJ_MLP)
+  if (c->cfg.objective == MAVG_OBJ_MLP && !c->shadow_fresh)
     CU(c, mlp_refresh_shared_operands(c), "operand refresh after the meta-update");
+  c->shadow_fresh = false;
   return MAVG_OK;
 }
 

@@ -67,6 +67,15 @@ struct MlpLayer {
   int64_t w_off, b_off;      // offsets (floats) inside a replica
 };
 
+// bf16 copy of the global model's weight matrices (the tensor-core path's shared operand at the
+// first step of a round): layer l's weights w[w_off[l] .. w_off[l] + total[l]) go to
+// dst[sh_off[l] ..).  All offsets and lengths are multiples of 4 elements.
+struct ShadowMap {
+  __nv_bfloat16* dst = nullptr;
+  int L = 0;
+  int64_t w_off[MAVG_MAX_LAYERS] = {}, total[MAVG_MAX_LAYERS] = {}, sh_off[MAVG_MAX_LAYERS] = {};
+};
+
 struct Workspace {           // byte offsets into the caller's scratch buffer
   size_t status = 0;         // int32[64]: [0] device wait-limit flag; bytes 64..71: round (int64)
   size_t losses = 0;         // float [P*K]
@@ -96,6 +105,8 @@ struct mavg_ctx {
   mavg::Workspace ws;
   std::vector<mavg::MlpLayer> layers;
   void* mlp = nullptr;        // state of the MLP path (owned by mlp files)
+  mavg::ShadowMap shadow;     // set by the tensor-core path; dst == nullptr otherwise
+  bool shadow_fresh = false;  // the last meta-update wrote the bf16 copy of w~ itself
   // per-launch timing (mavg_set_profiling): one event pair per launch, summed per kernel class
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;

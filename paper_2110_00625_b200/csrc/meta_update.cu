@@ -34,11 +34,13 @@ __device__ __forceinline__ void meta_scalar(float* rep, int64_t stride, float* w
 
 // U replica loads are kept in flight per thread; STREAM_ST selects evict-first stores for the
 // broadcast (replica sets far larger than L2) or plain stores (sets the next kernel re-reads).
-template <int U, bool STREAM_ST>
+// SHADOW: also writes the bf16 copy of the new w~'s weight matrices (see ShadowMap), which saves
+// the separate pass that would read w~ again.
+template <int U, bool STREAM_ST, bool SHADOW = false>
 __global__ void __launch_bounds__(256)
 k_meta_update(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
               float* __restrict__ v, int P, int64_t n, float mu, float zeta, float inv_p,
-              int read_v, int bcast) {
+              int read_v, int bcast, const ShadowMap sm = ShadowMap()) {
   const int64_t n4 = n >> 2;
   const int64_t stride4 = stride >> 2;
   float4* rep4 = reinterpret_cast<float4*>(rep);
@@ -76,6 +78,18 @@ k_meta_update(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
       w4[q] = wn;
       if (bcast)
         for (int j = 0; j < P; ++j) rep4[(size_t)j * stride4 + q] = wn;
+    }
+    if (SHADOW) {
+      const int64_t i = q << 2;
+      for (int l = 0; l < sm.L; ++l) {
+        const int64_t r = i - sm.w_off[l];
+        if (r >= 0 && r < sm.total[l]) {
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(wn.x, wn.y), h1 = __floats2bfloat162_rn(wn.z, wn.w);
+          *reinterpret_cast<uint2*>(sm.dst + sm.sh_off[l] + r) =
+              make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+          break;
+        }
+      }
     }
   }
   // ragged tail (n not a multiple of 4)
@@ -324,10 +338,16 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
     float* rep = c->buf.replicas + done;
     float* w = c->buf.global_w + done;
     float* v = c->buf.momentum + done;
+    c->shadow_fresh = false;
     if (big)
       k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
                                                           rest, mu, zeta, inv_p, read_v, bcast);
-    else
+    else if (c->shadow.dst && done == 0) {
+      k_meta_update<8, false, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
+                                                                 rest, mu, zeta, inv_p, read_v, bcast,
+                                                                 c->shadow);
+      c->shadow_fresh = true;
+    } else
       k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
                                                            rest, mu, zeta, inv_p, read_v, bcast);
     e = cudaGetLastError();

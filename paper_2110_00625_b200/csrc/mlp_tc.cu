@@ -493,6 +493,14 @@ mavg_status tc_setup(mavg_ctx* c) {
     for (int l = 2; l <= L; ++l)
       if (st->wgrad[l].slots != w1.slots || st->wgrad[l].a_bufs != w1.a_bufs) st->wgrad_merged = false;
   }
+  // the meta-update writes the bf16 copy of w~ itself where its vector kernel takes the whole model
+  c->shadow.dst = (__nv_bfloat16*)(ws + t.w16g);
+  c->shadow.L = L;
+  for (int l = 1; l <= L; ++l) {
+    c->shadow.w_off[l - 1] = c->layers[l - 1].w_off;
+    c->shadow.total[l - 1] = (int64_t)c->layers[l - 1].in * c->layers[l - 1].out;
+    c->shadow.sh_off[l - 1] = t.sh_off[l - 1];
+  }
   st->tail_ok = tail_fused_supported(&cfg) &&
                 P * ((cfg.dims[L - 1] + kBM - 1) / kBM) <= c->sm_count / 2;
   if (e == cudaSuccess && st->tail_ok) e = tail_fused_prepare();

@@ -157,7 +157,9 @@ mavg_status mavg_round(mavg_handle h, float *mean_loss);
 
 /* The same round for a caller whose model lives in HOST memory: copies w~ and v (n floats each,
  * HOST, read and written) to the device, re-broadcasts w~ to the replicas, runs the round,
- * copies w~ and v back and waits.  mean_loss as in mavg_round. */
+ * copies w~ and v back and waits.  The upload of v runs on a stream the handle owns, beside the
+ * local steps; both host arrays must stay untouched until the call returns.  mean_loss as in
+ * mavg_round. */
 mavg_status mavg_round_host(mavg_handle h, float *w_host, float *v_host, float *mean_loss);
 
 /* Per-round schedules (Algorithm 1 lets gamma_n and B_n vary with n; B stays fixed here). */

@@ -300,13 +300,25 @@ mavg_status mavg_round_host(mavg_handle h, float* w_host, float* v_host, float* 
   if (h->cfg.objective == MAVG_OBJ_NONE)
     return set_err(h, MAVG_ERR_STATE, "this handle has no learner level (MAVG_OBJ_NONE)");
   const size_t bytes = (size_t)h->cfg.n * sizeof(float);
+  if (!h->s_copy) {
+    CU(h, cudaStreamCreateWithFlags(&h->s_copy, cudaStreamNonBlocking), "copy stream");
+    CU(h, cudaEventCreateWithFlags(&h->ev_copy_fork, cudaEventDisableTiming), "copy event");
+    CU(h, cudaEventCreateWithFlags(&h->ev_copy_done, cudaEventDisableTiming), "copy event");
+  }
+  // v is first needed by the meta-update: its upload follows whatever the caller's stream did with
+  // the buffer before this call and runs beside the K local steps
+  // (submitted after w~, which the copy engine then serves first)
   CU(h, cudaMemcpyAsync(h->buf.global_w, w_host, bytes, cudaMemcpyHostToDevice, h->stream), "w~ upload");
-  CU(h, cudaMemcpyAsync(h->buf.momentum, v_host, bytes, cudaMemcpyHostToDevice, h->stream), "v upload");
+  CU(h, cudaEventRecord(h->ev_copy_fork, h->stream), "copy fork");
+  CU(h, cudaStreamWaitEvent(h->s_copy, h->ev_copy_fork, 0), "copy fork");
+  CU(h, cudaMemcpyAsync(h->buf.momentum, v_host, bytes, cudaMemcpyHostToDevice, h->s_copy), "v upload");
+  CU(h, cudaEventRecord(h->ev_copy_done, h->s_copy), "copy join");
   CU(h, launch_broadcast(h, false), "re-broadcast");
   h->replicas_equal_global = true;
   if (h->cfg.objective == MAVG_OBJ_MLP)
     CU(h, mlp_refresh_shared_operands(h), "operand refresh");
   mavg_status st = do_local_steps(h);
+  CU(h, cudaStreamWaitEvent(h->stream, h->ev_copy_done, 0), "copy join");   // also on an error return
   if (st != MAVG_OK) return st;
   st = do_meta_update(h);
   if (st != MAVG_OK) return st;
@@ -447,6 +459,9 @@ const char* mavg_last_error(mavg_handle h) {
 mavg_status mavg_destroy(mavg_handle h) {
   if (!h) return MAVG_OK;
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  if (h->ev_copy_fork) cudaEventDestroy(h->ev_copy_fork);
+  if (h->ev_copy_done) cudaEventDestroy(h->ev_copy_done);
+  if (h->s_copy) cudaStreamDestroy(h->s_copy);
   mlp_teardown(h);
   delete h;
   return MAVG_OK;

@@ -129,6 +129,9 @@ struct mavg_ctx {
   int graph_schedule = 0;
   int graph_w16_cur = 0;      // state of the doubled bf16 copy after the recorded steps
   int64_t graph_nodes = 0;
+  // mavg_round_host: the upload of v runs on a copy stream of its own, next to the local steps
+  cudaStream_t s_copy = nullptr;
+  cudaEvent_t ev_copy_fork = nullptr, ev_copy_done = nullptr;
 };
 
 namespace mavg {

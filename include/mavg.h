@@ -133,7 +133,12 @@ mavg_status mavg_workspace_bytes(const mavg_config *cfg, size_t *out_bytes);
 
 /* Algorithm 1, the two initialisation lines and the first "set w^j = w~": v <- 0, w^j <- w~_1
  * (the copies are skipped with defer_broadcast, see there).
- * Validates everything; on failure *out is NULL.  Enqueues the initialisation on the stream. */
+ * Validates everything; on failure *out is NULL.  Enqueues the initialisation on the stream.
+ * For an MLP handle on the tensor-core path whose P master copies together take at most half the
+ * L2, the call also raises the CUDA context's limit cudaLimitPersistingL2CacheSize to their size
+ * (capped by the device's maximum): the weight-gradient kernels then ask the L2 to keep the
+ * masters from one local step to the next instead of sending them through HBM.  The limit
+ * belongs to the calling process's context; mavg_destroy puts the previous value back. */
 mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_handle *out);
 
 /* Learner level of Algorithm 1 (inner loop over k): K SGD steps on all P replicas for the round
@@ -221,6 +226,11 @@ mavg_status mavg_get_profile(mavg_handle h, float *ms, int64_t *launches, int32_
 
 /* Waits for the stream; reports CUDA errors and a tripped device-side wait limit. */
 mavg_status mavg_sync(mavg_handle h);
+
+/* Waits for the stream, then returns every L2 line that this context asked to be kept (see
+ * mavg_create) to normal eviction; a no-op for handles that keep nothing.  For measurements that
+ * want a cold cache at the start of a round: lines kept this way survive an ordinary flush. */
+mavg_status mavg_cache_release(mavg_handle h);
 
 /* Message for the last failure on this handle ("" if none); with h == NULL, for the last failed
  * mavg_create / mavg_workspace_bytes of the calling thread.  Valid until the next call. */

@@ -21,7 +21,7 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams",
            "mavg_set_learner_momentum", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
-           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync", "mavg_last_error",
+           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync", "mavg_cache_release", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
@@ -97,6 +97,7 @@ def load_library():
                                              C.c_void_p]
     L.mavg_materialize_replicas.argtypes = [H]
     L.mavg_sync.argtypes = [H]
+    L.mavg_cache_release.argtypes = [H]
     L.mavg_last_error.argtypes = [H]
     L.mavg_last_error.restype = C.c_char_p
     L.mavg_destroy.argtypes = [H]
@@ -275,6 +276,10 @@ class Mavg:
 
     def sync(self):
         self._check(self.lib.mavg_sync(self.handle))
+
+    def l2_release(self):
+        """Wait for the stream and give up the L2 lines kept for the masters (cold-cache timing)."""
+        self._check(self.lib.mavg_cache_release(self.handle))
 
     def close(self):
         if getattr(self, "handle", None) is not None and self.handle:

@@ -262,6 +262,22 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
       delete c;
       return st;
     }
+    if (c->cfg.gemm_bf16 == 1 && masters_fit_l2(c)) {   // the tensor-core path
+      // Room in the L2 for the learners' masters (see mavg_create in mavg.h).  Without it the
+      // keep hints of the weight-gradient kernels have no effect; a refusal only costs speed.
+      int max_keep = 0;
+      size_t prev = 0;
+      const size_t want = (size_t)cfg->P * (size_t)buf->replica_stride * sizeof(float);
+      if (cudaDeviceGetAttribute(&max_keep, cudaDevAttrMaxPersistingL2CacheSize, dev) == cudaSuccess &&
+          max_keep > 0 && cudaDeviceGetLimit(&prev, cudaLimitPersistingL2CacheSize) == cudaSuccess &&
+          cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize,
+                             want < (size_t)max_keep ? want : (size_t)max_keep) == cudaSuccess) {
+        c->l2_keep = true;
+        c->l2_keep_prev = prev;
+      } else {
+        cudaGetLastError();
+      }
+    }
   }
   *out = c;
   return MAVG_OK;
@@ -456,8 +472,21 @@ const char* mavg_last_error(mavg_handle h) {
   return h->err.c_str();
 }
 
+mavg_status mavg_cache_release(mavg_handle h) {
+  CHECK_HANDLE(h);
+  CU(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  if (h->l2_keep) CU(h, cudaCtxResetPersistingL2Cache(), "L2 reset");
+  return MAVG_OK;
+}
+
 mavg_status mavg_destroy(mavg_handle h) {
   if (!h) return MAVG_OK;
+  if (h->l2_keep) {
+    cudaStreamSynchronize(h->stream);
+    cudaCtxResetPersistingL2Cache();
+    cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_keep_prev);
+    cudaGetLastError();
+  }
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_copy_fork) cudaEventDestroy(h->ev_copy_fork);
   if (h->ev_copy_done) cudaEventDestroy(h->ev_copy_done);

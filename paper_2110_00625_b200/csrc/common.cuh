@@ -129,12 +129,21 @@ struct mavg_ctx {
   int graph_schedule = 0;
   int graph_w16_cur = 0;      // state of the doubled bf16 copy after the recorded steps
   int64_t graph_nodes = 0;
+  // the context's persisting-L2 limit was raised for the masters (restored by mavg_destroy)
+  bool l2_keep = false;
+  size_t l2_keep_prev = 0;
   // mavg_round_host: the upload of v runs on a copy stream of its own, next to the local steps
   cudaStream_t s_copy = nullptr;
   cudaEvent_t ev_copy_fork = nullptr, ev_copy_done = nullptr;
 };
 
 namespace mavg {
+
+// All learners' fp32 masters together fit in half the L2: a step's weight-gradient kernels then
+// ask the L2 to keep them until the next step reads them again.
+inline bool masters_fit_l2(const mavg_ctx* c) {
+  return (size_t)c->cfg.P * (size_t)c->buf.replica_stride * sizeof(float) <= c->l2_bytes / 2;
+}
 
 // Momentum arguments of a local step; from_broadcast: the step starts from w^j = w~.
 inline MomArgs mom_args(const mavg_ctx* c, bool from_broadcast) {

@@ -185,6 +185,7 @@ WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs&
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
   g.w16_on_b = w.w16_on_b;
+  g.keep_w32 = c->l2_keep ? 1 : 0;
   g.gamma = c->cfg.local_lr;
   g.beta = mom.beta;
   g.read_u = mom.read_u;
@@ -246,6 +247,7 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
   g.w16_on_b = w.w16_on_b;
+  g.keep_w32 = c->l2_keep ? 1 : 0;
   g.gamma = c->cfg.local_lr;
   g.beta = mom.beta;
   g.read_u = mom.read_u;

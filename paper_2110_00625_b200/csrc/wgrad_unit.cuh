@@ -25,6 +25,14 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* s
       ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_3d_hint(const CUtensorMap* m, const void* src, int c0,
+                                                  int c1, int c2, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint"
+      " [%0, {%2, %3, %4}], [%1], %5;"
+      ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
@@ -47,6 +55,9 @@ struct WgradArgs {
   int slots;               // ring depth
   int a_bufs;              // 1 or 2 buffers for the dZ^T tile
   int w16_on_b;            // 1: the bf16 output tile is written over the slot's A^T slabs
+  int keep_w32;            // 1: master tiles are loaded and stored with the L2 evict-last hint
+                           //    (all learners' masters together fit in half the L2: they are
+                           //    read again one step later and should not go through HBM)
   float gamma;
   float beta;              // learner momentum (MOM)
   int read_u;              // 0: the stored u counts as zero and is not loaded
@@ -149,6 +160,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
     if (lane == 0) {
       uint32_t tile_ctr = tile_base, item_ctr = item_base;
       bool ok = true;
+      const uint64_t pol = l2_policy(g.keep_w32 != 0);
       for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
         int p, m0, nt0, nt;
         decode(item, p, m0, nt0, nt);
@@ -172,7 +184,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           const bool load_u = MOM && g.read_u;
           mbar_arrive_expect_tx(&sh.slot_full[s],
                                 (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0)));
-          tma_load_3d(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0);
+          tma_load_3d_hint(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0, pol);
           if (load_u) tma_load_3d(sl + kW32Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
             tma_load_3d(sl + b_off + (size_t)kb * (kBN * kBK * 2),
@@ -292,6 +304,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       // items whose tiles have all been handed to the TMA unit but may not have reached global
       // memory yet: (index after the item's last tile, learner); signalled kStoreLag tiles later
       int held = -1;          // slot whose stores are committed but not yet known to be read
+      const uint64_t pol = l2_policy(g.keep_w32 != 0);
       uint32_t pend_end[8];
       int pend_p[8];
       uint32_t ph = 0, pt = 0;
@@ -307,7 +320,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           }
           uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
-          tma_store_3d(&tm_w32, sl, i0, m0, p);
+          tma_store_3d_hint(&tm_w32, sl, i0, m0, p, pol);
           tma_store_3d(&tm_w16, sl + w16_off, i0, m0, p);
           if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes, i0, m0, p);
           tma_store_commit();

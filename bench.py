@@ -161,13 +161,13 @@ def run_reference(args):
 
 # DRAM read + write bytes per launch, averaged over the launches of a class in one local step of
 # the C2 workload, from the ncu capture summarised in profiles/step_kernels_c2.md (cold cache:
-# ncu flushes L2 before every kernel; in a running round most of this workload's 90 MB of state
-# stays in the 126 MB L2, so steady-state traffic is lower still).  Valid for the kernels as
+# ncu flushes L2 before every kernel; in a running round the fp32 masters stay in the L2 lines
+# set aside for them, so steady-state traffic is lower still: second table there).  Valid for the kernels as
 # captured; set an entry to None when its kernel changes.
 NCU_TRAFFIC_C2 = {
     # all layers' weight gradients (captured as the graph's two launches, layer 1 and layers 3 + 2)
-    "wgrad_sgd_gemm": 57.702656e6 + 21.394176e6 + 11.806976e6 + 0.007424e6,
-    "fwd_gemm": (31.498240e6 + 0.001536e6 + 5.325824e6) / 2,     # hidden layers 1 and 2
+    "wgrad_sgd_gemm": 57.703424e6 + 5.545216e6 + 11.806976e6 + 0.002560e6,
+    "fwd_gemm": (31.497728e6 + 0.010496e6 + 5.324800e6) / 2,     # hidden layers 1 and 2
     "dgrad_gemm": 6.381056e6,
 }
 

@@ -138,7 +138,9 @@ mavg_status mavg_workspace_bytes(const mavg_config *cfg, size_t *out_bytes);
  * L2, the call also raises the CUDA context's limit cudaLimitPersistingL2CacheSize to their size
  * (capped by the device's maximum): the weight-gradient kernels then ask the L2 to keep the
  * masters from one local step to the next instead of sending them through HBM.  The limit
- * belongs to the calling process's context; mavg_destroy puts the previous value back. */
+ * belongs to the calling process's context: it follows the largest request among the live
+ * handles on the device (never below the value found), and the mavg_destroy of the last of them
+ * puts the previous value back. */
 mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_handle *out);
 
 /* Learner level of Algorithm 1 (inner loop over k): K SGD steps on all P replicas for the round

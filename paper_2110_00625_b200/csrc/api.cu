@@ -4,6 +4,9 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <set>
 #include <new>
 
 #include "common.cuh"
@@ -182,6 +185,60 @@ namespace mavg {
 void set_thread_error(const std::string& msg) { g_create_error = msg; }
 }  // namespace mavg
 
+namespace {
+
+// The persisting-L2 limit belongs to the device's context, which every handle of the process on
+// that device shares: it is raised to the largest request among the live handles and put back to
+// what it was when the last of them goes.
+struct KeepState {
+  std::multiset<size_t> wants;
+  size_t prev = 0;
+};
+std::mutex g_keep_mu;
+std::map<int, KeepState> g_keep;
+
+bool keep_apply(int dev, const KeepState& k) {
+  int max_keep = 0;
+  if (cudaDeviceGetAttribute(&max_keep, cudaDevAttrMaxPersistingL2CacheSize, dev) != cudaSuccess ||
+      max_keep <= 0)
+    return false;
+  // never below what the context had before the first handle asked
+  const size_t want = *k.wants.rbegin() > k.prev ? *k.wants.rbegin() : k.prev;
+  return cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize,
+                            want < (size_t)max_keep ? want : (size_t)max_keep) == cudaSuccess;
+}
+
+bool keep_acquire(int dev, size_t want) {
+  std::lock_guard<std::mutex> lock(g_keep_mu);
+  KeepState& k = g_keep[dev];
+  if (k.wants.empty() && cudaDeviceGetLimit(&k.prev, cudaLimitPersistingL2CacheSize) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  k.wants.insert(want);
+  if (keep_apply(dev, k)) return true;
+  cudaGetLastError();
+  k.wants.erase(k.wants.find(want));
+  return false;
+}
+
+void keep_release(int dev, size_t want) {
+  std::lock_guard<std::mutex> lock(g_keep_mu);
+  KeepState& k = g_keep[dev];
+  auto it = k.wants.find(want);
+  if (it == k.wants.end()) return;
+  k.wants.erase(it);
+  if (k.wants.empty()) {
+    cudaCtxResetPersistingL2Cache();
+    cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, k.prev);
+  } else {
+    keep_apply(dev, k);
+  }
+  cudaGetLastError();
+}
+
+}  // namespace
+
 extern "C" {
 
 mavg_status mavg_workspace_bytes(const mavg_config* cfg, size_t* out_bytes) {
@@ -265,17 +322,11 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
     if (c->cfg.gemm_bf16 == 1 && masters_fit_l2(c)) {   // the tensor-core path
       // Room in the L2 for the learners' masters (see mavg_create in mavg.h).  Without it the
       // keep hints of the weight-gradient kernels have no effect; a refusal only costs speed.
-      int max_keep = 0;
-      size_t prev = 0;
       const size_t want = (size_t)cfg->P * (size_t)buf->replica_stride * sizeof(float);
-      if (cudaDeviceGetAttribute(&max_keep, cudaDevAttrMaxPersistingL2CacheSize, dev) == cudaSuccess &&
-          max_keep > 0 && cudaDeviceGetLimit(&prev, cudaLimitPersistingL2CacheSize) == cudaSuccess &&
-          cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize,
-                             want < (size_t)max_keep ? want : (size_t)max_keep) == cudaSuccess) {
+      if (keep_acquire(dev, want)) {
         c->l2_keep = true;
-        c->l2_keep_prev = prev;
-      } else {
-        cudaGetLastError();
+        c->l2_keep_want = want;
+        c->device = dev;
       }
     }
   }
@@ -483,9 +534,7 @@ mavg_status mavg_destroy(mavg_handle h) {
   if (!h) return MAVG_OK;
   if (h->l2_keep) {
     cudaStreamSynchronize(h->stream);
-    cudaCtxResetPersistingL2Cache();
-    cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_keep_prev);
-    cudaGetLastError();
+    keep_release(h->device, h->l2_keep_want);
   }
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_copy_fork) cudaEventDestroy(h->ev_copy_fork);

@@ -129,9 +129,10 @@ struct mavg_ctx {
   int graph_schedule = 0;
   int graph_w16_cur = 0;      // state of the doubled bf16 copy after the recorded steps
   int64_t graph_nodes = 0;
-  // the context's persisting-L2 limit was raised for the masters (restored by mavg_destroy)
+  // this handle holds a request on the context's persisting-L2 limit (given up by mavg_destroy)
   bool l2_keep = false;
-  size_t l2_keep_prev = 0;
+  size_t l2_keep_want = 0;
+  int device = 0;
   // mavg_round_host: the upload of v runs on a copy stream of its own, next to the local steps
   cudaStream_t s_copy = nullptr;
   cudaEvent_t ev_copy_fork = nullptr, ev_copy_done = nullptr;

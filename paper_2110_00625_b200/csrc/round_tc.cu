@@ -77,6 +77,7 @@ struct RoundParams {
   const float* global_w;
   int64_t rep_stride;
   float gamma;
+  int keep_w32;          // master tiles carry the L2 keep hint (see WgradArgs)
   int* counters;              // [CNT_KINDS][kRoundMaxLayers + 1][P], zero at launch
   int* status;
 };
@@ -375,6 +376,7 @@ k_mlp_round(const __grid_constant__ RoundParams rp) {
     g.items = P * y.w_m_tiles * y.w_n_chunks;
     g.slots = rp.w_slots; g.a_bufs = rp.w_a_bufs; g.w16_on_b = rp.w_on_b;
     g.gamma = rp.gamma;
+    g.keep_w32 = rp.keep_w32;
     g.status = rp.status;
     if (vb >= g.items) return;             // nothing of this layer falls to this block
     WgDeps dep{&rp, l, k};
@@ -583,6 +585,7 @@ cudaError_t tc_round_launch(mavg_ctx* c, int64_t round) {
   rp->replicas = c->buf.replicas; rp->global_w = c->buf.global_w;
   rp->rep_stride = c->buf.replica_stride;
   rp->gamma = cfg.local_lr;
+  rp->keep_w32 = c->l2_keep ? 1 : 0;
   rp->counters = (int*)(ws + t.round_ctr);
   rp->status = (int*)ws_ptr(c, c->ws.status);
   cudaError_t e = cudaMemsetAsync(rp->counters, 0, t.round_ctr_bytes, c->stream);

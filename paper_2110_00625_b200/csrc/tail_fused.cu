@@ -20,6 +20,7 @@ namespace {
 constexpr int kRows = 16;        // batch rows per block
 constexpr int kThreads = 256;
 constexpr int kMaxC = 32;
+static_assert(kThreads == 16 * kRows, "the softmax phase gives every row 16 lanes");
 
 struct TailArgs {
   const __nv_bfloat16* a_bm;     // A_{L-1} [P, B, in]
@@ -50,7 +51,7 @@ __global__ void __launch_bounds__(kThreads)
 k_last_layer_fused(const TailArgs g) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __shared__ float z[kRows][kMaxC + 1];     // logits, then unrounded dZ
-  __shared__ float zq[kRows][kMaxC + 1];    // dZ rounded to bf16 values
+  __shared__ __align__(16) float zq[kMaxC][kRows];   // dZ rounded to bf16 values, class-major
   __shared__ float row_loss[kRows];
   __shared__ float bias_s[kMaxC];
   __shared__ int label_s[kRows];
@@ -76,40 +77,75 @@ k_last_layer_fused(const TailArgs g) {
   }
   __syncthreads();
 
-  // forward: warp w takes rows 2w and 2w + 1; lanes split the contraction, two elements at a time
-  for (int rr = 0; rr < 2; ++rr) {
-    const int r = 2 * warp + rr;
-    const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)r * in);
-    for (int c = 0; c < C; ++c) {
-      const uint32_t* wrow = reinterpret_cast<const uint32_t*>(Ws + (size_t)c * in);
-      float acc = 0.f;
+  // forward: warp w takes rows 2w and 2w + 1; lanes split the contraction, two elements at a time.
+  // Two classes per pass for both rows: four independent chains, each the same sum in the same
+  // order as one chain at a time would give.
+  {
+    const int ra = 2 * warp, rb = ra + 1;
+    const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)ra * in);
+    const uint32_t* brow = reinterpret_cast<const uint32_t*>(As + (size_t)rb * in);
+    for (int c = 0; c < C; c += 2) {
+      const int c1 = c + 1 < C ? c + 1 : c;
+      const uint32_t* wrow0 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c * in);
+      const uint32_t* wrow1 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c1 * in);
+      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
       for (int k2 = lane; k2 < in / 2; k2 += 32) {
-        const uint32_t a = arow[k2], w = wrow[k2];
-        acc = fmaf(bf_lo(a), bf_lo(w), acc);
-        acc = fmaf(bf_hi(a), bf_hi(w), acc);
+        const uint32_t xa = arow[k2], xb = brow[k2], w0 = wrow0[k2], w1 = wrow1[k2];
+        a0 = fmaf(bf_lo(xa), bf_lo(w0), a0);
+        a1 = fmaf(bf_lo(xa), bf_lo(w1), a1);
+        b0 = fmaf(bf_lo(xb), bf_lo(w0), b0);
+        b1 = fmaf(bf_lo(xb), bf_lo(w1), b1);
+        a0 = fmaf(bf_hi(xa), bf_hi(w0), a0);
+        a1 = fmaf(bf_hi(xa), bf_hi(w1), a1);
+        b0 = fmaf(bf_hi(xb), bf_hi(w0), b0);
+        b1 = fmaf(bf_hi(xb), bf_hi(w1), b1);
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) z[r][c] = acc + bias_s[c];
+      for (int o = 16; o > 0; o >>= 1) {
+        a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+        a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+        b0 += __shfl_xor_sync(0xffffffffu, b0, o);
+        b1 += __shfl_xor_sync(0xffffffffu, b1, o);
+      }
+      if (lane == 0) {
+        z[ra][c] = a0 + bias_s[c];
+        z[rb][c] = b0 + bias_s[c];
+        if (c1 != c) {
+          z[ra][c1] = a1 + bias_s[c1];
+          z[rb][c1] = b1 + bias_s[c1];
+        }
+      }
     }
   }
   __syncthreads();
 
-  // softmax cross-entropy, one thread per row
-  if (tid < kRows) {
-    const int r = tid;
+  // softmax cross-entropy: 16 lanes per row (kThreads = 16 rows x 16 lanes), lane l holds the
+  // classes l and l + 16; maximum and sum of exponentials by butterflies inside the 16 lanes
+  {
+    const int r = tid >> 4, l = tid & 15;
     const int yb = label_s[r];
-    float mx = z[r][0];
-    for (int c = 1; c < C; ++c) mx = fmaxf(mx, z[r][c]);
-    float se = 0.f;
-    for (int c = 0; c < C; ++c) se += __expf(z[r][c] - mx);
+    const bool h0 = l < C, h1 = l + 16 < C;
+    const float v0 = h0 ? z[r][l] : -INFINITY, v1 = h1 ? z[r][l + 16] : -INFINITY;
+    float mx = fmaxf(v0, v1);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = (h0 ? __expf(v0 - mx) : 0.f) + (h1 ? __expf(v1 - mx) : 0.f);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
     const float lse = mx + __logf(se);
-    row_loss[r] = lse - z[r][yb];
     const float inv_b = 1.0f / (float)B;
-    for (int c = 0; c < C; ++c) {
-      const float gr = (__expf(z[r][c] - lse) - (c == yb ? 1.f : 0.f)) * inv_b;
-      z[r][c] = gr;
-      zq[r][c] = __bfloat162float(__float2bfloat16_rn(gr));
+    __syncwarp();                       // every lane of the row has read its logits
+    if (h0) {
+      if (l == yb) row_loss[r] = lse - v0;
+      const float gr = (__expf(v0 - lse) - (l == yb ? 1.f : 0.f)) * inv_b;
+      z[r][l] = gr;
+      zq[l][r] = __bfloat162float(__float2bfloat16_rn(gr));
+    }
+    if (h1) {
+      if (l + 16 == yb) row_loss[r] = lse - v1;
+      const float gr = (__expf(v1 - lse) - (l + 16 == yb ? 1.f : 0.f)) * inv_b;
+      z[r][l + 16] = gr;
+      zq[l + 16][r] = __bfloat162float(__float2bfloat16_rn(gr));
     }
   }
   __syncthreads();
@@ -138,35 +174,54 @@ k_last_layer_fused(const TailArgs g) {
     part[in + C] = s;
   }
 
-  // data gradient through the layer, masked by the activation below; thread per input column
+  // data gradient through the layer, masked by the activation below; a thread takes the input
+  // columns k and k + kThreads together (two independent sets of accumulators)
   if (g.dzp_bm) {
-    for (int k = tid; k < in; k += kThreads) {
-      float acc[kRows];
+    for (int k = tid; k < in; k += 2 * kThreads) {
+      const bool two = k + kThreads < in;
+      const int k1 = two ? k + kThreads : k;
+      float acc[kRows], bcc[kRows];
 #pragma unroll
-      for (int r = 0; r < kRows; ++r) acc[r] = 0.f;
+      for (int r = 0; r < kRows; ++r) acc[r] = bcc[r] = 0.f;
       for (int c = 0; c < C; ++c) {
         const float wv = __bfloat162float(Ws[(size_t)c * in + k]);
+        const float wu = __bfloat162float(Ws[(size_t)c * in + k1]);
+        const float4* zc = reinterpret_cast<const float4*>(zq[c]);
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) acc[r] = fmaf(zq[r][c], wv, acc[r]);
+        for (int r4 = 0; r4 < kRows / 4; ++r4) {
+          const float4 q4 = zc[r4];
+          acc[4 * r4 + 0] = fmaf(q4.x, wv, acc[4 * r4 + 0]);
+          acc[4 * r4 + 1] = fmaf(q4.y, wv, acc[4 * r4 + 1]);
+          acc[4 * r4 + 2] = fmaf(q4.z, wv, acc[4 * r4 + 2]);
+          acc[4 * r4 + 3] = fmaf(q4.w, wv, acc[4 * r4 + 3]);
+          bcc[4 * r4 + 0] = fmaf(q4.x, wu, bcc[4 * r4 + 0]);
+          bcc[4 * r4 + 1] = fmaf(q4.y, wu, bcc[4 * r4 + 1]);
+          bcc[4 * r4 + 2] = fmaf(q4.z, wu, bcc[4 * r4 + 2]);
+          bcc[4 * r4 + 3] = fmaf(q4.w, wu, bcc[4 * r4 + 3]);
+        }
       }
-      float colsum = 0.f;
-      uint32_t w[8];
+      auto finish = [&](float (&a)[kRows], int kk) {
+        float colsum = 0.f;
+        uint32_t w[8];
 #pragma unroll
-      for (int r = 0; r < kRows; ++r) {
-        const bool live = __bfloat162float(As[(size_t)r * in + k]) > 0.f;     // ReLU'(0) = 0
-        acc[r] = live ? acc[r] : 0.f;
-        colsum += acc[r];
-        g.dzp_bm[((size_t)p * B + r0 + r) * in + k] = __float2bfloat16_rn(acc[r]);
-      }
+        for (int r = 0; r < kRows; ++r) {
+          const bool live = __bfloat162float(As[(size_t)r * in + kk]) > 0.f;     // ReLU'(0) = 0
+          a[r] = live ? a[r] : 0.f;
+          colsum += a[r];
+          g.dzp_bm[((size_t)p * B + r0 + r) * in + kk] = __float2bfloat16_rn(a[r]);
+        }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
-        w[j] = *reinterpret_cast<uint32_t*>(&h2);
-      }
-      uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + k) * B + r0);
-      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-      part[k] = colsum;
+        for (int j = 0; j < 8; ++j) {
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(a[2 * j], a[2 * j + 1]);
+          w[j] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + kk) * B + r0);
+        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        part[kk] = colsum;
+      };
+      finish(acc, k);
+      if (two) finish(bcc, k1);
     }
   }
 }

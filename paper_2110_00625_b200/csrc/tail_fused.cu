@@ -18,9 +18,9 @@ namespace mavg {
 namespace {
 
 constexpr int kRows = 16;        // batch rows per block
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kMaxC = 32;
-static_assert(kThreads == 16 * kRows, "the softmax phase gives every row 16 lanes");
+static_assert(kThreads == 32 * kRows && kMaxC <= 32, "one warp per batch row, one lane per class");
 
 struct TailArgs {
   const __nv_bfloat16* a_bm;     // A_{L-1} [P, B, in]
@@ -46,7 +46,7 @@ struct TailArgs {
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
 
-// grid (B / 16, P), 256 threads.  Dynamic shared memory: W [C, in] bf16, A [16, in] bf16.
+// grid (B / 16, P), 512 threads (a warp per batch row).  Dynamic shared memory: W [C, in] bf16, A [16, in] bf16.
 __global__ void __launch_bounds__(kThreads)
 k_last_layer_fused(const TailArgs g) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -77,75 +77,66 @@ k_last_layer_fused(const TailArgs g) {
   }
   __syncthreads();
 
-  // forward: warp w takes rows 2w and 2w + 1; lanes split the contraction, two elements at a time.
-  // Two classes per pass for both rows: four independent chains, each the same sum in the same
-  // order as one chain at a time would give.
+  // forward: warp w takes row w; lanes split the contraction, two elements at a time.  Four
+  // classes per pass: four independent chains, each the same sum in the same order as one chain
+  // at a time would give.
   {
-    const int ra = 2 * warp, rb = ra + 1;
-    const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)ra * in);
-    const uint32_t* brow = reinterpret_cast<const uint32_t*>(As + (size_t)rb * in);
-    for (int c = 0; c < C; c += 2) {
-      const int c1 = c + 1 < C ? c + 1 : c;
+    const int r = warp;
+    const uint32_t* arow = reinterpret_cast<const uint32_t*>(As + (size_t)r * in);
+    for (int c = 0; c < C; c += 4) {
+      const int c1 = min(c + 1, C - 1), c2 = min(c + 2, C - 1), c3 = min(c + 3, C - 1);
       const uint32_t* wrow0 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c * in);
       const uint32_t* wrow1 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c1 * in);
-      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+      const uint32_t* wrow2 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c2 * in);
+      const uint32_t* wrow3 = reinterpret_cast<const uint32_t*>(Ws + (size_t)c3 * in);
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       for (int k2 = lane; k2 < in / 2; k2 += 32) {
-        const uint32_t xa = arow[k2], xb = brow[k2], w0 = wrow0[k2], w1 = wrow1[k2];
-        a0 = fmaf(bf_lo(xa), bf_lo(w0), a0);
-        a1 = fmaf(bf_lo(xa), bf_lo(w1), a1);
-        b0 = fmaf(bf_lo(xb), bf_lo(w0), b0);
-        b1 = fmaf(bf_lo(xb), bf_lo(w1), b1);
-        a0 = fmaf(bf_hi(xa), bf_hi(w0), a0);
-        a1 = fmaf(bf_hi(xa), bf_hi(w1), a1);
-        b0 = fmaf(bf_hi(xb), bf_hi(w0), b0);
-        b1 = fmaf(bf_hi(xb), bf_hi(w1), b1);
+        const uint32_t x = arow[k2], w0 = wrow0[k2], w1 = wrow1[k2], w2 = wrow2[k2], w3 = wrow3[k2];
+        a0 = fmaf(bf_lo(x), bf_lo(w0), a0);
+        a1 = fmaf(bf_lo(x), bf_lo(w1), a1);
+        a2 = fmaf(bf_lo(x), bf_lo(w2), a2);
+        a3 = fmaf(bf_lo(x), bf_lo(w3), a3);
+        a0 = fmaf(bf_hi(x), bf_hi(w0), a0);
+        a1 = fmaf(bf_hi(x), bf_hi(w1), a1);
+        a2 = fmaf(bf_hi(x), bf_hi(w2), a2);
+        a3 = fmaf(bf_hi(x), bf_hi(w3), a3);
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         a0 += __shfl_xor_sync(0xffffffffu, a0, o);
         a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-        b0 += __shfl_xor_sync(0xffffffffu, b0, o);
-        b1 += __shfl_xor_sync(0xffffffffu, b1, o);
+        a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+        a3 += __shfl_xor_sync(0xffffffffu, a3, o);
       }
       if (lane == 0) {
-        z[ra][c] = a0 + bias_s[c];
-        z[rb][c] = b0 + bias_s[c];
-        if (c1 != c) {
-          z[ra][c1] = a1 + bias_s[c1];
-          z[rb][c1] = b1 + bias_s[c1];
-        }
+        z[r][c] = a0 + bias_s[c];
+        if (c + 1 < C) z[r][c + 1] = a1 + bias_s[c + 1];
+        if (c + 2 < C) z[r][c + 2] = a2 + bias_s[c + 2];
+        if (c + 3 < C) z[r][c + 3] = a3 + bias_s[c + 3];
       }
     }
   }
   __syncthreads();
 
-  // softmax cross-entropy: 16 lanes per row (kThreads = 16 rows x 16 lanes), lane l holds the
-  // classes l and l + 16; maximum and sum of exponentials by butterflies inside the 16 lanes
+  // softmax cross-entropy: warp r takes row r, lane l class l; maximum and sum of exponentials
+  // by butterflies over the warp
   {
-    const int r = tid >> 4, l = tid & 15;
+    const int r = warp, l = lane;
     const int yb = label_s[r];
-    const bool h0 = l < C, h1 = l + 16 < C;
-    const float v0 = h0 ? z[r][l] : -INFINITY, v1 = h1 ? z[r][l + 16] : -INFINITY;
-    float mx = fmaxf(v0, v1);
+    const bool h = l < C;
+    const float v = h ? z[r][l] : -INFINITY;
+    float mx = v;
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float se = (h0 ? __expf(v0 - mx) : 0.f) + (h1 ? __expf(v1 - mx) : 0.f);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = h ? __expf(v - mx) : 0.f;
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
     const float lse = mx + __logf(se);
-    const float inv_b = 1.0f / (float)B;
-    __syncwarp();                       // every lane of the row has read its logits
-    if (h0) {
-      if (l == yb) row_loss[r] = lse - v0;
-      const float gr = (__expf(v0 - lse) - (l == yb ? 1.f : 0.f)) * inv_b;
+    if (h) {
+      if (l == yb) row_loss[r] = lse - v;
+      const float gr = (__expf(v - lse) - (l == yb ? 1.f : 0.f)) * (1.0f / (float)B);
       z[r][l] = gr;
       zq[l][r] = __bfloat162float(__float2bfloat16_rn(gr));
-    }
-    if (h1) {
-      if (l + 16 == yb) row_loss[r] = lse - v1;
-      const float gr = (__expf(v1 - lse) - (l + 16 == yb ? 1.f : 0.f)) * inv_b;
-      z[r][l + 16] = gr;
-      zq[l + 16][r] = __bfloat162float(__float2bfloat16_rn(gr));
     }
   }
   __syncthreads();
@@ -174,18 +165,14 @@ k_last_layer_fused(const TailArgs g) {
     part[in + C] = s;
   }
 
-  // data gradient through the layer, masked by the activation below; a thread takes the input
-  // columns k and k + kThreads together (two independent sets of accumulators)
+  // data gradient through the layer, masked by the activation below; thread per input column
   if (g.dzp_bm) {
-    for (int k = tid; k < in; k += 2 * kThreads) {
-      const bool two = k + kThreads < in;
-      const int k1 = two ? k + kThreads : k;
-      float acc[kRows], bcc[kRows];
+    for (int k = tid; k < in; k += kThreads) {
+      float acc[kRows];
 #pragma unroll
-      for (int r = 0; r < kRows; ++r) acc[r] = bcc[r] = 0.f;
+      for (int r = 0; r < kRows; ++r) acc[r] = 0.f;
       for (int c = 0; c < C; ++c) {
         const float wv = __bfloat162float(Ws[(size_t)c * in + k]);
-        const float wu = __bfloat162float(Ws[(size_t)c * in + k1]);
         const float4* zc = reinterpret_cast<const float4*>(zq[c]);
 #pragma unroll
         for (int r4 = 0; r4 < kRows / 4; ++r4) {
@@ -194,34 +181,26 @@ k_last_layer_fused(const TailArgs g) {
           acc[4 * r4 + 1] = fmaf(q4.y, wv, acc[4 * r4 + 1]);
           acc[4 * r4 + 2] = fmaf(q4.z, wv, acc[4 * r4 + 2]);
           acc[4 * r4 + 3] = fmaf(q4.w, wv, acc[4 * r4 + 3]);
-          bcc[4 * r4 + 0] = fmaf(q4.x, wu, bcc[4 * r4 + 0]);
-          bcc[4 * r4 + 1] = fmaf(q4.y, wu, bcc[4 * r4 + 1]);
-          bcc[4 * r4 + 2] = fmaf(q4.z, wu, bcc[4 * r4 + 2]);
-          bcc[4 * r4 + 3] = fmaf(q4.w, wu, bcc[4 * r4 + 3]);
         }
       }
-      auto finish = [&](float (&a)[kRows], int kk) {
-        float colsum = 0.f;
-        uint32_t w[8];
+      float colsum = 0.f;
+      uint32_t w[8];
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-          const bool live = __bfloat162float(As[(size_t)r * in + kk]) > 0.f;     // ReLU'(0) = 0
-          a[r] = live ? a[r] : 0.f;
-          colsum += a[r];
-          g.dzp_bm[((size_t)p * B + r0 + r) * in + kk] = __float2bfloat16_rn(a[r]);
-        }
+      for (int r = 0; r < kRows; ++r) {
+        const bool live = __bfloat162float(As[(size_t)r * in + k]) > 0.f;     // ReLU'(0) = 0
+        acc[r] = live ? acc[r] : 0.f;
+        colsum += acc[r];
+        g.dzp_bm[((size_t)p * B + r0 + r) * in + k] = __float2bfloat16_rn(acc[r]);
+      }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(a[2 * j], a[2 * j + 1]);
-          w[j] = *reinterpret_cast<uint32_t*>(&h2);
-        }
-        uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + kk) * B + r0);
-        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-        part[kk] = colsum;
-      };
-      finish(acc, k);
-      if (two) finish(bcc, k1);
+      for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t*>(&h2);
+      }
+      uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + k) * B + r0);
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      part[k] = colsum;
     }
   }
 }

@@ -2,7 +2,7 @@
 // cross-entropy loss, dZ_L, the data gradient through the layer (with the ReLU mask of the layer
 // below) and the two bias steps that hang on them.  With at most 32 classes these products are a
 // few hundred thousand multiply-adds per learner -- far too small for a tensor-core tile each to
-// pay for its launch and its tail -- so one block takes 16 batch rows of one learner through the
+// pay for its launch and its tail -- so one block takes 8 batch rows of one learner through the
 // whole sequence with the operands in shared memory:
 //   z[b, c]      = sum_k A[b, k] W[c, k] + bias[c]                  (bf16 operands, fp32 sums)
 //   loss_b       = logsumexp(z_b) - z_b[y_b];   dZ[b, c] = (softmax(z_b)[c] - [c == y_b]) / B
@@ -17,8 +17,8 @@
 namespace mavg {
 namespace {
 
-constexpr int kRows = 16;        // batch rows per block
-constexpr int kThreads = 512;
+constexpr int kRows = 8;         // batch rows per block (a multiple of 8: 16-byte transposed stores)
+constexpr int kThreads = 256;
 constexpr int kMaxC = 32;
 static_assert(kThreads == 32 * kRows && kMaxC <= 32, "one warp per batch row, one lane per class");
 
@@ -46,7 +46,7 @@ struct TailArgs {
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
 
-// grid (B / 16, P), 512 threads (a warp per batch row).  Dynamic shared memory: W [C, in] bf16, A [16, in] bf16.
+// grid (B / kRows, P), a warp per batch row.  Dynamic shared memory: W [C, in] bf16, A [kRows, in] bf16.
 __global__ void __launch_bounds__(kThreads)
 k_last_layer_fused(const TailArgs g) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -142,21 +142,21 @@ k_last_layer_fused(const TailArgs g) {
   __syncthreads();
 
   float* part = g.part + ((size_t)p * nblk + blk) * (in + C + 1);
-  // dZ_L transposed: class c, this block's 16 rows (32 contiguous bytes); partial bias gradient
+  // dZ_L transposed: class c, this block's rows (contiguous, 16 bytes per 8 rows); partial bias gradient
   if (tid < C) {
     const int c = tid;
-    uint32_t w[8];
+    uint32_t w[kRows / 2];
     float s = 0.f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < kRows / 2; ++j) {
       __nv_bfloat162 h2 = __floats2bfloat162_rn(z[2 * j][c], z[2 * j + 1][c]);
       w[j] = *reinterpret_cast<uint32_t*>(&h2);
       s += z[2 * j][c];
       s += z[2 * j + 1][c];
     }
     uint4* dst = reinterpret_cast<uint4*>(g.dz_t + ((size_t)p * C + c) * B + r0);
-    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+#pragma unroll
+    for (int v = 0; v < kRows / 8; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
     part[in + c] = s;
   }
   if (tid == kThreads - 1) {
@@ -184,7 +184,7 @@ k_last_layer_fused(const TailArgs g) {
         }
       }
       float colsum = 0.f;
-      uint32_t w[8];
+      uint32_t w[kRows / 2];
 #pragma unroll
       for (int r = 0; r < kRows; ++r) {
         const bool live = __bfloat162float(As[(size_t)r * in + k]) > 0.f;     // ReLU'(0) = 0
@@ -193,13 +193,13 @@ k_last_layer_fused(const TailArgs g) {
         g.dzp_bm[((size_t)p * B + r0 + r) * in + k] = __float2bfloat16_rn(acc[r]);
       }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < kRows / 2; ++j) {
         __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
         w[j] = *reinterpret_cast<uint32_t*>(&h2);
       }
       uint4* dst = reinterpret_cast<uint4*>(g.dzp_mb + ((size_t)p * in + k) * B + r0);
-      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+#pragma unroll
+      for (int v = 0; v < kRows / 8; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
       part[k] = colsum;
     }
   }

@@ -68,12 +68,25 @@ k_last_layer_fused(const TailArgs g) {
   if (tid < C) bias_s[tid] = bias_in[g.b_off + tid];
   if (tid >= 32 && tid < 32 + kRows) label_s[tid - 32] = g.labels[(size_t)p * B + r0 + tid - 32];
   {
+    // W and the rows as one list of 16-byte pieces; a thread has up to six loads in flight before
+    // it stores the first (written as a plain copy loop, each load would wait for the store before)
     const uint4* wsrc = reinterpret_cast<const uint4*>(g.w16 + (size_t)p * g.w16_stride);
-    uint4* wdst = reinterpret_cast<uint4*>(Ws);
-    for (int i = tid; i < C * in / 8; i += kThreads) wdst[i] = wsrc[i];
     const uint4* asrc = reinterpret_cast<const uint4*>(g.a_bm + ((size_t)p * B + r0) * in);
-    uint4* adst = reinterpret_cast<uint4*>(As);
-    for (int i = tid; i < kRows * in / 8; i += kThreads) adst[i] = asrc[i];
+    uint4* dst = reinterpret_cast<uint4*>(Ws);            // A follows W in shared memory
+    const int nw = C * in / 8, total = nw + kRows * in / 8;
+    for (int i0 = tid; i0 < total; i0 += 6 * kThreads) {
+      uint4 v[6];
+#pragma unroll
+      for (int j = 0; j < 6; ++j) {
+        const int i = i0 + j * kThreads;
+        if (i < total) v[j] = i < nw ? wsrc[i] : asrc[i - nw];
+      }
+#pragma unroll
+      for (int j = 0; j < 6; ++j) {
+        const int i = i0 + j * kThreads;
+        if (i < total) dst[i] = v[j];
+      }
+    }
   }
   __syncthreads();
 

@@ -11,7 +11,10 @@ What pins each oracle function (tests/test_oracle_pins.py):
                           kurtosis 2.7 of the four-lane sum; range
   bf16 rounding           torch's float32 -> bfloat16 conversion on every upper half-word
   mlp_loss_grad           torch.autograd in float64 (fp32 mode); central differences; ln(C) at
-                          zero weights; bf16 mode = fp32 mode on inputs that are bf16-exact
+                          zero weights; bf16 mode: an independent float64 restatement that applies
+                          torch's bf16 conversion to W, activations and dZ where the products read
+                          them (leaving any one rounding out is detected), bias gradient from the
+                          unrounded dZ
   meta_update             mu = 0 is K-AVG (plain mean); identical replicas; the auxiliary
                           sequence z_n; unrolled momentum sum by brute force; first round
   local_steps + round     closed-form two-term recurrence on a diagonal quadratic; P=K=1, mu=0 is

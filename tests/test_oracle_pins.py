@@ -218,6 +218,94 @@ def test_mlp_bf16_mode(oracle):
     assert np.abs(ga - gb).max() < 2.0 ** -8 * np.abs(ga).max()
 
 
+def _q_torch(a):
+    """fp32 -> bf16 -> fp32 through torch's conversion (round to nearest even), as float64."""
+    t = torch.tensor(np.asarray(a, dtype=np.float32))
+    return t.to(torch.bfloat16).to(torch.float32).numpy().astype(np.float64)
+
+
+def _mlp_bf16_restated(dims, w, X, y, drop=None):
+    """The bf16-operand minibatch gradient written out again in numpy float64: every operand of a
+    matrix product (weights, activations, dZ) is passed through torch's bf16 conversion at the
+    place the workload statement puts it; the bias add, ReLU, softmax, dZ_L and the bias gradient
+    use unrounded values.  Stored quantities (pre-activations, dZ) are fp32 like the oracle's.
+    drop names ONE rounding to leave out (None: the statement itself) -- used to show that each
+    rounding moves the result far beyond the comparison tolerance."""
+    def q(a, name):
+        return np.asarray(a, dtype=np.float64) if drop == name else _q_torch(a)
+    L, B = len(dims) - 1, len(y)
+    Ws, bs, off = [], [], 0
+    for l in range(L):
+        Ws.append(w[off:off + dims[l + 1] * dims[l]].reshape(dims[l + 1], dims[l])); off += Ws[-1].size
+        bs.append(w[off:off + dims[l + 1]].astype(np.float64)); off += dims[l + 1]
+    act = [q(X, "x")]
+    zs = [None]
+    for l in range(1, L + 1):
+        z = (act[l - 1] @ q(Ws[l - 1], "w_fwd").T + bs[l - 1]).astype(np.float32)
+        zs.append(z)
+        act.append(q(np.maximum(z, 0), "act") if l < L else z.astype(np.float64))
+    zL = zs[L].astype(np.float64)
+    lse = np.log(np.exp(zL - zL.max(1, keepdims=True)).sum(1)) + zL.max(1)
+    loss = float(np.mean(lse - zL[np.arange(B), y]))
+    onehot = np.eye(dims[-1])[y]
+    dz = ((np.exp(zL - lse[:, None]) - onehot) / B).astype(np.float32)
+    gW, gb = [None] * L, [None] * L
+    for l in range(L, 0, -1):
+        gb[l - 1] = dz.astype(np.float64).sum(0)                       # from the unrounded dZ
+        gW[l - 1] = q(dz, "dz_wgrad").T @ act[l - 1]
+        if l > 1:
+            da = q(dz, "dz_dgrad") @ q(Ws[l - 1], "w_dgrad")
+            dz = np.where(zs[l - 1] > 0, da, 0.0).astype(np.float32)   # ReLU'(0) = 0
+    grad = np.concatenate([np.concatenate([gW[l].reshape(-1), gb[l]]) for l in range(L)])
+    return loss, grad
+
+
+@pytest.mark.parametrize("dims,B", [([16, 24, 5], 8), ([24, 16, 8, 4], 12)])
+def test_mlp_bf16_operand_rounding_restated(oracle, dims, B):
+    # Which operands the bf16 mode rounds, and where, pinned by an independent restatement that
+    # calls torch's conversion explicitly.  Inputs are generic fp32 values (not bf16-exact), so
+    # that every rounding matters.
+    r = np.random.default_rng(11)
+    n = oracle.mlp_param_count(dims)
+    w = (0.4 * r.standard_normal(n)).astype(np.float32)
+    X = r.standard_normal((B, dims[0])).astype(np.float32)
+    y = r.integers(0, dims[-1], B).astype(np.int32)
+    loss, grad = oracle.mlp_loss_grad(dims, w, X, y, bf16=True)
+    want_loss, want = _mlp_bf16_restated(dims, w, X, y)
+    scale = np.abs(want).max()
+    tol = 2e-6
+    assert abs(loss - want_loss) < tol * max(1.0, abs(want_loss))
+    assert np.abs(grad - want).max() < tol * scale
+    # the bias gradients come from the unrounded dZ: they agree with a rounding-free sum of the
+    # restatement's dZ to fp32 resolution (checked inside `want` above), and no weight gradient
+    # of a hidden layer equals its fp32-mode value
+    _, g32 = oracle.mlp_loss_grad(dims, w, X, y, bf16=False)
+    assert np.abs(grad - g32).max() > 100 * tol * scale
+    # Each single rounding left out of the restatement moves it away from the oracle by far more
+    # than the tolerance: the comparison above would fail if the oracle dropped that rounding.
+    for name in ("x", "w_fwd", "act", "dz_wgrad", "dz_dgrad", "w_dgrad"):
+        _, mut = _mlp_bf16_restated(dims, w, X, y, drop=name)
+        assert np.abs(grad - mut).max() > 50 * tol * scale, name
+
+
+def test_mlp_bf16_bias_gradient_is_not_rounded(oracle):
+    # dZ_L values are chosen by construction to sit far from bf16 grid points: one layer, zero
+    # weights => p = 1/C for every class, dZ = (1/C - onehot)/B, which is not bf16-exact for
+    # C = 10, B = 3.  The bias gradient must be the exact column sum of those values.
+    dims, B = [8, 10], 3
+    w = np.zeros(oracle.mlp_param_count(dims), dtype=np.float32)
+    X = np.random.default_rng(5).standard_normal((B, 8)).astype(np.float32)
+    y = np.array([1, 1, 7], dtype=np.int32)
+    _, grad = oracle.mlp_loss_grad(dims, w, X, y, bf16=True)
+    dz = ((0.1 - np.eye(10)[y]) / B).astype(np.float32).astype(np.float64)
+    assert np.abs(grad[-10:] - dz.sum(0)).max() < 1e-7     # stored in fp32
+    rounded = _q_torch(dz).sum(0)
+    assert np.abs(rounded - dz.sum(0)).max() > 1e-5       # rounding dZ first would have shown
+    # and the weight gradient does use the rounded dZ (and the rounded inputs)
+    want = _q_torch(dz).T @ _q_torch(X)
+    assert np.abs(grad[:-10].reshape(10, 8) - want).max() < 1e-7
+
+
 # ---------------------------------------------------------------------------------- meta level
 def _state(oracle, n=257, P=5, mu=0.9, zeta=1.0, seed=0, stride=None):
     r = np.random.default_rng(seed)

@@ -3,10 +3,14 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mavg|reference]
 
 A step is one full round -- K_local SGD steps on all P learners, then the fused meta-update --
-of the CIFAR-shaped MLP workload (3072-512-512-10, bf16 GEMM operands, fp32 masters, P=8,
-K_local=8, B=128) on seeded synthetic data.  Prints ONE JSON line (rank 0).  With --gpus N > 1
-every rank runs an independent replica of the same workload on its own GPU (the method is
-simulated on one GPU; there is no exchange between GPUs), and `value` is the sum over ranks.
+of the large MLP workload (3072-2048-2048-2048-10, bf16 GEMM operands, fp32 masters, P=32,
+K_local=16, B=64: the largest configuration of the workload list that fits one GPU, and the one
+whose kernels are bound by HBM) on seeded synthetic data.  Prints ONE JSON line (rank 0); the same
+line carries, as extra keys, the CIFAR-shaped MLP (3072-512-512-10, P=8, K=8, B=128), the full
+round at 25.6 M parameters with seeded pseudo-gradients (K = 1 and 64) and the meta-update sweep
+at 11.2 M parameters.  With --gpus N > 1 every rank runs an independent replica of the same
+workload on its own GPU (the method is simulated on one GPU; there is no exchange between GPUs),
+and `value` is the sum over ranks.
 
 --impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same
 workload; it is a deliberately plain program and only a baseline.
@@ -27,7 +31,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "learner-samples/sec per MAVG round; meta-update HBM GB/s vs peak (1 B200)"
 UNIT = "learner-samples/s"
-WORKLOAD = "C2"
+WORKLOAD = "C4"
 
 
 def measured_peaks():
@@ -103,6 +107,13 @@ def workload_inputs(name=None):
     return cfg, x, y, w1
 
 
+def workload_label(name, cfg):
+    kind = {"C2": "CIFAR-shaped MLP", "C4": "large MLP"}.get(name, "MLP")
+    return (f"{name} {kind} {'-'.join(map(str, cfg['dims']))}, P={cfg['P']}, K={cfg['K']}, "
+            f"B={cfg['B']}, mu={cfg['mu']}, gamma={cfg['gamma']}, 50000 synthetic samples, labels "
+            "from a random teacher")
+
+
 def flop_per_sample(dims):
     # forward + weight gradient for every layer, data gradient for all but the first
     macs = sum(dims[l] * dims[l + 1] for l in range(len(dims) - 1))
@@ -125,32 +136,44 @@ def cpu_oracle_rate(cfg, x, y, w1, k_sample, reps=1):
     return units / statistics.median(times), threads, times
 
 
+def bounded_oracle_sample(cfg, x, y, w1, budget_s):
+    """Sizes a sample of the workload that the oracle finishes in about budget_s seconds: k_s of
+    the K local steps on p_s of the P learners (+ their meta-update).  One (learner, step) is the
+    smallest piece; it is timed first, on one thread."""
+    from oracle import oracle as O
+    _, _, t_cal = cpu_oracle_rate(dict(cfg, P=1), x, y, w1, 1, reps=1)
+    t1 = max(t_cal[0], 1e-6)
+    threads = min(cfg["P"], O.max_threads())
+    pieces = max(1, int(budget_s / t1 * threads))          # (learner, step) pieces that fit
+    p_s = int(min(cfg["P"], max(1, pieces)))
+    k_s = int(min(cfg["K"], max(1, pieces // p_s)))
+    return p_s, k_s, t1
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    cfg, x, y, w1 = workload_inputs()
-    # Bounded sample per step: one of the K local steps on p_s of the P learners (+ their
-    # meta-update), p_s sized from one calibration step so that the whole run stays near 100 s.
-    k_sample = 1
-    one = dict(cfg, P=1)
-    _, _, t_cal = cpu_oracle_rate(one, x, y, w1, k_sample, reps=1)
+    name = args.workload if args.workload in ("C2", "C4") else WORKLOAD
+    cfg, x, y, w1 = workload_inputs(name)
+    # Bounded sample per step, sized from one calibration piece so that the whole run stays near
+    # two minutes.
     total = args.warmup + args.steps
-    p_s = int(max(1, min(cfg["P"], 100.0 / max(total, 1) / max(t_cal[0], 1e-6))))
+    p_s, k_s, t1 = bounded_oracle_sample(cfg, x, y, w1, 120.0 / max(total, 1))
     sub = dict(cfg, P=p_s)
-    rate, threads, times = cpu_oracle_rate(sub, x, y, w1, k_sample, reps=total)
+    rate, threads, times = cpu_oracle_rate(sub, x, y, w1, k_s, reps=total)
     timed = times[args.warmup:]
-    units = p_s * k_sample * cfg["B"]
+    units = p_s * k_s * cfg["B"]
     value = units * len(timed) / sum(timed)
-    sample = (f"each step = 1 of the {cfg['K']} local steps on {p_s} of the {cfg['P']} learners "
+    sample = (f"each step = {k_s} of the {cfg['K']} local steps on {p_s} of the {cfg['P']} learners "
               f"(B={cfg['B']}) + their meta-update = {units} learner-samples")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(timed) / len(timed),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": "C2 CIFAR-shaped MLP 3072-512-512-10, P=8, K=8, B=128, mu=0.9 "
-                               "(bounded sample per step)", "global_batch": cfg["P"] * cfg["B"]},
+        "config": {"workload": workload_label(name, cfg) + " (bounded sample per step)",
+                   "global_batch": cfg["P"] * cfg["B"]},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -159,27 +182,24 @@ def run_reference(args):
     return 0
 
 
-# DRAM read + write bytes per launch, averaged over the launches of a class in one local step of
-# the C2 workload, from the ncu capture summarised in profiles/step_kernels_c2.md (cold cache:
-# ncu flushes L2 before every kernel; in a running round the fp32 masters stay in the L2 lines
-# set aside for them, so steady-state traffic is lower still: second table there).  Valid for the kernels as
-# captured; set an entry to None when its kernel changes.
-NCU_TRAFFIC_C2 = {
-    # all layers' weight gradients (captured as the graph's two launches, layer 1 and layers 3 + 2)
-    "wgrad_sgd_gemm": 57.703424e6 + 5.545216e6 + 11.806976e6 + 0.002560e6,
-    "fwd_gemm": (31.497728e6 + 0.010496e6 + 5.324800e6) / 2,     # hidden layers 1 and 2
-    "dgrad_gemm": 6.381056e6,
+# DRAM read + write bytes of ONE launch of the dominant kernel class, from the committed ncu
+# captures (profiles/): None when no capture of the kernel as it stands exists.  The large MLP
+# holds ~4.5 GB on the device at P = 32; its capture is taken with 8 learners (same layer shapes,
+# kernels and tile plans) and scaled by 4, since every kernel's traffic is proportional to P.
+NCU_TRAFFIC = {
+    "C2": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
+    "C4": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
 }
 
 
-def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False):
-    """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
+def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False):
+    """Bytes that must cross HBM per ROUND for each kernel class (weights streamed once per
+    product, activations in and out), and their total."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
     nW = [dims[l] * dims[l + 1] for l in range(L)]
     n = sum(nW) + sum(dims[1:])
     rows = P * B
-    out = {}
     per_round = {
         # replicas, w~, v read; v, w~ and (unless the copies are deferred) the replicas written
         "meta_update": dict(bytes=((4 if deferred else 8) * P + 16) * n, flops=0),
@@ -195,6 +215,13 @@ def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momen
                                - (4 * (P - 1) * sum(nW) if tensor_path else 0),
                                flops=K * 2 * rows * sum(nW)),
     }
+    return per_round
+
+
+def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False):
+    """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
+    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum)
+    out = {}
     for name, (ms, cnt) in prof.items():
         if cnt == 0 or ms <= 0:
             continue
@@ -212,35 +239,44 @@ def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momen
     return out
 
 
-def meta_update_sweep(m, torch, peaks, reps=5):
-    """Meta-update alone at the ResNet-18-sized sweep: n = 11.2 M, P in {4, 16, 64}, mu in {0, 0.9}."""
+def meta_update_sweep(m, torch, peaks, reps=7, inner=10):
+    """Meta-update alone at the ResNet-18-sized sweep: n = 11.2 M, P in {4, 16, 64}, mu in {0, 0.9}.
+    Per repetition: fresh replicas ~ N(0, 0.01) around the current model (untimed), L2 flushed by a
+    256 MiB memset, then `inner` meta-updates back to back inside one event pair (their time does
+    not depend on the data; each of them streams more than the L2 holds); also one launch alone
+    right after a flush (`cold_gbs`)."""
     n = 11_200_000
     res = []
     w1 = (0.05 * torch.randn(n, generator=torch.Generator().manual_seed(1))).numpy()
     for P in (4, 16, 64):
         for mu in (0.0, 0.9):
             g = m.Mavg(w1, P=P, K=1, local_lr=0.1, mu=mu, objective=m.OBJ_NONE)
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
             gen = torch.Generator(device=g.device).manual_seed(P)
-            times = []
-            for u in range(3 + reps):
-                # replicas ~ N(0, 0.01) around the current global model (untimed)
+            times, cold = [], []
+            for u in range(2 + reps):
                 g.replicas[:, :n] = g.w[None, :] + 0.1 * torch.randn((P, n), device=g.device,
                                                                      generator=gen)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                g.meta_update()
-                b.record()
-                b.synchronize()
-                if u >= 3:
-                    times.append(a.elapsed_time(b))
+                for count, sink in ((1, cold), (inner, times)):
+                    flush.zero_()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    for _ in range(count):
+                        g.meta_update()
+                    b.record()
+                    b.synchronize()
+                    if u >= 2:
+                        sink.append(a.elapsed_time(b) / count)
             g.sync()
             by = ((8 * P + 16) - (4 if mu == 0.0 else 0)) * n
             ms = statistics.median(times)
             res.append(dict(P=P, mu=mu, n=n, ms=ms, gbs=by / ms / 1e6,
                             frac_measured=by / ms / 1e6 / peaks["hbm_gbs"],
-                            frac_nominal_8tbs=by / ms / 1e6 / 8000.0))
+                            frac_nominal_8tbs=by / ms / 1e6 / 8000.0,
+                            cold_gbs=by / statistics.median(cold) / 1e6,
+                            launches_per_timing=inner))
             g.close()
-            del g
+            del g, flush
             torch.cuda.empty_cache()
     return res
 
@@ -262,22 +298,22 @@ def whole_job_value(units_per_step, steps, total_ms, world):
     return world * units_per_step * steps / (total_ms * 1e-3)
 
 
-def run_pseudograd(args, m, torch, peaks, rank):
+def pseudograd_rounds(args, m, torch, peaks, Ks, steps):
     """Full round at the ResNet-50-sized vector (n = 25.6 M, P = 16) with seeded pseudo-gradients:
-    one line per K with the local pass, the meta-update and the whole round."""
+    per K the local pass, the meta-update and the whole round."""
     from paper_2110_00625_b200 import workloads as W
     cfg = W.CONFIGS["C5"]
     n, P = cfg["n"], cfg["P"]
     w1 = W.global_model(n)
     out = []
-    for K in cfg["K"]:
+    for K in Ks:
         g = m.Mavg(w1, P=P, K=K, local_lr=cfg["gamma"], mu=0.9, seed=W.BASE_SEED,
                    objective=m.OBJ_PSEUDOGRAD, sigma=cfg["sigma"], defer_broadcast=not args.no_defer,
                    learner_momentum=args.beta)
         for _ in range(3):
             g.round()
         g.sync()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
         for a, b, c in ev:
             a.record(); g.local_steps(); b.record(); g.meta_update(); c.record()
         torch.cuda.synchronize()
@@ -286,21 +322,176 @@ def run_pseudograd(args, m, torch, peaks, rank):
         # the local pass reads w~ once (every learner starts from it) and writes P learner models;
         # the meta-update reads them with w~ and v and writes w~, v and, unless deferred, P copies
         meta_b = ((8 if args.no_defer else 4) * P + 16) * n
+        local_b = ((12 if args.beta else 4) * P + 4) * n
+        var_rate = P * K * n / (loc * 1e-3)
         out.append(dict(K=K, local_ms=loc, meta_ms=met, round_ms=loc + met,
                         learner_steps_per_s=P * K / ((loc + met) * 1e-3),
-                        local_gbs=((12 if args.beta else 4) * P + 4) * n / loc / 1e6,
+                        local_gbs=local_b / loc / 1e6,
+                        local_frac_hbm=local_b / loc / 1e6 / peaks["hbm_gbs"],
                         learner_momentum=args.beta,
-                        variates_per_s=P * K * n / (loc * 1e-3),
+                        variates_per_s=var_rate,
+                        local_frac_alu=var_rate / PSEUDOGRAD_ALU_PEAK_VARIATES,
                         meta_gbs=meta_b / met / 1e6,
                         meta_frac_measured=meta_b / met / 1e6 / peaks["hbm_gbs"],
                         defer_broadcast=not args.no_defer))
         g.close()
         del g
         torch.cuda.empty_cache()
+    return out
+
+
+# Peak rate of the K-fused pseudo-gradient pass when the integer pipe binds (variates/s): see the
+# derivation in the design document (instructions per variate from the kernel's own count, issue
+# rate of 148 SMs x 4 schedulers x 1 warp instruction per clock at the maximum SM clock).
+PSEUDOGRAD_INSTR_PER_VARIATE = 30.0
+PSEUDOGRAD_ALU_PEAK_VARIATES = 148 * 4 * 32 * 1.965e9 / PSEUDOGRAD_INSTR_PER_VARIATE
+
+
+def run_pseudograd(args, m, torch, peaks, rank):
+    from paper_2110_00625_b200 import workloads as W
+    out = pseudograd_rounds(args, m, torch, peaks, W.CONFIGS["C5"]["K"], args.steps)
     if rank == 0:
         print(json.dumps({"workload": "C5 full round, n=25.6M fp32, P=16, seeded pseudo-gradients",
                           "steps": args.steps, "results": out}))
     return 0
+
+
+def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, with_cpu, with_e2e,
+                with_clocks):
+    """Times `steps` rounds of an MLP workload three ways: device-resident (one event pair per
+    round, L2 flushed between rounds), end to end through mavg_round_host, and per kernel class.
+    Returns the pieces of the JSON line."""
+    cfg, x, y, w1 = workload_inputs(name)
+    if args.learners:
+        cfg["P"] = args.learners      # reduced-size captures under a profiler only
+
+    # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
+    cpu = None
+    if with_cpu:
+        p_s, k_s, t1 = bounded_oracle_sample(cfg, x, y, w1, 20.0)
+        rate, threads, times = cpu_oracle_rate(dict(cfg, P=p_s), x, y, w1, k_s)
+        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"one round cut to {k_s} of {cfg['K']} local steps on {p_s} of "
+                         f"{cfg['P']} learners + their meta-update ({p_s * k_s * cfg['B']} "
+                         f"learner-samples, {times[0]:.1f} s)"}
+
+    mode = args.gemm
+    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"],
+               block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
+               dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}",
+               defer_broadcast=not args.no_defer, learner_momentum=args.beta, l2_keep=args.l2_keep)
+    g.set_schedule(args.schedule)
+    units = cfg["P"] * cfg["K"] * cfg["B"]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        g.round()
+    g.sync()
+
+    # ---- timed region: device-resident inputs -------------------------------------------------
+    sampler = ClockSampler(local) if with_clocks else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+           torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    l0 = g.launch_count()
+    barrier()
+    if sampler:
+        sampler.start()
+    t_wall0 = time.perf_counter()
+    for a, mid, b in ev:
+        if args.l2_keep:
+            g.l2_release()                 # masters the library asked the L2 to keep: let go
+        flush.zero_()                      # L2 flush, outside the step's event pair
+        a.record()
+        g.local_steps()
+        mid.record()
+        g.meta_update()
+        b.record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop() if sampler else None
+    launches = g.launch_count() - l0
+    step_ms = [a.elapsed_time(b) for a, _, b in ev]
+    meta_ms = [mid.elapsed_time(b) for _, mid, b in ev]
+    total_ms = sum(step_ms)
+    g.sync()
+
+    # ---- end to end: model in host memory, copies inside the timed region ----------------------
+    e2e_ms = 0.0
+    if with_e2e:
+        wh = torch.from_numpy(w1.copy()).pin_memory()
+        vh = torch.zeros(g.n).pin_memory()
+        for _ in range(2):
+            g.round_host(wh, vh)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            g.round_host(wh, vh)
+        b.record()
+        barrier()
+        e2e_ms = a.elapsed_time(b)
+
+    # ---- per-kernel device times: the same steps again with an event pair around every launch ---
+    g.set_profiling(True)
+    g.get_profile(reset=True)
+    psteps = min(steps, 20)
+    for _ in range(psteps):
+        if args.l2_keep:
+            g.l2_release()
+        flush.zero_()
+        g.round()
+    prof = g.get_profile(reset=True)
+    g.set_profiling(False)
+    kern = kernel_rooflines(cfg, prof, psteps, peaks, mode == 1, deferred=not args.no_defer,
+                            momentum=args.beta != 0.0)
+    n = g.n
+    g.close()
+    del g, flush
+    torch.cuda.empty_cache()
+
+    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=torch.device("cuda", local))
+
+    # the roofline object describes the kernel class a local step spends most of its time in
+    timed = {k: v for k, v in kern.items() if "gbs" in v and k != "meta_update"}
+    dom = max(timed, key=lambda k: timed[k]["ms_total"]) if timed else None
+    roof = None
+    if dom:
+        e = timed[dom]
+        hbm_time = e["bytes_per_launch"] / (peaks["hbm_gbs"] * 1e9)
+        tensor_time = (e.get("tflops", 0) and
+                       e["tflops"] * 1e12 * e["ms_per_launch"] * 1e-3 /
+                       (peaks["bf16_tflops_sustained"] * 1e12))
+        if tensor_time and tensor_time > hbm_time:
+            roof = {"bound": "tensor", "achieved": e["tflops"],
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": e["frac_tensor"], "traffic": None}
+        else:
+            roof = {"bound": "hbm", "achieved": e["gbs"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": e["frac_hbm"], "traffic": None}
+        roof["kernel"] = dom
+        roof["peak_source"] = peaks["source"]
+        roof["bytes_per_launch"] = e["bytes_per_launch"]
+        roof["ms_per_launch"] = e["ms_per_launch"]
+        if mode == 1 and not args.learners and not args.beta:
+            roof["traffic"] = NCU_TRAFFIC.get(name, {}).get(dom)
+    # the whole round against the HBM roofline: every class's algorithmic bytes / the round's time
+    per_round = algorithmic_bytes(cfg, mode == 1, deferred=not args.no_defer,
+                                  momentum=args.beta != 0.0)
+    round_bytes = sum(v["bytes"] for v in per_round.values())
+    ms_round = total_ms / steps
+    return dict(
+        cfg=cfg, n=n, units=units, total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
+        clocks=clocks, cpu=cpu, kern=kern, roof=roof, t_wall=t_wall, mode=mode,
+        meta_in_round={"ms": statistics.median(meta_ms),
+                       "gbs": per_round["meta_update"]["bytes"] / statistics.median(meta_ms) / 1e6},
+        round_roofline={"bytes_per_round": round_bytes, "gbs": round_bytes / ms_round / 1e6,
+                        "frac_hbm": round_bytes / ms_round / 1e6 / peaks["hbm_gbs"]},
+        tflops_round=flop_per_sample(cfg["dims"]) * units * steps / (total_ms * 1e-3) / 1e12)
 
 
 def run_mavg(args):
@@ -320,155 +511,64 @@ def run_mavg(args):
     if args.workload == "C5":
         return run_pseudograd(args, m, torch, peaks, rank)
     if args.sweep_only:
-        print(json.dumps({"meta_update_sweep": meta_update_sweep(m, torch, peaks, reps=2)}))
+        print(json.dumps({"meta_update_sweep": meta_update_sweep(m, torch, peaks, reps=3)}))
         return 0
-    cfg, x, y, w1 = workload_inputs(args.workload)
-    if args.learners:
-        cfg["P"] = args.learners      # reduced-size captures under a profiler only
 
-    # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        k_sample = 4 if args.workload == "C2" else 1
-        rate, threads, times = cpu_oracle_rate(cfg, x, y, w1, k_sample)
-        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"one round cut to {k_sample} of {cfg['K']} local steps on all "
-                         f"{cfg['P']} learners + meta-update ({cfg['P'] * k_sample * cfg['B']} "
-                         f"learner-samples, {times[0]:.1f} s)"}
+    single = rank == 0 and world == 1
+    r = measure_mlp(args.workload, args, m, torch, dist, peaks, world, rank, local, args.steps,
+                    with_cpu=single and not args.no_cpu_baseline, with_e2e=True, with_clocks=True)
+    extras = {}
+    if single and not args.no_extras:
+        # the other workloads of the list, shorter, in the same process and on the same line
+        other = "C2" if args.workload == "C4" else "C4"
+        o = measure_mlp(other, args, m, torch, dist, peaks, world, rank, local,
+                        steps=min(args.steps, 50), with_cpu=False, with_e2e=False, with_clocks=False)
+        extras[other] = {
+            "workload": workload_label(other, o["cfg"]), "ms_per_round": o["total_ms"] / min(args.steps, 50),
+            "learner_samples_per_s": whole_job_value(o["units"], min(args.steps, 50), o["total_ms"], 1),
+            "tflops_round": o["tflops_round"], "round_roofline": o["round_roofline"],
+            "kernels": {k: {q: v[q] for q in ("ms_per_launch", "gbs", "frac_hbm", "tflops") if q in v}
+                        for k, v in o["kern"].items()},
+            "meta_update_in_round": o["meta_in_round"]}
+        extras["C5"] = {"workload": "C5 full round, n=25.6M fp32, P=16, seeded pseudo-gradients, mu=0.9",
+                        "results": pseudograd_rounds(args, m, torch, peaks, (1, 64), 20)}
+    sweep = meta_update_sweep(m, torch, peaks) if single and not args.no_sweep else None
 
-    mode = args.gemm
-    g = m.Mavg(w1, P=cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"],
-               block_lr=cfg["zeta"], B=cfg["B"], seed=0x211000625, objective=m.OBJ_MLP,
-               dims=cfg["dims"], gemm_bf16=mode, x=x, y=y, x_bf16=True, device=f"cuda:{local}",
-               defer_broadcast=not args.no_defer, learner_momentum=args.beta)
-    g.set_schedule(args.schedule)
-    units = cfg["P"] * cfg["K"] * cfg["B"]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=g.device)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        g.round()
-    g.sync()
-
-    # ---- timed region: device-resident inputs -------------------------------------------------
-    sampler = ClockSampler(local)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
-           torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    l0 = g.launch_count()
-    barrier()
-    sampler.start()
-    t_wall0 = time.perf_counter()
-    for a, mid, b in ev:
-        g.l2_release()                     # masters the library asked the L2 to keep: let go
-        flush.zero_()                      # L2 flush, outside the step's event pair
-        a.record()
-        g.local_steps()
-        mid.record()
-        g.meta_update()
-        b.record()
-    barrier()
-    t_wall = time.perf_counter() - t_wall0
-    clocks = sampler.stop()
-    launches = g.launch_count() - l0
-    step_ms = [a.elapsed_time(b) for a, _, b in ev]
-    meta_ms = [mid.elapsed_time(b) for _, mid, b in ev]
-    total_ms = sum(step_ms)
-    g.sync()
-
-    # ---- end to end: model in host memory, copies inside the timed region ----------------------
-    wh = torch.from_numpy(w1.copy()).pin_memory()
-    vh = torch.zeros(g.n).pin_memory()
-    for _ in range(2):
-        g.round_host(wh, vh)
-    barrier()
-    t0 = time.perf_counter()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(args.steps):
-        g.round_host(wh, vh)
-    b.record()
-    barrier()
-    e2e_ms = a.elapsed_time(b)
-
-    # ---- per-kernel device times: the same steps again with an event pair around every launch ---
-    g.set_profiling(True)
-    g.get_profile(reset=True)
-    for _ in range(args.steps):
-        g.l2_release()
-        flush.zero_()
-        g.round()
-    prof = g.get_profile(reset=True)
-    g.set_profiling(False)
-    kern = kernel_rooflines(cfg, prof, args.steps, peaks, mode == 1, deferred=not args.no_defer,
-                            momentum=args.beta != 0.0)
-
-    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=g.device)
-
-    line = None
     if rank == 0:
-        # the roofline object describes the kernel with the longest launches of a local step (a
-        # class can hold more than one kernel: the forward products of the hidden layers are two
-        # different kernels, each shorter than the weight-gradient launch)
-        timed = {k: v for k, v in kern.items() if "gbs" in v and k != "meta_update"}
-        dom = max(timed, key=lambda k: timed[k]["ms_per_launch"]) if timed else None
-        roof = None
-        if dom:
-            e = timed[dom]
-            hbm_time = e["bytes_per_launch"] / (peaks["hbm_gbs"] * 1e9)
-            tensor_time = (e.get("tflops", 0) and
-                           e["tflops"] * 1e12 * e["ms_per_launch"] * 1e-3 /
-                           (peaks["bf16_tflops_sustained"] * 1e12))
-            if tensor_time and tensor_time > hbm_time:
-                roof = {"bound": "tensor", "achieved": e["tflops"],
-                        "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                        "frac": e["frac_tensor"], "traffic": None}
-            else:
-                roof = {"bound": "hbm", "achieved": e["gbs"], "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": e["frac_hbm"], "traffic": None}
-            roof["kernel"] = dom
-            roof["peak_source"] = peaks["source"]
-            if args.workload == "C2" and mode == 1 and not args.learners and not args.beta:
-                roof["traffic"] = NCU_TRAFFIC_C2.get(dom)
-        sweep = meta_update_sweep(m, torch, peaks) if world == 1 and not args.no_sweep else None
-        n = g.n
+        cfg, n, steps = r["cfg"], r["n"], args.steps
+        clocks = r["clocks"]
         line = {
-            "metric": METRIC, "value": whole_job_value(units, args.steps, total_ms, world), "unit": UNIT,
-            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if mode else "f32", "data": "synthetic",
-            "config": {"workload": f"{args.workload} CIFAR-shaped MLP {'-'.join(map(str, cfg['dims']))}, "
-                                   f"P={cfg['P']}, K={cfg['K']}, B={cfg['B']}, mu={cfg['mu']}, "
-                                   "gamma=0.05, 50000 synthetic samples, labels from a random teacher",
+            "metric": METRIC, "value": whole_job_value(r["units"], steps, r["total_ms"], world),
+            "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup,
+            "ms_per_step": r["total_ms"] / steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if r["mode"] else "f32", "data": "synthetic",
+            "config": {"workload": workload_label(args.workload, cfg),
                        "global_batch": cfg["P"] * cfg["B"], "parallelism": "replicas only",
                        "gemm": {1: "tcgen05 tensor cores", 2: "CUDA cores, bf16-rounded operands",
-                                0: "CUDA cores fp32"}[mode],
+                                0: "CUDA cores fp32"}[r["mode"]],
                        "defer_broadcast": not args.no_defer, "learner_momentum": args.beta,
-                       "schedule": ["CUDA graph of per-product launches, fused last layer",
+                       "l2_keep": bool(args.l2_keep),
+                       "schedule": ["CUDA graph of per-product launches",
                                     "one persistent kernel per round",
                                     "CUDA graph of per-product launches, all on tensor cores"][args.schedule],
-                       "l2": "between steps, outside the step's events: kept lines released, then flushed by a 256 MiB memset",
+                       "l2": "flushed between steps by a 256 MiB memset, outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
                        "reasons": clocks["reasons"], "samples": clocks["samples"]},
-            "e2e": {"value": whole_job_value(units, args.steps, e2e_ms, world), "unit": UNIT,
+            "e2e": {"value": whole_job_value(r["units"], steps, r["e2e_ms"], world), "unit": UNIT,
                     "h2d_bytes_per_step": 8 * n, "d2h_bytes_per_step": 8 * n + 4},
-            "gpu_launches": launches,
-            "roofline": roof,
-            "cpu_baseline": cpu,
-            "wall_s_timed_region": t_wall,
-            "meta_update_in_round": {"ms": statistics.median(meta_ms),
-                                     "gbs": ((8 if args.no_defer else 4) * cfg["P"] + 16) * n
-                                            / statistics.median(meta_ms) / 1e6},
-            "kernels": kern,
+            "gpu_launches": r["launches"],
+            "roofline": r["roof"],
+            "cpu_baseline": r["cpu"],
+            "wall_s_timed_region": r["t_wall"],
+            "round_roofline": r["round_roofline"],
+            "meta_update_in_round": r["meta_in_round"],
+            "kernels": r["kern"],
             "meta_update_sweep": sweep,
-            "tflops_round": flop_per_sample(cfg["dims"]) * units * args.steps / (total_ms * 1e-3) / 1e12,
+            "tflops_round": r["tflops_round"],
+            "other_workloads": extras or None,
         }
         print(json.dumps(line))
-    g.close()
     if world > 1:
         dist.destroy_process_group()
     return 0
@@ -477,14 +577,14 @@ def run_mavg(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mavg", choices=["mavg", "reference"])
     ap.add_argument("--gemm", type=int, default=1, choices=[1, 2],
                     help="1: tensor cores (default); 2: CUDA cores with bf16-rounded operands")
-    ap.add_argument("--workload", default="C2", choices=["C2", "C4", "C5"],
-                    help="C2 is the benchmark workload; C4 (large MLP) and C5 (pseudo-gradient "
-                         "round at 25.6 M parameters) print the same measurements for context")
+    ap.add_argument("--workload", default=WORKLOAD, choices=["C2", "C4", "C5"],
+                    help="C4 (large MLP) is the benchmark workload; C2 (CIFAR-shaped MLP) as the "
+                         "main workload, or C5 (pseudo-gradient round at 25.6 M parameters) alone")
     ap.add_argument("--learners", type=int, default=0,
                     help="override P (for small profiler captures; not a benchmark setting)")
     ap.add_argument("--sweep-only", action="store_true",
@@ -497,6 +597,10 @@ def main():
                          "product on tensor cores (1 and 2 for comparison)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the other workloads that the default line carries as extra keys")
+    ap.add_argument("--l2-keep", action="store_true",
+                    help="ask the library to set L2 aside for the learners' masters (small models)")
     ap.add_argument("--no-defer", action="store_true",
                     help="write the P copies of w~ in the meta-update instead of folding them into "
                          "the next round's first local step")

@@ -112,6 +112,15 @@ typedef struct {
    * learners restart from w~ (the first local step after a (re-)broadcast). */
   float learner_momentum;         /* beta, 0 <= beta < 1 */
   int32_t learner_momentum_reset; /* 0 or 1 */
+  int32_t l2_keep;   /* 0 (default): the library leaves the L2 cache's partitioning alone.
+                        1: an MLP handle on the tensor-core path whose P master copies together
+                        take at most half the L2 asks mavg_create to set aside that much of the
+                        L2 for them (see mavg_create); ignored by every other handle.  This is an
+                        opt-in because the set-aside belongs to the whole CUDA context: while it is
+                        in force, every streaming kernel of the process -- this library's
+                        meta-update of a large model included -- has only the rest of the L2 and
+                        was measured 25-30 % slower (6.2 -> 4.4 TB/s), against a gain of 2-3 % on
+                        a small MLP round. */
 } mavg_config;
 
 /* Caller-owned DEVICE buffers.  Every base pointer must be 16-byte aligned. */
@@ -134,13 +143,14 @@ mavg_status mavg_workspace_bytes(const mavg_config *cfg, size_t *out_bytes);
 /* Algorithm 1, the two initialisation lines and the first "set w^j = w~": v <- 0, w^j <- w~_1
  * (the copies are skipped with defer_broadcast, see there).
  * Validates everything; on failure *out is NULL.  Enqueues the initialisation on the stream.
- * For an MLP handle on the tensor-core path whose P master copies together take at most half the
- * L2, the call also raises the CUDA context's limit cudaLimitPersistingL2CacheSize to their size
- * (capped by the device's maximum): the weight-gradient kernels then ask the L2 to keep the
- * masters from one local step to the next instead of sending them through HBM.  The limit
- * belongs to the calling process's context: it follows the largest request among the live
- * handles on the device (never below the value found), and the mavg_destroy of the last of them
- * puts the previous value back. */
+ * With cfg->l2_keep = 1, for an MLP handle on the tensor-core path whose P master copies together
+ * take at most half the L2, the call also raises the CUDA context's limit
+ * cudaLimitPersistingL2CacheSize to their size (capped by the device's maximum): the
+ * weight-gradient kernels then ask the L2 to keep the masters from one local step to the next
+ * instead of sending them through HBM.  The limit belongs to the calling process's context: it
+ * follows the largest request among the live handles on the device (never below the value
+ * found), and the mavg_destroy of the last of them puts the previous value back.  Without
+ * l2_keep the library never touches that limit. */
 mavg_status mavg_create(const mavg_config *cfg, const mavg_buffers *buf, mavg_handle *out);
 
 /* Learner level of Algorithm 1 (inner loop over k): K SGD steps on all P replicas for the round
@@ -181,7 +191,8 @@ mavg_status mavg_set_learner_momentum(mavg_handle h, float beta, int32_t reset);
 mavg_status mavg_get_batch_indices(mavg_handle h, int64_t round, int32_t learner, int32_t step,
                                    int32_t *out);
 
-/* The P*K minibatch losses of the last mavg_local_steps, out[j*K + k-1] (HOST); waits. */
+/* The P*K minibatch losses of the last mavg_local_steps, out[j*K + k-1] (HOST); waits.
+ * MAVG_ERR_STATE for objectives without a loss (everything but MAVG_OBJ_MLP). */
 mavg_status mavg_get_losses(mavg_handle h, float *out);
 
 /* Number of completed meta-updates (the next round is this + 1), and its setter for resuming
@@ -228,6 +239,19 @@ mavg_status mavg_get_profile(mavg_handle h, float *ms, int64_t *launches, int32_
 
 /* Waits for the stream; reports CUDA errors and a tripped device-side wait limit. */
 mavg_status mavg_sync(mavg_handle h);
+
+/* Every wait inside the kernels (on an mbarrier, on another block's counter) gives up after a time
+ * limit instead of spinning forever; the kernel then records an error code, lets its own copies
+ * in flight land, frees what it holds and returns, and the next mavg_sync reports
+ * MAVG_ERR_TIMEOUT and clears the record (the paper has no counterpart: this is failure detection
+ * of the engine itself).  The default limit is 2 s.  mavg_set_wait_limit changes it for this
+ * handle's later launches (microseconds, >= 1; 0 restores the default); stream-ordered.
+ * mavg_selftest_wait launches a one-warp kernel that waits on a barrier nobody will ever arrive
+ * on, so that the wait runs out: after it, mavg_sync must return MAVG_ERR_TIMEOUT once and
+ * MAVG_OK afterwards, and the handle must work as before.  Nothing traps or faults; the kernel
+ * returns by itself after the limit. */
+mavg_status mavg_set_wait_limit(mavg_handle h, int32_t microseconds);
+mavg_status mavg_selftest_wait(mavg_handle h);
 
 /* Waits for the stream, then returns every L2 line that this context asked to be kept (see
  * mavg_create) to normal eviction; a no-op for handles that keep nothing.  For measurements that

@@ -21,7 +21,8 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams",
            "mavg_set_learner_momentum", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
-           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync", "mavg_cache_release", "mavg_last_error",
+           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync",
+           "mavg_set_wait_limit", "mavg_selftest_wait", "mavg_cache_release", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
@@ -40,6 +41,7 @@ class Config(C.Structure):
         ("stream", C.c_void_p),
         ("defer_broadcast", C.c_int32),
         ("learner_momentum", C.c_float), ("learner_momentum_reset", C.c_int32),
+        ("l2_keep", C.c_int32),
     ]
 
 
@@ -97,6 +99,8 @@ def load_library():
                                              C.c_void_p]
     L.mavg_materialize_replicas.argtypes = [H]
     L.mavg_sync.argtypes = [H]
+    L.mavg_set_wait_limit.argtypes = [H, C.c_int32]
+    L.mavg_selftest_wait.argtypes = [H]
     L.mavg_cache_release.argtypes = [H]
     L.mavg_last_error.argtypes = [H]
     L.mavg_last_error.restype = C.c_char_p
@@ -110,7 +114,8 @@ def load_library():
 
 def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE, n=0, dims=None,
                 gemm_bf16=0, sigma=0.0, x_ptr=0, x_dtype=X_F32, y_ptr=0, n_samples=0, stream=0,
-                defer_broadcast=False, learner_momentum=0.0, learner_momentum_reset=False):
+                defer_broadcast=False, learner_momentum=0.0, learner_momentum_reset=False,
+                l2_keep=False):
     cfg = Config()
     cfg.P, cfg.K, cfg.B = P, K, B
     cfg.local_lr, cfg.block_lr, cfg.mu = local_lr, block_lr, mu
@@ -128,6 +133,7 @@ def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NON
     cfg.defer_broadcast = 1 if defer_broadcast else 0
     cfg.learner_momentum = learner_momentum
     cfg.learner_momentum_reset = 1 if learner_momentum_reset else 0
+    cfg.l2_keep = 1 if l2_keep else 0
     return cfg
 
 
@@ -154,7 +160,7 @@ class Mavg:
     def __init__(self, w1, P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NONE,
                  dims=None, gemm_bf16=0, sigma=0.0, x=None, y=None, x_bf16=False, stride=None,
                  device="cuda:0", stream=None, defer_broadcast=False, learner_momentum=0.0,
-                 learner_momentum_reset=False, with_learner_u=None):
+                 learner_momentum_reset=False, with_learner_u=None, l2_keep=False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -178,7 +184,8 @@ class Mavg:
         sptr = stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream
         self.cfg = make_config(P, K, local_lr, mu, block_lr, B, seed, objective, n, dims, gemm_bf16,
                                sigma, x_ptr, X_BF16 if x_bf16 else X_F32, y_ptr, n_samples, sptr,
-                               defer_broadcast, learner_momentum, learner_momentum_reset)
+                               defer_broadcast, learner_momentum, learner_momentum_reset,
+                               l2_keep)
         # learner momentum buffers u^j [P, stride]: allocated when beta != 0 or on request (a
         # handle that switches the momentum on later with set_learner_momentum)
         if with_learner_u is None:
@@ -276,6 +283,13 @@ class Mavg:
 
     def sync(self):
         self._check(self.lib.mavg_sync(self.handle))
+
+    def set_wait_limit(self, microseconds):
+        self._check(self.lib.mavg_set_wait_limit(self.handle, int(microseconds)))
+
+    def selftest_wait(self):
+        """Launches the kernel whose wait cannot be satisfied (see mavg_selftest_wait)."""
+        self._check(self.lib.mavg_selftest_wait(self.handle))
 
     def l2_release(self):
         """Wait for the stream and give up the L2 lines kept for the masters (cold-cache timing)."""

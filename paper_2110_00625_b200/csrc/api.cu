@@ -10,6 +10,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 using namespace mavg;
 
@@ -39,6 +40,8 @@ mavg_status validate_config(const mavg_config* cfg, std::string* why) {
     return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum must be in [0, 1)");
   if (cfg->learner_momentum_reset != 0 && cfg->learner_momentum_reset != 1)
     return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum_reset must be 0 or 1");
+  if (cfg->l2_keep != 0 && cfg->l2_keep != 1)
+    return fail(why, MAVG_ERR_INVALID_ARG, "l2_keep must be 0 or 1");
   if (cfg->learner_momentum != 0.f && cfg->objective == MAVG_OBJ_NONE)
     return fail(why, MAVG_ERR_INVALID_ARG, "learner_momentum needs a learner level (objective)");
   switch (cfg->objective) {
@@ -130,6 +133,21 @@ __global__ void k_mean_loss(const float* __restrict__ losses, int count, float* 
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (threadIdx.x == 0) out[0] = s / (float)count;
   }
+}
+
+// A wait that cannot be satisfied: one warp, a barrier that expects an arrival nobody makes.  The
+// bounded wait gives up after the handle's limit, records `code` and the kernel returns.
+__global__ void k_selftest_wait(int* status, int code) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) tc::mbar_wait(&bar, 0, &abort_flag, status, code);
+  __syncwarp();
 }
 
 mavg_status do_local_steps(mavg_ctx* c) {
@@ -293,6 +311,7 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
   c->stream = (cudaStream_t)cfg->stream;
   c->ws = ws;
   c->sm_count = prop.multiProcessorCount;
+  c->device = dev;
   c->l2_bytes = (size_t)prop.l2CacheSize;
 
   e = cudaMemsetAsync(ws_ptr(c, c->ws.status), 0, 256, c->stream);
@@ -319,7 +338,7 @@ mavg_status mavg_create(const mavg_config* cfg, const mavg_buffers* buf, mavg_ha
       delete c;
       return st;
     }
-    if (c->cfg.gemm_bf16 == 1 && masters_fit_l2(c)) {   // the tensor-core path
+    if (c->cfg.l2_keep == 1 && c->cfg.gemm_bf16 == 1 && masters_fit_l2(c)) {   // opt-in, tensor-core path
       // Room in the L2 for the learners' masters (see mavg_create in mavg.h).  Without it the
       // keep hints of the weight-gradient kernels have no effect; a refusal only costs speed.
       const size_t want = (size_t)cfg->P * (size_t)buf->replica_stride * sizeof(float);
@@ -445,6 +464,10 @@ mavg_status mavg_get_batch_indices(mavg_handle h, int64_t round, int32_t learner
 mavg_status mavg_get_losses(mavg_handle h, float* out) {
   CHECK_HANDLE(h);
   if (!out) return set_err(h, MAVG_ERR_INVALID_ARG, "out is NULL");
+  // only the MLP objective has a loss; for the others K may have grown past the K the loss
+  // buffer was sized for (mavg_set_hparams bounds K for MLP handles only)
+  if (h->cfg.objective != MAVG_OBJ_MLP)
+    return set_err(h, MAVG_ERR_STATE, "minibatch losses exist for the MLP objective only");
   CU(h, cudaMemcpyAsync(out, ws_ptr(h, h->ws.losses), (size_t)h->cfg.P * h->cfg.K * sizeof(float),
                         cudaMemcpyDeviceToHost, h->stream), "loss read-back");
   CU(h, cudaStreamSynchronize(h->stream), "stream synchronize");
@@ -515,6 +538,24 @@ mavg_status mavg_sync(mavg_handle h) {
     cudaMemsetAsync(ws_ptr(h, h->ws.status), 0, sizeof(int32_t), h->stream);
     return set_err(h, MAVG_ERR_TIMEOUT, msg);
   }
+  return MAVG_OK;
+}
+
+mavg_status mavg_set_wait_limit(mavg_handle h, int32_t microseconds) {
+  CHECK_HANDLE(h);
+  if (microseconds < 0) return set_err(h, MAVG_ERR_INVALID_ARG, "the wait limit must be >= 0 microseconds");
+  h->wait_limit_us = microseconds;
+  // status[1] of the handle's status area; the copy is taken from pageable memory before the call returns
+  CU(h, cudaMemcpyAsync(ws_ptr(h, h->ws.status) + sizeof(int32_t), &h->wait_limit_us, sizeof(int32_t),
+                        cudaMemcpyHostToDevice, h->stream), "wait limit upload");
+  return MAVG_OK;
+}
+
+mavg_status mavg_selftest_wait(mavg_handle h) {
+  CHECK_HANDLE(h);
+  k_selftest_wait<<<1, 32, 0, h->stream>>>((int*)ws_ptr(h, h->ws.status), 99);
+  h->launches++;
+  CU(h, cudaGetLastError(), "self-test kernel");
   return MAVG_OK;
 }
 

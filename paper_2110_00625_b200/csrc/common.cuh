@@ -77,7 +77,8 @@ struct ShadowMap {
 };
 
 struct Workspace {           // byte offsets into the caller's scratch buffer
-  size_t status = 0;         // int32[64]: [0] device wait-limit flag; bytes 64..71: round (int64)
+  size_t status = 0;         // int32[64]: [0] code of the first wait that ran out; [1] wait limit in
+                             // microseconds (0: default); bytes 64..71: round (int64)
   size_t losses = 0;         // float [P*K]
   size_t loss_mean = 0;      // float [1]
   size_t idx = 0;            // int32 [P*B] sample indices of the current step
@@ -97,6 +98,7 @@ struct mavg_ctx {
   mavg_status sticky = MAVG_OK;
   std::string err;
   int sm_count = 148;
+  int32_t wait_limit_us = 0;  // mirrored in status[1] on the device
   size_t l2_bytes = 0;
   bool replicas_equal_global = true;  // every learner's model is w~: true between a (re-)broadcast
                                       // and the next local step

@@ -154,7 +154,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
         for (int i = max(0, issued - stages); i < issued; ++i) {
           const uint64_t t0 = global_timer_ns();
           while (!mbar_try_wait(&sh.full_bar[(it0 + i) % stages], ((it0 + i) / stages) & 1))
-            if (global_timer_ns() - t0 > kWaitLimitNs) break;
+            if (global_timer_ns() - t0 > wait_limit_ns(g.status)) break;
         }
       }
     }
@@ -249,7 +249,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             const uint64_t t0 = global_timer_ns();
             while (!(got = mbar_try_wait_cluster(&sh.recv_bar, 0))) {
               if (*abortp) break;
-              if (global_timer_ns() - t0 > kWaitLimitNs) {
+              if (global_timer_ns() - t0 > wait_limit_ns(g.status)) {
                 *abortp = 1;
                 atomicCAS(g.status, 0, (int)ERR_EPILOGUE);
                 break;

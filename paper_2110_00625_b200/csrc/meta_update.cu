@@ -126,6 +126,8 @@ k_broadcast(float* __restrict__ rep, int64_t stride, const float* __restrict__ w
 // w^j - w~ in ascending j, form v and w~, and one thread sends the two result tiles back and
 // the w~ tile to every replica with bulk stores.  Bytes in flight per SM are set by the ring
 // (tens of KB), not by registers, which is what a pass with 2P+4 concurrent streams needs.
+// What is left of n after the last whole tile is done by the consumers of the last block with
+// plain loads and stores (the same arithmetic in the same order).
 enum { ERR_META_PRODUCER = 31, ERR_META_CONSUMER = 32 };
 
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes,
@@ -149,11 +151,24 @@ __device__ __forceinline__ void bulk_wait_read_all() {
 __device__ __forceinline__ void mbar_arrive_plain(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc::smem_u32(bar)) : "memory");
 }
+// Barrier 1 over the `threads` consumer threads that also ORs a predicate over them: every
+// consumer learns whether any of them gave up a wait, so that they all leave the tile loop in the
+// same iteration and nobody is left behind at a counted barrier.
+__device__ __forceinline__ bool consumers_any(bool pred, int threads) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+      "barrier.red.or.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)pred), "r"(threads)
+      : "memory");
+  return r != 0;
+}
 
 template <int T, int G, int STAGES, int THREADS>
 __global__ void __launch_bounds__(THREADS + 32)
 k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ w,
-                   float* __restrict__ v, int P, int64_t n_tiles, float mu, float zeta,
+                   float* __restrict__ v, int P, int64_t n, float mu, float zeta,
                    float inv_p, int read_v, int bcast, int* status) {
   extern __shared__ __align__(128) uint8_t sm[];
   float* st_rep = reinterpret_cast<float*>(sm);            // [STAGES][G][T]
@@ -164,6 +179,7 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
   constexpr int kWarps = THREADS / 32;
   constexpr int PER = T / THREADS;                          // elements per thread, multiple of 4
   const int tid = threadIdx.x;
+  const int64_t n_tiles = n / T;
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
       tc::mbar_init(&full[s], 1);
@@ -204,11 +220,14 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
     }
     return;
   }
+  // Consumers.  A consumer whose wait is abandoned does not leave on its own: it carries `failed`
+  // to the tile's first barrier, which tells every consumer, and they all leave together there
+  // (before anything of the tile is stored).  The producer's waits end through abort_flag.
   uint32_t sc = 0, tcount = 0;
   const int lane = tid & 31;
   for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tcount) {
     const int b = tcount & 1;
-    if (!tc::mbar_wait(&wv_full[b], (tcount >> 1) & 1, abortp, status, ERR_META_CONSUMER)) return;
+    bool failed = !tc::mbar_wait(&wv_full[b], (tcount >> 1) & 1, abortp, status, ERR_META_CONSUMER);
     float wt[PER], acc[PER];
 #pragma unroll
     for (int i = 0; i < PER; i += 4) {
@@ -217,9 +236,12 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
       wt[i] = x.x; wt[i + 1] = x.y; wt[i + 2] = x.z; wt[i + 3] = x.w;
       acc[i] = acc[i + 1] = acc[i + 2] = acc[i + 3] = 0.f;
     }
-    for (int gi = 0; gi < groups; ++gi, ++sc) {
+    for (int gi = 0; gi < groups && !failed; ++gi, ++sc) {
       const int s = sc % STAGES;
-      if (!tc::mbar_wait(&full[s], (sc / STAGES) & 1, abortp, status, ERR_META_CONSUMER)) return;
+      if (!tc::mbar_wait(&full[s], (sc / STAGES) & 1, abortp, status, ERR_META_CONSUMER)) {
+        failed = true;
+        break;
+      }
       const int cnt = min(G, P - gi * G);
       for (int u = 0; u < cnt; ++u) {                       // ascending j
 #pragma unroll
@@ -237,7 +259,7 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
     }
     // the result buffers of the tile before last must have been read by their stores
     if (tid == 0) bulk_wait_read_all();
-    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
+    if (consumers_any(failed, THREADS)) break;
 #pragma unroll
     for (int i = 0; i < PER; i += 4) {
       float4 vt = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -267,22 +289,51 @@ k_meta_update_bulk(float* __restrict__ rep, int64_t stride, float* __restrict__ 
     }
   }
   if (tid == 0) bulk_wait_read_all();
+  // the ragged end of the vector: fewer than T elements, by the last block's consumers
+  if (blockIdx.x == gridDim.x - 1) {
+    const int64_t i0 = n_tiles * T;
+    const int64_t rest4 = (n - i0) >> 2;
+    for (int64_t q = tid; q < rest4; q += THREADS) {
+      const int64_t i = i0 + 4 * q;
+      const float4 wt = *reinterpret_cast<const float4*>(w + i);
+      float4 vt = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (read_v) vt = *reinterpret_cast<const float4*>(v + i);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int j = 0; j < P; ++j)
+        acc4(acc, sub4(*reinterpret_cast<const float4*>(rep + (size_t)j * stride + i), wt));
+      float4 vn, wn;
+      vn.x = fmaf(mu, vt.x, zeta * (acc.x * inv_p));
+      vn.y = fmaf(mu, vt.y, zeta * (acc.y * inv_p));
+      vn.z = fmaf(mu, vt.z, zeta * (acc.z * inv_p));
+      vn.w = fmaf(mu, vt.w, zeta * (acc.w * inv_p));
+      wn.x = wt.x + vn.x; wn.y = wt.y + vn.y; wn.z = wt.z + vn.z; wn.w = wt.w + vn.w;
+      *reinterpret_cast<float4*>(v + i) = vn;
+      *reinterpret_cast<float4*>(w + i) = wn;
+      if (bcast)
+        for (int j = 0; j < P; ++j) *reinterpret_cast<float4*>(rep + (size_t)j * stride + i) = wn;
+    }
+    if (tid < (n & 3))
+      meta_scalar(rep, stride, w, v, P, (n & ~(int64_t)3) + tid, mu, zeta, inv_p, read_v != 0,
+                  bcast != 0);
+  }
 }
 
+// The opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the kernel.
 template <int T, int G, int STAGES, int THREADS>
-cudaError_t launch_bulk(mavg_ctx* c, int64_t n_tiles, float mu, float zeta, float inv_p,
-                        int read_v, int bcast) {
+cudaError_t launch_bulk(mavg_ctx* c, float mu, float zeta, float inv_p, int read_v, int bcast) {
   const size_t smem = ((size_t)STAGES * G * T + 8 * (size_t)T) * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static uint64_t attr_set[4] = {0, 0, 0, 0};   // one bit per device ordinal (< 256)
+  const int dev = c->device & 255;
+  if (!(attr_set[dev >> 6] >> (dev & 63) & 1)) {
     cudaError_t e = cudaFuncSetAttribute(k_meta_update_bulk<T, G, STAGES, THREADS>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev >> 6] |= (uint64_t)1 << (dev & 63);
   }
+  const int64_t n_tiles = c->cfg.n / T;
   const int grid = (int)(n_tiles < c->sm_count ? n_tiles : c->sm_count);
   k_meta_update_bulk<T, G, STAGES, THREADS><<<grid, THREADS + 32, smem, c->stream>>>(
-      c->buf.replicas, c->buf.replica_stride, c->buf.global_w, c->buf.momentum, c->cfg.P, n_tiles,
+      c->buf.replicas, c->buf.replica_stride, c->buf.global_w, c->buf.momentum, c->cfg.P, c->cfg.n,
       mu, zeta, inv_p, read_v, bcast, (int*)ws_ptr(c, c->ws.status));
   return cudaGetLastError();
 }
@@ -319,39 +370,36 @@ cudaError_t launch_meta_update(mavg_ctx* c) {
   const int bcast = c->cfg.defer_broadcast ? 0 : 1;
   c->replicas_materialized = bcast != 0;
   // A replica set that fits in L2 is about to be re-read by the next round's first local step:
-  // it takes the plain-store kernel, which leaves it there.  Larger sets with more than 8
-  // replicas go through the bulk-copy kernel tile by tile (measured faster from P = 16 up; with
-  // few replicas the register kernel already keeps enough loads in flight); what is left of n
-  // after the last whole tile, short vectors and small P take the register kernel with
-  // evict-first stores.
+  // it takes the register kernel with plain stores, which leaves it there (and writes the bf16
+  // copy of w~ on the way where a tensor-core handle asks for it).  Larger sets go through the
+  // bulk-copy kernel, whose ring shape is picked by P (measured at n = 11.2 M on a B200: each of
+  // the three is the fastest, by 2-8 %, in its range; the register kernel with evict-first
+  // stores was 3-8 % behind them at every P from 4 to 64).
   const bool big = (size_t)P * (size_t)n * 4 > c->l2_bytes / 2;
-  int64_t done = 0;
   prof_begin(c, MAVG_K_META);
   cudaError_t e = cudaSuccess;
-  if (big && P > 8 && n >= (int64_t)4096 * c->sm_count * 4) {
-    done = n / 4096 * 4096;
-    e = launch_bulk<4096, 2, 3, 512>(c, n / 4096, mu, zeta, inv_p, read_v, bcast);
-  }
-  if (e == cudaSuccess && done < n) {
-    const int64_t rest = n - done;
-    int grid = grid_for(c, rest >> 2, 256, 8);
-    float* rep = c->buf.replicas + done;
-    float* w = c->buf.global_w + done;
-    float* v = c->buf.momentum + done;
-    c->shadow_fresh = false;
+  c->shadow_fresh = false;
+  if (big && n >= (int64_t)4096 * c->sm_count * 4) {
+    if (P <= 4) e = launch_bulk<2048, 4, 3, 256>(c, mu, zeta, inv_p, read_v, bcast);
+    else if (P <= 8 || P >= 24) e = launch_bulk<2048, 6, 2, 512>(c, mu, zeta, inv_p, read_v, bcast);
+    else e = launch_bulk<4096, 3, 2, 512>(c, mu, zeta, inv_p, read_v, bcast);
+  } else {
+    int grid = grid_for(c, n >> 2, 256, 8);
+    float* rep = c->buf.replicas;
+    float* w = c->buf.global_w;
+    float* v = c->buf.momentum;
     if (big)
       k_meta_update<8, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
-                                                          rest, mu, zeta, inv_p, read_v, bcast);
-    else if (c->shadow.dst && done == 0) {
+                                                          n, mu, zeta, inv_p, read_v, bcast);
+    else if (c->shadow.dst) {
       k_meta_update<8, false, true><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
-                                                                 rest, mu, zeta, inv_p, read_v, bcast,
+                                                                 n, mu, zeta, inv_p, read_v, bcast,
                                                                  c->shadow);
       c->shadow_fresh = true;
     } else
       k_meta_update<8, false><<<grid, 256, 0, c->stream>>>(rep, c->buf.replica_stride, w, v, P,
-                                                           rest, mu, zeta, inv_p, read_v, bcast);
+                                                           n, mu, zeta, inv_p, read_v, bcast);
     e = cudaGetLastError();
-    if (done > 0) c->launches++;
   }
   prof_end(c);
   return e;

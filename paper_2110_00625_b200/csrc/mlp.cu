@@ -57,11 +57,6 @@ namespace {
 __global__ void k_set_round(int64_t* dst, int64_t round) { *dst = round; }
 
 cudaError_t run_steps(mavg_ctx* c, int64_t round) {
-  // the CUDA-core path reads every learner's own copy from the first step on
-  if (!use_tensor_cores(&c->cfg) && c->replicas_equal_global && !c->replicas_materialized) {
-    cudaError_t e = launch_broadcast(c, false, /*force_copies=*/true);
-    if (e != cudaSuccess) return e;
-  }
   for (int k = 1; k <= c->cfg.K; ++k) {
     cudaError_t e = use_tensor_cores(&c->cfg) ? tc_step(c, round, k) : simt_step(c, round, k);
     if (e != cudaSuccess) return e;
@@ -135,6 +130,14 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
     if (e != cudaSuccess) return e;
     c->replicas_equal_global = false;
     return cudaSuccess;
+  }
+  // The CUDA-core path reads every learner's own copy from the first step on: a deferred
+  // re-broadcast (Algorithm 1, "set w^j = w~") is carried out here, on the caller's stream and
+  // outside the recorded graph, so that a replay never depends on whether the copies happened to
+  // exist when the graph was recorded.
+  if (!use_tensor_cores(&c->cfg) && c->replicas_equal_global && !c->replicas_materialized) {
+    cudaError_t e = launch_broadcast(c, false, /*force_copies=*/true);
+    if (e != cudaSuccess) return e;
   }
   const bool want_graph = !c->profiling && !c->graph_disabled && c->replicas_equal_global;
   if (!want_graph) return run_steps(c, round);

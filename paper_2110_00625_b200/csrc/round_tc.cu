@@ -107,7 +107,7 @@ __device__ __forceinline__ bool wait_count(const int* ctr, int target, int* stat
   while (ld_acquire(ctr) < target) {
     if ((++spins & 0x3F) == 0) {
       if (*(volatile int*)status != 0) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > wait_limit_ns(status)) {
         atomicCAS(status, 0, (int)ERR_ROUND_DEP);
         return false;
       }

@@ -47,6 +47,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait here
 
+// The limit a wait observes: the handle's status area holds, after the error word status[0], the
+// limit in microseconds in status[1] (0: the default above).  Read only on the slow path.
+__device__ __forceinline__ uint64_t wait_limit_ns(const int* status) {
+  const int us = *reinterpret_cast<const volatile int*>(status + 1);
+  return us > 0 ? (uint64_t)us * 1000ull : kWaitLimitNs;
+}
+
 // Waits for the phase with the given parity.  Returns false if the wait was abandoned: the time
 // limit ran out (then *abort_flag and the global status word are set) or another role of this
 // block had already set *abort_flag.
@@ -58,7 +65,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0x3FF) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > wait_limit_ns(status)) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;

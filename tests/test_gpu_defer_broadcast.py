@@ -152,3 +152,20 @@ def test_mlp_deferred_launch_by_launch_and_round_host():
     a.sync(); b.sync()
     assert _same(a.w, b.w) and _same(a.v, b.v)
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("mode", [0, 2])
+def test_cuda_core_graph_recorded_after_materialize(mode):
+    # CUDA-core path with deferred copies: the graph of a round's local steps is first recorded in
+    # a round whose copies had been written on request just before.  Every later replay must still
+    # start the learners from w~ (the copies are made outside the recorded graph), bit for bit
+    # like a handle that always writes them.
+    m = _mavg()
+    dims = [40, 24, 10] if mode == 0 else [64, 48, 10]
+    a, b = _mlp_pair(m, mode, dims, 16, 3, 2)
+    b.materialize_replicas()          # copies exist when the first round records the graph
+    for r in range(3):
+        a.round(); b.round()
+        a.sync(); b.sync()
+        assert _same(a.w, b.w) and _same(a.v, b.v), r
+    a.close(); b.close()

@@ -1,5 +1,6 @@
-"""The L2 set-aside for the learners' masters (tensor-core MLP handles whose P master copies fit in
-half the L2): it may change speed only.  Rounds with lines released in between give the same bits
+"""The opt-in L2 set-aside for the learners' masters (l2_keep = 1; tensor-core MLP handles whose P
+master copies fit in half the L2): it may change speed only, and a handle that does not ask for it
+leaves the context's limit alone.  Rounds with lines released in between give the same bits
 as rounds without; the context's limit follows the largest request among the live handles and is
 back at its old value when the last of them is closed (checked in a process of its own, where no
 other test's handle is alive)."""
@@ -15,9 +16,10 @@ pytestmark = pytest.mark.gpu
 SEED = 0x211000625
 
 
-def _handle(m, cfg, x, y, w1, P=None):
+def _handle(m, cfg, x, y, w1, P=None, l2_keep=True):
     return m.Mavg(w1, P=P or cfg["P"], K=cfg["K"], local_lr=cfg["gamma"], mu=cfg["mu"], B=cfg["B"],
-                  seed=SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1, x=x, y=y)
+                  seed=SEED, objective=m.OBJ_MLP, dims=cfg["dims"], gemm_bf16=1, x=x, y=y,
+                  l2_keep=l2_keep)
 
 
 def _small():
@@ -33,13 +35,17 @@ def test_release_keeps_the_bits():
     m, cfg, x, y, w1 = _small()
     a = _handle(m, cfg, x, y, w1)
     b = _handle(m, cfg, x, y, w1)
+    c = _handle(m, cfg, x, y, w1, l2_keep=False)
     for _ in range(3):
         a.round()
         b.round()
         b.l2_release()
-    a.sync(); b.sync()
-    assert np.array_equal(a.w.cpu().numpy(), b.w.cpu().numpy())
-    assert np.array_equal(a.v.cpu().numpy(), b.v.cpu().numpy())
+        c.round()
+    a.sync(); b.sync(); c.sync()
+    for other in (b, c):
+        assert np.array_equal(a.w.cpu().numpy(), other.w.cpu().numpy())
+        assert np.array_equal(a.v.cpu().numpy(), other.v.cpu().numpy())
+    c.close()
     b.close()
     a.close()
 
@@ -60,6 +66,10 @@ CHILD = textwrap.dedent("""
     err, most = cudart.cudaDeviceGetAttribute(cudart.cudaDeviceAttr.cudaDevAttrMaxPersistingL2CacheSize, 0)
     m, cfg, x, y, w1 = _small()
     before = limit()
+    z = _handle(m, cfg, x, y, w1, P=3, l2_keep=False)   # the default: limit untouched
+    assert limit() == before
+    z.round(); z.sync(); z.close()
+    assert limit() == before
     a = _handle(m, cfg, x, y, w1, P=3)
     la = limit()
     b = _handle(m, cfg, x, y, w1, P=8)

@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from tests.util import l2_rel, outlier_fraction, rel_err
+from tests.util import assert_tiles_close, l2_rel, outlier_fraction, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -116,7 +116,12 @@ def test_bf16_small_cifar_shaped(oracle, mode):
         lo, _ = o.run_round()
         assert abs(lg - lo) <= 2e-2 * abs(lo), (r, lg, lo)
         assert rel_err(g.w.cpu().numpy(), o.w) <= 5e-2, r
-        _check_update(g.v.cpu().numpy(), o.v, l2_tol=5e-2, frac=None)   # free-running: drift adds up
+        # free-running rounds: the drift of single bf16 roundings adds up over the steps, so v is
+        # held in the 2-norm and, element by element, to a bounded share of outliers -- overall
+        # and inside every output tile
+        _check_update(g.v.cpu().numpy(), o.v, l2_tol=5e-2, frac=0.02)
+        assert_tiles_close(g.v.cpu().numpy(), o.v, c["dims"], l2_tol=5e-2, frac=0.05,
+                           what=f"v after round {r + 1}")
     g.sync()
 
 
@@ -149,6 +154,7 @@ def test_bf16_teacher_forced_step(oracle):
             step_g = gr[j, :g.n].astype(np.float64) - o.w
             step_o = o.replicas[j, :g.n].astype(np.float64) - o.w
             _check_update(step_g, step_o)
+            assert_tiles_close(step_g, step_o, c["dims"], what=f"mode {mode} learner {j}")
         assert np.abs(g.get_losses() - losses_o).max() <= 2e-3 * losses_o.max()
         g.close()
 
@@ -252,6 +258,9 @@ def test_tc_shapes_teacher_forced(oracle, dims, B, P, K):
         step_g = gr[j, :g.n].astype(np.float64) - w1
         step_o = o.replicas[j, :g.n].astype(np.float64) - w1
         assert l2_rel(step_g, step_o) <= 3e-2, j
+        # every 128 x 32 output tile of every layer and every bias vector on its own: a wrong
+        # edge tile, contraction tail or split fix-up cannot hide in the norm of the whole step
+        assert_tiles_close(step_g, step_o, dims, what=f"learner {j}")
     lg = g.round(want_loss=True)       # and a full round on top: finite, graph path
     assert np.isfinite(lg) and torch.isfinite(g.w).all()
     g.close()

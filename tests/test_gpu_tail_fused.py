@@ -7,7 +7,7 @@ after one step from identical weights they must agree far more tightly than the 
 import numpy as np
 import pytest
 
-from tests.util import l2_rel, rel_err
+from tests.util import assert_tiles_close, l2_rel, outlier_fraction, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -61,6 +61,7 @@ def test_one_step_agrees_with_the_tensor_core_last_layer(shape):
         w0 = a.w.cpu().numpy()
         assert l2_rel(ra[j] - w0, rb[j] - w0) <= 5e-3, j
         assert rel_err(ra[j], rb[j]) <= 1e-3, j
+        assert_tiles_close(ra[j] - w0, rb[j] - w0, cfg["dims"], what=f"learner {j}")
     a.close(); b.close()
 
 
@@ -76,6 +77,9 @@ def test_rounds_against_the_oracle(oracle, dims, P, B):
         assert abs(lg - lo) <= 2e-2 * abs(lo), (r, lg, lo)
         assert rel_err(g.w.cpu().numpy(), o.w) <= 5e-2, r
         assert l2_rel(g.v.cpu().numpy(), o.v) <= 5e-2, r
+        assert outlier_fraction(g.v.cpu().numpy(), o.v, 5e-2) <= 0.02, r
+        assert_tiles_close(g.v.cpu().numpy(), o.v, dims, l2_tol=5e-2, frac=0.05,
+                           what=f"v after round {r + 1}")
     g.close()
 
 

@@ -26,3 +26,54 @@ def l2_rel(x, y):
     x = np.asarray(x, dtype=np.float64).reshape(-1)
     y = np.asarray(y, dtype=np.float64).reshape(-1)
     return float(np.linalg.norm(x - y) / max(np.linalg.norm(y), 1e-30))
+
+
+def mlp_layout(dims):
+    """[(w_off, out, in, b_off)] of the flat per-replica layout [W_1 (out x in), b_1, W_2, ...]."""
+    out, off = [], 0
+    for l in range(len(dims) - 1):
+        i, o = dims[l], dims[l + 1]
+        out.append((off, o, i, off + o * i))
+        off += o * i + o
+    return out
+
+
+def tile_errors(got, want, dims, tile=(128, 32), out_tol=5e-2):
+    """Per output tile of every weight matrix (tile[0] rows x tile[1] columns, the unit a block of
+    the tensor-core kernels produces) and per bias vector: (label, l2 error, outlier fraction).
+    The l2 error of a tile is ||got - want|| over max(||want||, a quarter of what a tile of the
+    layer's rms magnitude would weigh) -- the floor keeps tiles that are (nearly) all zero, e.g.
+    rows of dead hidden units, from dividing by nothing.  Outliers are elements whose error
+    exceeds out_tol of max(|want_i|, rms of the layer)."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    want = np.asarray(want, dtype=np.float64).reshape(-1)
+    res = []
+    for l, (w_off, o, i, b_off) in enumerate(mlp_layout(dims), start=1):
+        G = got[w_off:w_off + o * i].reshape(o, i)
+        W = want[w_off:w_off + o * i].reshape(o, i)
+        rms = max(float(np.sqrt(np.mean(W * W))), 1e-30)
+        for r0 in range(0, o, tile[0]):
+            for c0 in range(0, i, tile[1]):
+                g = G[r0:r0 + tile[0], c0:c0 + tile[1]]
+                w = W[r0:r0 + tile[0], c0:c0 + tile[1]]
+                den = max(float(np.linalg.norm(w)), 0.25 * rms * np.sqrt(w.size))
+                frac = float(np.mean(np.abs(g - w) / np.maximum(np.abs(w), rms) > out_tol))
+                res.append((f"W{l}[{r0}:{r0 + tile[0]},{c0}:{c0 + tile[1]}]",
+                            float(np.linalg.norm(g - w)) / den, frac))
+        gb, wb = got[b_off:b_off + o], want[b_off:b_off + o]
+        rb = max(float(np.sqrt(np.mean(wb * wb))), 1e-30)
+        den = max(float(np.linalg.norm(wb)), 0.25 * rb * np.sqrt(o))
+        frac = float(np.mean(np.abs(gb - wb) / np.maximum(np.abs(wb), rb) > out_tol))
+        res.append((f"b{l}", float(np.linalg.norm(gb - wb)) / den, frac))
+    return res
+
+
+def assert_tiles_close(got, want, dims, l2_tol=2e-2, out_tol=5e-2, frac=0.02, tile=(128, 32),
+                       what=""):
+    """Every tile and every bias vector within l2_tol in the 2-norm and with at most `frac` of its
+    elements beyond out_tol: one wrong edge tile fails, however small its share of the layer."""
+    bad = [(lab, e, f) for lab, e, f in tile_errors(got, want, dims, tile, out_tol)
+           if e > l2_tol or f > frac]
+    assert not bad, f"{what}: {len(bad)} tile(s) off, worst first: " + \
+        ", ".join(f"{lab} l2={e:.3g} out={f:.3g}" for lab, e, f in
+                  sorted(bad, key=lambda t: -t[1])[:4])

@@ -303,7 +303,7 @@ def pseudograd_rounds(args, m, torch, peaks, Ks, steps):
     per K the local pass, the meta-update and the whole round."""
     from paper_2110_00625_b200 import workloads as W
     cfg = W.CONFIGS["C5"]
-    n, P = cfg["n"], cfg["P"]
+    n, P = args.n or cfg["n"], cfg["P"]
     w1 = W.global_model(n)
     out = []
     for K in Ks:
@@ -349,7 +349,8 @@ PSEUDOGRAD_ALU_PEAK_VARIATES = 148 * 4 * 32 * 1.965e9 / PSEUDOGRAD_INSTR_PER_VAR
 
 def run_pseudograd(args, m, torch, peaks, rank):
     from paper_2110_00625_b200 import workloads as W
-    out = pseudograd_rounds(args, m, torch, peaks, W.CONFIGS["C5"]["K"], args.steps)
+    Ks = [int(k) for k in args.ks.split(",")] if args.ks else W.CONFIGS["C5"]["K"]
+    out = pseudograd_rounds(args, m, torch, peaks, Ks, args.steps)
     if rank == 0:
         print(json.dumps({"workload": "C5 full round, n=25.6M fp32, P=16, seeded pseudo-gradients",
                           "steps": args.steps, "results": out}))
@@ -587,6 +588,9 @@ def main():
                          "main workload, or C5 (pseudo-gradient round at 25.6 M parameters) alone")
     ap.add_argument("--learners", type=int, default=0,
                     help="override P (for small profiler captures; not a benchmark setting)")
+    ap.add_argument("--n", type=int, default=0,
+                    help="override the vector length of --workload C5 (small profiler captures)")
+    ap.add_argument("--ks", default="", help="comma-separated K values for --workload C5")
     ap.add_argument("--sweep-only", action="store_true",
                     help="run only the meta-update sweep (profiler captures)")
     ap.add_argument("--beta", type=float, default=0.0,

@@ -23,7 +23,6 @@
 
 #include <algorithm>
 
-#include "gemm_sk.cuh"
 #include "gemm_unit.cuh"
 #include "mlp.cuh"
 #include "tc_ptx.cuh"
@@ -173,27 +172,6 @@ GemmPlan plan_partial(int M, int N, int K, int P, int sm_count, bool tile_n) {
   return g;
 }
 
-// Plan of the persistent launch for a forward / dgrad product whose default plan `base` is one
-// unsplit tile per (learner, 128 rows) with the whole batch as its N tile, or use = 0: it pays
-// where those tiles outnumber the SMs (tile counts that do not divide by the SM count then cost
-// a partly empty last wave, and every tile its own pipeline fill and drain).
-SkPlan plan_sk(int M, int B, int K, int P, int sm_count, const GemmPlan& base) {
-  SkPlan s{};
-  if (base.splits != 1 || base.n_tiles != 1 || base.BN != B || B > 128) return s;
-  if ((long)P * base.m_tiles < sm_count) return s;
-  s.nkb = (K + kBK - 1) / kBK;
-  if (s.nkb < 4) return s;
-  s.mt2 = (M + kSkRows - 1) / kSkRows;
-  s.total = (long long)P * s.mt2 * s.nkb;
-  s.grid = (int)std::min<long long>(sm_count, s.total);
-  const int stage_bytes = 2 * kATileBytes + B * kBK * 2;
-  s.stages = std::min(kMaxStages, (216 * 1024) / stage_bytes);
-  s.tmem_cols = 32;
-  while ((int)s.tmem_cols < 4 * B) s.tmem_cols <<= 1;
-  s.use = 1;
-  return s;
-}
-
 TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   TcLayout t{};
   const int L = cfg->n_layers, P = cfg->P, B = cfg->B;
@@ -245,28 +223,6 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
   t.w16b_stride = L >= 3 ? (int64_t)up((size_t)cfg->dims[L - 2] * cfg->dims[L - 1], 64) : 0;
   t.w16b = take(L >= 3 ? (size_t)P * t.w16b_stride * 2 : 16);
-  {
-    // persistent forward / dgrad launches: two partial-tile slots per block, a counter per tile
-    size_t part = 16, ctr = 16;
-    for (int l = 1; l <= L; ++l) {
-      SkPlan f{}, d{};
-      if (l < L)
-        f = plan_sk(cfg->dims[l], B, cfg->dims[l - 1], P, sm_count,
-                    plan_partial(cfg->dims[l], B, cfg->dims[l - 1], P, sm_count, true));
-      if (l > 1)
-        d = plan_sk(cfg->dims[l - 1], B, cfg->dims[l], P, sm_count,
-                    plan_partial(cfg->dims[l - 1], B, cfg->dims[l], P, sm_count, false));
-      for (const SkPlan& s : {f, d})
-        if (s.use) {
-          part = std::max(part, (size_t)2 * s.grid * B * kSkRows * sizeof(float));
-          ctr = std::max(ctr, (size_t)P * s.mt2 * sizeof(int));
-        }
-    }
-    t.sk_part_bytes = part;
-    t.sk_part = take(part);
-    t.sk_ctr_bytes = ctr;
-    t.sk_ctr = take(ctr);
-  }
   t.end = off;
   return t;
 }
@@ -399,41 +355,6 @@ cudaError_t launch_gemm_ks(mavg_ctx* c, const CUtensorMap& a, const CUtensorMap&
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <int EPI>
-cudaError_t launch_gemm_sk(mavg_ctx* c, int cls, const CUtensorMap& a, const CUtensorMap& b,
-                           const SkPlan& pl, const TcArgs& t) {
-  TcState* st = (TcState*)c->mlp;
-  char* ws = (char*)c->buf.workspace;
-  SkArgs g{};
-  g.M = t.M; g.N = t.N;
-  g.mt2 = pl.mt2; g.nkb = pl.nkb; g.stages = pl.stages; g.P = c->cfg.P; g.total = pl.total;
-  g.a_batched = t.a_batched; g.a_mn = t.a_mn;
-  g.tmem_cols = pl.tmem_cols;
-  g.part = (float*)(ws + st->lay.sk_part);
-  g.tile_ctr = (int*)(ws + st->lay.sk_ctr);
-  g.bias_rep = t.bias_rep; g.bias_off = t.bias_off;
-  g.bias_in = t.bias_in; g.bias_in_stride = t.bias_in_stride;
-  g.out_bm = t.out_bm; g.out_mb = t.out_mb; g.mask_mb = t.mask_mb;
-  g.rep_stride = c->buf.replica_stride;
-  g.gamma = c->cfg.local_lr;
-  g.mom = t.mom;
-  g.status = (int*)ws_ptr(c, c->ws.status);
-  cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((unsigned)std::min(pl.grid, c->sm_count));
-  lc.blockDim = dim3(kSkThreads);
-  lc.dynamicSmemBytes = (size_t)pl.stages * (2 * kATileBytes + t.N * kBK * 2) + 1024;
-  lc.stream = c->stream;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = at;
-  lc.numAttrs = 1;
-  prof_begin(c, cls);
-  cudaError_t e = cudaLaunchKernelEx(&lc, k_tc_gemm_sk<EPI>, a, b, g);
-  prof_end(c);
-  return e != cudaSuccess ? e : cudaGetLastError();
-}
-
 }  // namespace
 
 bool tc_shapes_ok(const mavg_config* cfg, std::string* why) {
@@ -485,11 +406,8 @@ mavg_status tc_setup(mavg_ctx* c) {
     st->fwd_ks[l] = GemmPlan{};
     st->fwd_ks[l].splits = 1;
     if (l < L) st->fwd_ks[l] = plan_cluster_split(st->fwd[l], out, B, in);
-    st->fwd_sk[l] = SkPlan{};
-    st->dgrad_sk[l] = SkPlan{};
-    if (l < L) st->fwd_sk[l] = plan_sk(out, B, in, P, kPlanSmCount, st->fwd[l]);
     st->wgrad_mom = c->buf.learner_u != nullptr;
-    st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count, st->wgrad_mom);
+    st->wgrad[l] = plan_wgrad_stream(out, in, B, P, c->sm_count, st->wgrad_mom, !masters_fit_l2(c));
     if (st->wgrad_mom)
       ok = ok && encode_any(st, &st->u32[l], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
                             c->buf.learner_u + c->layers[l - 1].w_off, in, out, P, in,
@@ -544,7 +462,6 @@ mavg_status tc_setup(mavg_ctx* c) {
                           &why);
     if (l > 1) {
       st->dgrad[l] = plan_partial(in, B, out, P, kPlanSmCount, false);
-      st->dgrad_sk[l] = plan_sk(in, B, out, P, kPlanSmCount, st->dgrad[l]);
       ok = ok && encode_map(st, &st->dz[l], bf(t.dz[l]), out, B, P, dz_ld, (int64_t)B * dz_ld,
                             st->dgrad[l].BN, &why);
     }
@@ -559,8 +476,7 @@ mavg_status tc_setup(mavg_ctx* c) {
   const void* kernels[] = {(const void*)k_tc_gemm<EPI_FWD_HIDDEN, 1>, (const void*)k_tc_gemm<EPI_FWD_HIDDEN, 2>,
                            (const void*)k_tc_gemm<EPI_FWD_LAST, 1>,   (const void*)k_tc_gemm<EPI_FWD_LAST, 2>,
                            (const void*)k_tc_gemm<EPI_DGRAD, 1>,      (const void*)k_tc_gemm<EPI_DGRAD, 2>,
-                           (const void*)k_tc_gemm_ks, (const void*)k_tc_gemm_sk<EPI_FWD_HIDDEN>,
-                           (const void*)k_tc_gemm_sk<EPI_DGRAD>};
+                           (const void*)k_tc_gemm_ks};
   for (const void* k : kernels)
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
@@ -596,7 +512,7 @@ mavg_status tc_setup(mavg_ctx* c) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ws + t.counters, 0, t.counters_bytes, c->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ws + t.sk_ctr, 0, t.sk_ctr_bytes, c->stream);
+
   if (e != cudaSuccess) {
     c->err = std::string("tensor-core path set-up: ") + cudaGetErrorString(e);
     cudaGetLastError();   // reported here; do not leave it pending for a later call
@@ -727,8 +643,6 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
       if (c->schedule == 0 && st->fwd_ks[l].splits > 1)
         TC_TRY(launch_gemm_ks(c, wm, l == 1 ? st->x_in_ks[xb] : st->act_in_ks[l], st->fwd_ks[l], g));
-      else if (c->schedule == 0 && st->fwd_sk[l].use && st->fwd_sk[l].grid <= c->sm_count)
-        TC_TRY(launch_gemm_sk<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd_sk[l], g));
       else
         TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
     } else if (fused_tail) {
@@ -798,12 +712,8 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.mask_mb = bfp(t.act_t[l - 1]);
       g.a_mn = 1;
       g.mom = mom;
-      if (c->schedule == 0 && st->dgrad_sk[l].use && st->dgrad_sk[l].grid <= c->sm_count)
-        TC_TRY(launch_gemm_sk<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : w_mn(l),
-                                         st->dz[l], st->dgrad_sk[l], g));
-      else
-        TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : w_mn(l),
-                                      st->dz[l], st->dgrad[l], g));
+      TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : w_mn(l),
+                                    st->dz[l], st->dgrad[l], g));
     }
     const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
     if (merged) continue;        // all layers' weight gradients follow in one launch

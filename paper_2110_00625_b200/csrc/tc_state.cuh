@@ -23,14 +23,9 @@ struct TcLayout {
   size_t tail_part;                          // partial sums of the fused last-layer kernel
   size_t w16b;                               // second bf16 copy of layer L-1's weights [P, w16b_stride]
   int64_t w16b_stride;
-  size_t sk_part, sk_part_bytes;             // partial tiles and tile counters of the persistent
-  size_t sk_ctr, sk_ctr_bytes;               // forward / dgrad launch (gemm_sk.cuh)
   size_t end;
 };
 
-// Persistent forward / dgrad launch (gemm_sk.cuh): use == 0 where the product keeps the
-// one-tile-per-block kernel.
-struct SkPlan { int use, mt2, nkb, stages, grid; uint32_t tmem_cols; long long total; };
 
 struct GemmPlan { int m_tiles, n_tiles, splits, kb_per_split, nkb, BN, stages, two_per_sm; uint32_t tmem_cols; };
 
@@ -72,7 +67,6 @@ struct TcState {
   int round_stages = 0, round_grid = 0;
   size_t round_smem = 0;
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
-  SkPlan fwd_sk[MAVG_MAX_LAYERS + 1], dgrad_sk[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap
   cudaStream_t s_wgrad = nullptr, s_gather = nullptr;

@@ -128,7 +128,28 @@ k_wgrad_sgd_multi(const __grid_constant__ WgradMultiParams mp) {
 
 }  // namespace
 
-WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum) {
+// longest run of column tiles of one work item
+#ifndef MAVG_WGRAD_CHUNK_CAP
+#define MAVG_WGRAD_CHUNK_CAP 16
+#endif
+constexpr long kWgradChunkCap = MAVG_WGRAD_CHUNK_CAP;
+// deepest ring the plan may choose (at most kMaxSlots)
+#ifndef MAVG_WGRAD_SLOT_CAP
+#define MAVG_WGRAD_SLOT_CAP 6
+#endif
+// the same two for a launch that streams its masters through HBM
+#ifndef MAVG_WGRAD_STREAM_CHUNK
+#define MAVG_WGRAD_STREAM_CHUNK 8
+#endif
+#ifndef MAVG_WGRAD_STREAM_SLOTS
+#define MAVG_WGRAD_STREAM_SLOTS 4
+#endif
+constexpr long kWgradStreamChunk = MAVG_WGRAD_STREAM_CHUNK;
+constexpr int kWgradStreamSlots = MAVG_WGRAD_STREAM_SLOTS;
+constexpr int kWgradSlotCap = MAVG_WGRAD_SLOT_CAP < wgrad::kMaxSlots ? MAVG_WGRAD_SLOT_CAP : wgrad::kMaxSlots;
+
+WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum,
+                            bool streaming) {
   WgradPlan w{};
   w.nkb = (B + kBK - 1) / kBK;
   w.m_tiles = (out + kBM - 1) / kBM;
@@ -136,7 +157,8 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   const long total = (long)P * w.m_tiles * w.n_tiles;
   long chunk = total / (5L * sm_count);
   if (chunk < 1) chunk = 1;
-  if (chunk > 16) chunk = 16;
+  if (chunk > kWgradChunkCap) chunk = kWgradChunkCap;
+  if (streaming && chunk > kWgradStreamChunk) chunk = kWgradStreamChunk;
   if (chunk > w.n_tiles) chunk = w.n_tiles;
   w.chunk = (int)chunk;
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
@@ -152,7 +174,8 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
     w.a_bufs = 1;
     w.slots = (budget - a_bytes) / slot_bytes;
   }
-  if (w.slots > kMaxSlots) w.slots = kMaxSlots;
+  if (w.slots > kWgradSlotCap) w.slots = kWgradSlotCap;
+  if (streaming && w.slots > kWgradStreamSlots) w.slots = kWgradStreamSlots;
   w.smem = (size_t)w.a_bufs * a_bytes + (size_t)w.slots * slot_bytes + 1024;
   w.grid = w.items < sm_count ? w.items : sm_count;
   return w;

@@ -14,7 +14,12 @@ struct WgradPlan {
 constexpr int kWgradTileRows = 128;   // rows of out per tile (box rows of the dZ^T and master maps)
 constexpr int kWgradTileCols = 32;    // columns of in per tile
 
-WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum = false);
+// streaming: the learners' masters do not stay in the L2 from one step to the next, so the kernel
+// is a stream through HBM; the ring is then kept shallow and the runs of column tiles short
+// (measured on the large MLP, B = 64: 4 slots and runs of 4 to 8 tiles give 0.84 of the copy
+// bandwidth against 0.80 with 6 slots and runs of 16, and 0.67 with 3 slots).
+WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum = false,
+                            bool streaming = false);
 cudaError_t wgrad_stream_prepare();
 // dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
 // w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128

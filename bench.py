@@ -340,10 +340,12 @@ def pseudograd_rounds(args, m, torch, peaks, Ks, steps):
     return out
 
 
-# Peak rate of the K-fused pseudo-gradient pass when the integer pipe binds (variates/s): see the
-# derivation in the design document (instructions per variate from the kernel's own count, issue
-# rate of 148 SMs x 4 schedulers x 1 warp instruction per clock at the maximum SM clock).
-PSEUDOGRAD_INSTR_PER_VARIATE = 30.0
+# Peak rate of the K-fused pseudo-gradient pass when instruction issue binds (variates/s): the
+# kernel executes 29.5 instructions per variate (ncu: 4.717e8 warp instructions for 5.12e8
+# variates at n = 2 M, P = 16, K = 16, profiles/pseudograd_k16.md; 64-bit SplitMix64 arithmetic on
+# 32-bit ALUs), against an issue rate of 148 SMs x 4 schedulers x 1 warp instruction (32 lanes)
+# per clock at the maximum SM clock of 1965 MHz.
+PSEUDOGRAD_INSTR_PER_VARIATE = 29.5
 PSEUDOGRAD_ALU_PEAK_VARIATES = 148 * 4 * 32 * 1.965e9 / PSEUDOGRAD_INSTR_PER_VARIATE
 
 

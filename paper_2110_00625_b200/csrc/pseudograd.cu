@@ -10,10 +10,13 @@
 namespace mavg {
 namespace {
 
+// (sum of the four 16-bit lanes of h - 131070) * c.  The lane sums are two 2-way 16-bit dot
+// products with the weights (1, 1), chained through their addend, which starts at -131070
+// (modular arithmetic: the same integer as extracting and adding the lanes one by one).
 __device__ __forceinline__ float ih4(uint64_t h, float c) {
-  uint32_t lo = (uint32_t)h, hi = (uint32_t)(h >> 32);
-  int32_t s = (int32_t)((lo & 0xFFFFu) + (lo >> 16) + (hi & 0xFFFFu) + (hi >> 16));
-  return (float)(s - 131070) * c;
+  const uint32_t lo = (uint32_t)h, hi = (uint32_t)(h >> 32);
+  const uint32_t s = __dp2a_lo(hi, 0x0101u, __dp2a_lo(lo, 0x0101u, (uint32_t)-131070));
+  return (float)(int32_t)s * c;
 }
 
 // grid = (x, P); dynamic shared memory holds the K step keys of learner blockIdx.y.

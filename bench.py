@@ -150,6 +150,46 @@ def bounded_oracle_sample(cfg, x, y, w1, budget_s):
     return p_s, k_s, t1
 
 
+def oracle_table():
+    """The oracle timed on this host for every workload of the list (bounded samples where a full
+    round would take minutes), with the threads it used.  Context figures for the results table."""
+    from oracle import oracle as O
+    from paper_2110_00625_b200 import workloads as W
+    cores = O.max_threads()
+    out = {"host_threads_available": cores}
+    # C1: one full round, median of 3
+    cfg, x, y, w1 = workload_inputs("C1")
+    rate, th, times = cpu_oracle_rate(cfg, x, y, w1, cfg["K"], reps=3)
+    out["C1"] = dict(learner_samples_per_s=rate, threads=th, seconds_per_round=statistics.median(times),
+                     sample="full round")
+    for name, budget in (("C2", 15.0), ("C4", 20.0)):
+        cfg, x, y, w1 = workload_inputs(name)
+        p_s, k_s, t1 = bounded_oracle_sample(cfg, x, y, w1, budget)
+        rate, th, times = cpu_oracle_rate(dict(cfg, P=p_s), x, y, w1, k_s)
+        out[name] = dict(learner_samples_per_s=rate, threads=th, seconds=times[0],
+                         single_thread_seconds_per_learner_step=t1,
+                         sample=f"{k_s} of {cfg['K']} local steps on {p_s} of {cfg['P']} learners + meta-update")
+    # C3: the meta-update alone, n = 11.2 M, P = 16 (single thread: the oracle's loop over elements)
+    n, P = W.CONFIGS["C3"]["n"], 16
+    w1 = W.global_model(n)
+    o = O.Mavg(w1, P=P, K=1, gamma=0.1, mu=0.9)
+    o.replicas[:, :n] = w1[None, :] + np.float32(0.1)
+    t0 = time.perf_counter(); o.meta_update(); t = time.perf_counter() - t0
+    out["C3"] = dict(P=P, seconds_per_update=t, gbs=(8 * P + 16) * n / t / 1e9, threads=1,
+                     sample="one meta-update at P = 16")
+    # C5: one full round at K = 1 and K = 4 (local steps over the learners in parallel + meta-update)
+    c5 = W.CONFIGS["C5"]
+    w1 = W.global_model(c5["n"])
+    for K in (1, 4):
+        o = O.Mavg(w1, P=c5["P"], K=K, gamma=c5["gamma"], mu=0.9, seed=W.BASE_SEED,
+                   objective=O.OBJ_PSEUDOGRAD, sigma=c5["sigma"], threads=min(c5["P"], cores))
+        t0 = time.perf_counter(); o.run_round(); t = time.perf_counter() - t0
+        out[f"C5_K{K}"] = dict(seconds_per_round=t, learner_steps_per_s=c5["P"] * K / t,
+                               threads=min(c5["P"], cores), sample="one full round")
+    print(json.dumps({"oracle_table": out}))
+    return 0
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -603,6 +643,8 @@ def main():
                          "product on tensor cores (1 and 2 for comparison)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--oracle-table", action="store_true",
+                    help="time the CPU oracle on every workload of the list (context figures)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other workloads that the default line carries as extra keys")
     ap.add_argument("--l2-keep", action="store_true",
@@ -613,6 +655,8 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "mavg":
         args.warmup = 3
+    if args.oracle_table:
+        return oracle_table()
     if args.impl == "reference":
         return run_reference(args)
     return run_mavg(args)

@@ -144,9 +144,10 @@ def bounded_oracle_sample(cfg, x, y, w1, budget_s):
     _, _, t_cal = cpu_oracle_rate(dict(cfg, P=1), x, y, w1, 1, reps=1)
     t1 = max(t_cal[0], 1e-6)
     threads = min(cfg["P"], O.max_threads())
-    pieces = max(1, int(budget_s / t1 * threads))          # (learner, step) pieces that fit
-    p_s = int(min(cfg["P"], max(1, pieces)))
-    k_s = int(min(cfg["K"], max(1, pieces // p_s)))
+    waves = max(1, int(budget_s / t1))                     # pieces one thread can take in turn
+    p_s = int(min(cfg["P"], threads * waves))              # whole waves of learners over the threads
+    per_step = -(-p_s // threads)                          # waves one local step costs
+    k_s = int(min(cfg["K"], max(1, waves // per_step)))
     return p_s, k_s, t1
 
 
@@ -228,7 +229,9 @@ def run_reference(args):
 # kernels and tile plans) and scaled by 4, since every kernel's traffic is proportional to P.
 NCU_TRAFFIC = {
     "C2": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
-    "C4": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
+    # profiles/step_kernels_c4_p8.md: sums over one step's launches of the class at P = 8, times 4,
+    # divided by the launches of the class (4 weight-gradient, 4 forward, 3 dgrad launches per step)
+    "C4": {"wgrad_sgd_gemm": 1022.16e6, "fwd_gemm": 252.39e6, "dgrad_gemm": 198.53e6},
 }
 
 
@@ -591,9 +594,8 @@ def run_mavg(args):
                                 0: "CUDA cores fp32"}[r["mode"]],
                        "defer_broadcast": not args.no_defer, "learner_momentum": args.beta,
                        "l2_keep": bool(args.l2_keep),
-                       "schedule": ["CUDA graph of per-product launches",
-                                    "one persistent kernel per round",
-                                    "CUDA graph of per-product launches, all on tensor cores"][args.schedule],
+                       "schedule": {0: "CUDA graph of per-product launches",
+                                    2: "CUDA graph of per-product launches, plain tensor-core tiles"}[args.schedule],
                        "l2": "flushed between steps by a 256 MiB memset, outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
@@ -637,10 +639,9 @@ def main():
                     help="run only the meta-update sweep (profiler captures)")
     ap.add_argument("--beta", type=float, default=0.0,
                     help="learner-level momentum (0 = Algorithm 1 as printed, the benchmark setting)")
-    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
-                    help="0: CUDA graph with the fused last-layer kernel (default); 1: the K local "
-                         "steps of a round as one persistent kernel; 2: CUDA graph with every "
-                         "product on tensor cores (1 and 2 for comparison)")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 2],
+                    help="0: the default CUDA graph; 2: the graph with every product as plain "
+                         "tensor-core tiles (for comparison)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--oracle-table", action="store_true",

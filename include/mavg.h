@@ -223,17 +223,15 @@ typedef enum {
 mavg_status mavg_set_profiling(mavg_handle h, int32_t on);
 /* Schedule of the tensor-core MLP learner level (the paper has no counterpart).
  *   MAVG_SCHED_GRAPH (default): one launch per matrix product, the K steps of a round replayed
- *     from a CUDA graph; the last layer (at most 32 classes: forward, loss, dZ_L, its data
- *     gradient and the bias steps) runs as one CUDA-core kernel.
- *   MAVG_SCHED_ROUND_KERNEL: where the shapes allow it (2 to 5 layers, no product that splits its
- *     contraction over blocks, no learner-level momentum), the K local steps of a round run as ONE
- *     persistent kernel whose blocks hand work to each other through counters in the workspace;
- *     other shapes fall back to MAVG_SCHED_GRAPH_TC.
- *   MAVG_SCHED_GRAPH_TC: the graph with every product, the last layer's too, on tensor cores.
- * The last two run the same tiles and compute the same bits; the default differs from them in the
- * summation order of the last layer only.  Profiled rounds (mavg_set_profiling) take the
- * per-launch form of the graph schedules. */
-typedef enum { MAVG_SCHED_GRAPH = 0, MAVG_SCHED_ROUND_KERNEL = 1, MAVG_SCHED_GRAPH_TC = 2 } mavg_schedule;
+ *     from a CUDA graph; where the last layer's tensor-core tiles would leave most of the GPU idle
+ *     (at most 32 classes, few learners) that layer -- forward, loss, dZ_L, its data gradient and
+ *     the bias steps -- runs as one CUDA-core kernel, and hidden-layer forward products may split
+ *     their contraction over a thread-block cluster.
+ *   MAVG_SCHED_GRAPH_TC: the same graph with every product as plain one-tile-per-block
+ *     tensor-core launches.  The two differ in the summation order of the products they run
+ *     differently, nothing else; this one exists for comparison.
+ * Profiled rounds (mavg_set_profiling) take the launch-by-launch form of the chosen schedule. */
+typedef enum { MAVG_SCHED_GRAPH = 0, MAVG_SCHED_GRAPH_TC = 2 } mavg_schedule;
 mavg_status mavg_set_schedule(mavg_handle h, int32_t mode);
 mavg_status mavg_get_profile(mavg_handle h, float *ms, int64_t *launches, int32_t reset);
 

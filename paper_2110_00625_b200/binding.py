@@ -10,7 +10,7 @@ import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 OBJ_NONE, OBJ_PSEUDOGRAD, OBJ_MLP = 0, 1, 2
-SCHED_GRAPH, SCHED_ROUND_KERNEL, SCHED_GRAPH_TC = 0, 1, 2
+SCHED_GRAPH, SCHED_GRAPH_TC = 0, 2
 X_F32, X_BF16 = 0, 1
 MAX_LAYERS = 8
 
@@ -270,8 +270,8 @@ class Mavg:
         self._check(self.lib.mavg_set_profiling(self.handle, int(bool(on))))
 
     def set_schedule(self, mode):
-        """0: CUDA graph with the fused last layer (default); 1: one persistent kernel per round;
-        2: CUDA graph with every product on tensor cores."""
+        """0: CUDA graph with the fused last layer and cluster-split forward where they pay
+        (default); 2: CUDA graph with every product as plain tensor-core tiles."""
         self._check(self.lib.mavg_set_schedule(self.handle, int(mode)))
 
     def get_profile(self, reset=True):

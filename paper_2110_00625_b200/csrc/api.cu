@@ -507,7 +507,8 @@ mavg_status mavg_set_profiling(mavg_handle h, int32_t on) {
 
 mavg_status mavg_set_schedule(mavg_handle h, int32_t mode) {
   CHECK_HANDLE(h);
-  if (mode < 0 || mode > 2) return set_err(h, MAVG_ERR_INVALID_ARG, "schedule must be 0, 1 or 2");
+  if (mode != MAVG_SCHED_GRAPH && mode != MAVG_SCHED_GRAPH_TC)
+    return set_err(h, MAVG_ERR_INVALID_ARG, "schedule must be MAVG_SCHED_GRAPH (0) or MAVG_SCHED_GRAPH_TC (2)");
   h->schedule = mode;
   return MAVG_OK;
 }

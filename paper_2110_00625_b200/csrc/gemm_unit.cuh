@@ -1,7 +1,7 @@
 // One output tile of a forward or dgrad product on tcgen05, with the layer's tail fused: the
 // roles (TMA producer, MMA issuer, epilogue warps) of a block that already has its barriers
-// initialised and its tensor memory allocated.  Shared by the one-tile-per-block kernel of
-// mlp_tc.cu and by the whole-round kernel of round_tc.cu.
+// initialised and its tensor memory allocated.  Used by the one-tile-per-block kernel and the
+// cluster-split kernel of mlp_tc.cu.
 #pragma once
 #include <cuda.h>
 

@@ -124,13 +124,6 @@ cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round) {
   // The usual round starts from the broadcast state and is replayed from a graph.  Rounds that
   // start elsewhere (local steps called twice in a row), profiled rounds and handles whose
   // capture failed once take the launch-by-launch path.
-  // Where the whole-round kernel covers the problem, the K steps are one launch of it.
-  if (use_tensor_cores(&c->cfg) && !c->profiling && c->schedule == 1 && tc_round_supported(c)) {
-    cudaError_t e = tc_round_launch(c, round);
-    if (e != cudaSuccess) return e;
-    c->replicas_equal_global = false;
-    return cudaSuccess;
-  }
   // The CUDA-core path reads every learner's own copy from the first step on: a deferred
   // re-broadcast (Algorithm 1, "set w^j = w~") is carried out here, on the caller's stream and
   // outside the recorded graph, so that a replay never depends on whether the copies happened to

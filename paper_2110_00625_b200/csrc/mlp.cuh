@@ -61,10 +61,6 @@ cudaError_t tail_fused_prepare();
 cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t);    // the products, dZ, partial sums
 cudaError_t launch_tail_finish(mavg_ctx* c, const TailLaunch& t);   // bias steps and loss from the partials
 
-// Whole-round kernel (round_tc.cu): all K local steps of a round in one launch.
-bool tc_round_supported(mavg_ctx* c);
-cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
-
 int tc_get_w16_cur(mavg_ctx* c);            // which bf16 copy of the doubled layer is current
 void tc_set_w16_cur(mavg_ctx* c, int cur);
 

@@ -218,8 +218,6 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.counters = take(t.counters_bytes);
   t.w16 = take((size_t)P * t.n16 * 2);
   t.w16g = take((size_t)t.n16 * 2);
-  t.round_ctr_bytes = (size_t)4 * (MAVG_MAX_LAYERS + 1) * P * sizeof(int);
-  t.round_ctr = take(t.round_ctr_bytes);
   t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
   t.w16b_stride = L >= 3 ? (int64_t)up((size_t)cfg->dims[L - 2] * cfg->dims[L - 1], 64) : 0;
   t.w16b = take(L >= 3 ? (size_t)P * t.w16b_stride * 2 : 16);
@@ -481,7 +479,6 @@ mavg_status tc_setup(mavg_ctx* c) {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
   if (e == cudaSuccess) e = wgrad_stream_prepare();
-  if (e == cudaSuccess) e = tc_round_prepare(c);
   // The fused CUDA-core last layer pays where the tensor-core products of that layer would leave
   // most of the GPU idle (few learners, narrow layer below); with many tiles the tensor-core
   // kernels are the faster ones.

@@ -1,5 +1,5 @@
 // Host-side state of the tensor-core MLP path: workspace layout, launch plans and tensor maps.
-// Built by mlp_tc.cu, also read by the whole-round kernel's launcher (round_tc.cu).
+// Built and used by mlp_tc.cu.
 #pragma once
 #include <cuda.h>
 
@@ -19,7 +19,6 @@ struct TcLayout {
   size_t part, part_bytes;
   size_t counters, counters_bytes;
   size_t w16, w16g;
-  size_t round_ctr, round_ctr_bytes;         // completion counters of the whole-round kernel
   size_t tail_part;                          // partial sums of the fused last-layer kernel
   size_t w16b;                               // second bf16 copy of layer L-1's weights [P, w16b_stride]
   int64_t w16b_stride;
@@ -62,10 +61,6 @@ struct TcState {
   CUtensorMap w_b, w_mn_b, w16_st_b;
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   bool wgrad_merged = false;                  // all layers' weight gradients in one launch
-  // whole-round kernel (round_tc.cu)
-  bool round_ok = false;
-  int round_stages = 0, round_grid = 0;
-  size_t round_smem = 0;
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap
@@ -75,10 +70,6 @@ struct TcState {
 };
 
 
-// round_tc.cu: all K local steps of a round in one persistent kernel.
-bool tc_round_supported(mavg_ctx* c);
-cudaError_t tc_round_prepare(mavg_ctx* c);
-cudaError_t tc_round_launch(mavg_ctx* c, int64_t round);
 int tc_get_w16_cur(mavg_ctx* c);
 void tc_set_w16_cur(mavg_ctx* c, int cur);
 

@@ -71,7 +71,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   const uint32_t tmem_base = sh.tmem_slot;
   grid_dependency_wait();
   wgrad_run<MOM>(tm_dzt, tm_at, tm_w32, tm_w32_in, tm_w16, tm_u, g, (int)blockIdx.x,
-                 (int)gridDim.x, smem, sh, tmem_base, NoDeps());
+                 (int)gridDim.x, smem, sh, tmem_base);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, 64);
@@ -118,7 +118,7 @@ k_wgrad_sgd_multi(const __grid_constant__ WgradMultiParams mp) {
   for (int s = 0; s < mp.n; ++s) {
     const int vb = ((int)blockIdx.x + mp.rot[s]) % grid;
     wgrad_run<MOM>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.g[s], vb,
-                   grid, smem, sh, tmem_base, NoDeps(), tiles, items);
+                   grid, smem, sh, tmem_base, tiles, items);
     wgrad_run_totals(mp.g[s], vb, grid, tiles, items);
   }
   tc_fence_before_sync();

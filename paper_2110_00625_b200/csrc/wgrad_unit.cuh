@@ -1,5 +1,5 @@
-// Roles of the streaming weight-gradient + SGD block (see wgrad_tc.cu for the scheme): shared by
-// the stand-alone kernel and by the whole-round kernel of round_tc.cu.
+// Roles of the streaming weight-gradient + SGD block (see wgrad_tc.cu for the scheme), used by its
+// one-layer and its several-layers kernel.
 #pragma once
 #include <cuda.h>
 
@@ -65,17 +65,6 @@ struct WgradArgs {
 };
 
 
-// Waits until all but the last N store groups of this thread have been written to global memory.
-constexpr int kStoreLag = 4;
-template <int N>
-__device__ __forceinline__ void tma_store_wait_pending() {
-  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
-}
-// Waits until every store group of this thread has been written to global memory.
-__device__ __forceinline__ void tma_store_wait_all() {
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-
 struct WgradShared {
   uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
   uint64_t tmem_full[2], tmem_empty[2];
@@ -109,26 +98,17 @@ __device__ __forceinline__ void wgrad_run_totals(const WgradArgs& g, int vblock,
   }
 }
 
-// Dependency hooks of a run: the producer thread calls inputs_ready(p) before it loads anything
-// of an item of learner p; with kSignals the store thread calls item_done(p) once the item's
-// tiles have reached global memory.  A stand-alone launch needs neither.
-struct NoDeps {
-  static constexpr bool kSignals = false;
-  __device__ __forceinline__ bool inputs_ready(int, volatile int*) const { return true; }
-  __device__ __forceinline__ void item_done(int) const {}
-};
-
 // Work items vblock, vblock + vgrid, ... of the launch described by g.  Barriers initialised
 // (phase 0) and a block-wide barrier passed before; 64 columns of tensor memory at tmem_base.
 // A block that makes several runs keeps using the same barriers (g.slots and g.a_bufs must not
 // change): tile_base and item_base are the tiles and items of its earlier runs, see
 // wgrad_run_totals.
-template <bool MOM, typename Dep>
+template <bool MOM>
 __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUtensorMap& tm_at,
                                           const CUtensorMap& tm_w32, const CUtensorMap& tm_w32_in,
                                           const CUtensorMap& tm_w16, const CUtensorMap& tm_u,
                                           const WgradArgs& g, int vblock, int vgrid, uint8_t* smem,
-                                          WgradShared& sh, uint32_t tmem_base, const Dep& dep,
+                                          WgradShared& sh, uint32_t tmem_base,
                                           uint32_t tile_base = 0, uint32_t item_base = 0) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
@@ -166,7 +146,6 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
         decode(item, p, m0, nt0, nt);
         const int ab = item_ctr % g.a_bufs;
         const uint32_t a_use = item_ctr / g.a_bufs;
-        if (!dep.inputs_ready(p, abortp)) break;
         if (!mbar_wait(&sh.a_empty[ab], (a_use & 1) ^ 1, abortp, g.status, ERR_WG_PRODUCER)) break;
         mbar_arrive_expect_tx(&sh.a_full[ab], (uint32_t)a_bytes);
         for (int kb = 0; kb < g.nkb; ++kb)
@@ -301,13 +280,8 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
     if (lane == 0) {
       uint32_t tile_ctr = tile_base;
       bool ok = true;
-      // items whose tiles have all been handed to the TMA unit but may not have reached global
-      // memory yet: (index after the item's last tile, learner); signalled kStoreLag tiles later
       int held = -1;          // slot whose stores are committed but not yet known to be read
       const uint64_t pol = l2_policy(g.keep_w32 != 0);
-      uint32_t pend_end[8];
-      int pend_p[8];
-      uint32_t ph = 0, pt = 0;
       for (int item = vblock; item < g.items && ok; item += vgrid) {
         int p, m0, nt0, nt;
         decode(item, p, m0, nt0, nt);
@@ -342,28 +316,11 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
               mbar_arrive(&sh.slot_empty[s]);
             }
           }
-          if (Dep::kSignals) {
-            // all but the last kStoreLag store groups are in global memory
-            tma_store_wait_pending<kStoreLag>();
-            while (ph != pt && pend_end[ph & 7] + kStoreLag <= tile_ctr + 1) {
-              dep.item_done(pend_p[ph & 7]);
-              ++ph;
-            }
-          }
-        }
-        if (Dep::kSignals && ok) {
-          pend_end[pt & 7] = tile_ctr;
-          pend_p[pt & 7] = p;
-          ++pt;
         }
       }
       if (held >= 0) {
         tma_store_wait_read<0>();
         mbar_arrive(&sh.slot_empty[held]);
-      }
-      if (Dep::kSignals && ok) {
-        tma_store_wait_all();
-        for (; ph != pt; ++ph) dep.item_done(pend_p[ph & 7]);
       }
     }
     __syncwarp();

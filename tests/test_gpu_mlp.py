@@ -226,6 +226,8 @@ def test_tc_hparam_change_and_repeated_local_steps():
         a.set_hparams(0, 0.05, 1.0, 0.9)
     with pytest.raises(_mavg().MavgError):
         a.set_hparams(2, 0.05, 1.0, 1.0)
+    with pytest.raises(_mavg().MavgError):
+        a.set_schedule(1)               # only MAVG_SCHED_GRAPH (0) and MAVG_SCHED_GRAPH_TC (2) exist
 
 
 @pytest.mark.parametrize("dims,B,P,K", [

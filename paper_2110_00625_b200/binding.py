@@ -133,7 +133,7 @@ def make_config(P, K, local_lr, mu, block_lr=1.0, B=1, seed=0, objective=OBJ_NON
     cfg.defer_broadcast = 1 if defer_broadcast else 0
     cfg.learner_momentum = learner_momentum
     cfg.learner_momentum_reset = 1 if learner_momentum_reset else 0
-    cfg.l2_keep = 1 if l2_keep else 0
+    cfg.l2_keep = int(l2_keep)
     return cfg
 
 

@@ -76,6 +76,37 @@ def test_meta_update_c3_shape_reduced(oracle, P, mu):
     assert rel_err(g.v.cpu().numpy(), o.v) <= META_TOL
 
 
+@pytest.mark.parametrize("n,P,mu,defer", [
+    (6_000_001, 3, 0.9, False),     # ring of 4 replica tiles x 3 stages (P <= 4), n % 4 = 1
+    (2_500_003, 8, 0.0, False),     # ring of 6 x 2 (5 <= P <= 8), v not read, n % 4 = 3
+    (2_500_003, 12, 0.9, True),     # ring of 3 x 2 with 4096-element tiles, copies deferred
+    (2_500_002, 26, 0.9, False),    # ring of 6 x 2 (P >= 24), last group of 2 replicas
+])
+def test_meta_update_bulk_kernel_rings_and_ragged_end(oracle, n, P, mu, defer):
+    # replica sets larger than the L2 with at least 2.4 M elements take the bulk-copy kernel; its
+    # three ring shapes, a last group with fewer replicas than the ring's width, and the end of
+    # the vector that is not a whole tile (nor a whole float4), done inside the same launch
+    m = _mavg()
+    w1 = m.workloads.global_model(n, seed=9)
+    g = m.Mavg(w1, P=P, K=1, local_lr=0.1, mu=mu, objective=m.OBJ_NONE, defer_broadcast=defer)
+    o = oracle.Mavg(w1, P=P, K=1, gamma=0.1, mu=mu, stride=g.stride)
+    for u in range(2):
+        reps = m.workloads.perturbed_replicas(o.w, P, 0.1, update=u, seed=21, stride=g.stride)
+        o.replicas[:] = reps
+        g.replicas.copy_(torch.from_numpy(reps))
+        g.meta_update()
+        o.meta_update()
+    g.sync()
+    assert rel_err(g.w.cpu().numpy(), o.w) <= META_TOL
+    assert rel_err(g.v.cpu().numpy(), o.v) <= META_TOL
+    got = g.replicas.cpu().numpy()
+    if defer:       # the copies are left to the next local step: the array is untouched
+        assert np.array_equal(got[:, :n], reps[:, :n])
+    else:           # every replica is an exact copy of the new global model, ragged end included
+        assert all(np.array_equal(got[j, :n], g.w.cpu().numpy()) for j in (0, P // 2, P - 1))
+    g.close()
+
+
 @pytest.mark.parametrize("K", [1, 4, 16, 64])
 @pytest.mark.parametrize("mu", [0.0, 0.9])
 def test_pseudograd_rounds(oracle, K, mu):
@@ -173,3 +204,20 @@ def test_determinism():
         g.sync()
         outs.append((g.w.cpu().numpy(), g.v.cpu().numpy()))
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_losses_exist_for_the_mlp_objective_only():
+    # a pseudo-gradient handle may raise K far beyond the K its loss buffer was sized for; asking
+    # it for losses must be refused, not served from beyond the buffer
+    m = _mavg()
+    w1 = m.workloads.global_model(1000, seed=2)
+    g = m.Mavg(w1, P=16, K=1, local_lr=0.05, mu=0.9, seed=5, objective=m.OBJ_PSEUDOGRAD, sigma=0.03)
+    g.set_hparams(64, 0.05, 1.0, 0.9)
+    g.round()
+    g.sync()
+    with pytest.raises(m.MavgError) as err:
+        g.get_losses()
+    assert err.value.status == 3          # MAVG_ERR_STATE
+    g.round()                             # the handle is not poisoned by the refusal
+    g.sync()
+    g.close()

@@ -54,6 +54,7 @@ def _cfg(**kw):
     (dict(objective=2, dims=[4, 3], n=15, B=2, x_ptr=256, y_ptr=256, n_samples=2), 1),
     (dict(objective=2, dims=[4, 3], n=15, B=2, x_ptr=264, y_ptr=256, n_samples=10), 2),
     (dict(objective=2, dims=[4, 3], n=15, B=2, x_ptr=256, y_ptr=256, n_samples=10, gemm_bf16=3), 1),
+    (dict(l2_keep=2), 1),                 # a flag: 0 or 1
     # widths that are not multiples of 8 are outside the tensor-core path
     (dict(objective=2, dims=[4, 3], n=15, B=2, x_ptr=256, y_ptr=256, n_samples=10, gemm_bf16=1), 4),
 ])
@@ -98,6 +99,9 @@ def test_workspace_size_and_buffer_checks(lib):
     assert lib.mavg_destroy(None) == 0
     assert lib.mavg_round(None, None) == 1
     assert lib.mavg_sync(None) == 1
+    assert lib.mavg_set_wait_limit(None, 100) == 1
+    assert lib.mavg_selftest_wait(None) == 1
+    assert lib.mavg_set_schedule(None, 0) == 1
 
 
 def test_create_without_a_device_fails_cleanly(lib):

@@ -231,18 +231,28 @@ NCU_TRAFFIC = {
     "C2": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
     # profiles/step_kernels_c4_p8.md: sums over one step's launches of the class at P = 8, times 4,
     # divided by the launches of the class (4 weight-gradient, 4 forward, 3 dgrad launches per step)
-    "C4": {"wgrad_sgd_gemm": 1024.5e6, "fwd_gemm": 252.4e6, "dgrad_gemm": 198.7e6},
+    "C4": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
 }
 
 
-def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False):
+def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=0):
     """Bytes that must cross HBM per ROUND for each kernel class (weights streamed once per
-    product, activations in and out), and their total."""
+    product, activations in and out), and their total.  fwd_run_tiles > 0: in steps 1..K-1 the
+    layer-1 weight-gradient launch also forms the next step's layer-1 forward product (no bf16
+    copy of layer 1 written or read in those steps; instead one fp32 partial sum [128, B] per
+    learner, row tile and run of fwd_run_tiles column tiles, written there and read by the
+    kernel that finishes the layer, and the next batch read once more)."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
     nW = [dims[l] * dims[l + 1] for l in range(L)]
     n = sum(nW) + sum(dims[1:])
     rows = P * B
+    fwd_delta = wgrad_delta = 0
+    if fwd_run_tiles > 0 and K > 1:
+        n_tiles = -(-dims[0] // 32)
+        partial = P * -(-dims[1] // 128) * -(-n_tiles // fwd_run_tiles) * B * 128 * 4
+        fwd_delta = (K - 1) * (partial - 2 * P * nW[0] - 2 * rows * dims[0])
+        wgrad_delta = (K - 1) * (partial - 2 * P * nW[0] + 2 * rows * dims[0])
     per_round = {
         # replicas, w~, v read; v, w~ and (unless the copies are deferred) the replicas written
         "meta_update": dict(bytes=((4 if deferred else 8) * P + 16) * n, flops=0),
@@ -258,12 +268,15 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False):
                                - (4 * (P - 1) * sum(nW) if tensor_path else 0),
                                flops=K * 2 * rows * sum(nW)),
     }
+    per_round["fwd_gemm"]["bytes"] += fwd_delta
+    per_round["wgrad_sgd_gemm"]["bytes"] += wgrad_delta
     return per_round
 
 
-def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False):
+def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False,
+                     fwd_run_tiles=0):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
-    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum)
+    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles)
     out = {}
     for name, (ms, cnt) in prof.items():
         if cnt == 0 or ms <= 0:
@@ -493,8 +506,10 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
         g.round()
     prof = g.get_profile(reset=True)
     g.set_profiling(False)
+    plan = g.get_step_plan()
+    fwd_run_tiles = plan["fwd_run_tiles"] if plan["fwd_with_wgrad"] and args.schedule == 0 else 0
     kern = kernel_rooflines(cfg, prof, psteps, peaks, mode == 1, deferred=not args.no_defer,
-                            momentum=args.beta != 0.0)
+                            momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles)
     n = g.n
     g.close()
     del g, flush
@@ -527,11 +542,11 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
             roof["traffic"] = NCU_TRAFFIC.get(name, {}).get(dom)
     # the whole round against the HBM roofline: every class's algorithmic bytes / the round's time
     per_round = algorithmic_bytes(cfg, mode == 1, deferred=not args.no_defer,
-                                  momentum=args.beta != 0.0)
+                                  momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles)
     round_bytes = sum(v["bytes"] for v in per_round.values())
     ms_round = total_ms / steps
     return dict(
-        cfg=cfg, n=n, units=units, total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
+        cfg=cfg, n=n, units=units, fwd_run_tiles=fwd_run_tiles, total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
         clocks=clocks, cpu=cpu, kern=kern, roof=roof, t_wall=t_wall, mode=mode,
         meta_in_round={"ms": statistics.median(meta_ms),
                        "gbs": per_round["meta_update"]["bytes"] / statistics.median(meta_ms) / 1e6},
@@ -596,6 +611,9 @@ def run_mavg(args):
                        "l2_keep": bool(args.l2_keep),
                        "schedule": {0: "CUDA graph of per-product launches",
                                     2: "CUDA graph of per-product launches, plain tensor-core tiles"}[args.schedule],
+                       "layer1_forward": ("inside the layer's weight-gradient launch of the step before "
+                                          f"(steps 2..K; partial sums per {r['fwd_run_tiles']} column tiles)"
+                                          if r["fwd_run_tiles"] else "a launch of its own"),
                        "l2": "flushed between steps by a 256 MiB memset, outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],

@@ -204,6 +204,21 @@ mavg_status mavg_set_round(mavg_handle h, int64_t round);
 /* Kernels launched by this handle so far. */
 mavg_status mavg_get_launch_count(mavg_handle h, int64_t *count);
 
+/* How one local step of the learner level (Algorithm 1's inner loop) is laid out in launches, for
+ * measurement and tests; out: HOST array of MAVG_PLAN_COUNT entries.  All entries are 0 for
+ * handles without the MLP objective.  MAVG_ERR_INVALID_ARG for a NULL argument. */
+typedef enum {
+  MAVG_PLAN_TENSOR_PATH = 0,    /* 1: the products run on the tensor cores (bf16 operands) */
+  MAVG_PLAN_WGRAD_MERGED = 1,   /* 1: all layers' weight gradients + SGD share one launch */
+  MAVG_PLAN_FWD_WITH_WGRAD = 2, /* 1: under the default schedule, layer 1's weight-gradient launch
+                                   of steps 1..K-1 also forms the next step's layer-1 forward
+                                   product from the updated tiles (no bf16 copy of layer 1 is
+                                   written in those steps) */
+  MAVG_PLAN_FWD_RUN_TILES = 3,  /* with FWD_WITH_WGRAD: column tiles per partial sum */
+  MAVG_PLAN_COUNT = 4
+} mavg_plan_entry;
+mavg_status mavg_get_step_plan(mavg_handle h, int32_t *out);
+
 /* Measurement aid (the paper has no counterpart).  While profiling is on, every kernel launch of
  * this handle is bracketed by a pair of CUDA events on the stream.  mavg_get_profile waits for the
  * stream and returns, per kernel class, the summed device time in milliseconds and the number of

@@ -21,9 +21,10 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_materialize_replicas", "mavg_round", "mavg_round_host", "mavg_set_hparams",
            "mavg_set_learner_momentum", "mavg_get_batch_indices",
            "mavg_get_losses", "mavg_get_round", "mavg_set_round", "mavg_get_launch_count",
-           "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync",
+           "mavg_get_step_plan", "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync",
            "mavg_set_wait_limit", "mavg_selftest_wait", "mavg_cache_release", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
+PLAN_ENTRIES = ["tensor_path", "wgrad_merged", "fwd_with_wgrad", "fwd_run_tiles"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
 
@@ -91,6 +92,7 @@ def load_library():
     L.mavg_get_round.argtypes = [H, C.POINTER(C.c_int64)]
     L.mavg_set_round.argtypes = [H, C.c_int64]
     L.mavg_get_launch_count.argtypes = [H, C.POINTER(C.c_int64)]
+    L.mavg_get_step_plan.argtypes = [H, C.POINTER(C.c_int32)]
     L.mavg_set_profiling.argtypes = [H, C.c_int32]
     L.mavg_set_schedule.argtypes = [H, C.c_int32]
     L.mavg_get_profile.argtypes = [H, C.c_void_p, C.c_void_p, C.c_int32]
@@ -265,6 +267,11 @@ class Mavg:
         r = C.c_int64()
         self.lib.mavg_get_launch_count(self.handle, C.byref(r))
         return r.value
+
+    def get_step_plan(self):
+        out = (C.c_int32 * len(PLAN_ENTRIES))()
+        self._check(self.lib.mavg_get_step_plan(self.handle, out))
+        return dict(zip(PLAN_ENTRIES, out))
 
     def set_profiling(self, on):
         self._check(self.lib.mavg_set_profiling(self.handle, int(bool(on))))

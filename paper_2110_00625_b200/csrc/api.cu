@@ -498,6 +498,13 @@ mavg_status mavg_get_launch_count(mavg_handle h, int64_t* count) {
   return MAVG_OK;
 }
 
+mavg_status mavg_get_step_plan(mavg_handle h, int32_t* out) {
+  if (!h || !out) return MAVG_ERR_INVALID_ARG;
+  for (int i = 0; i < MAVG_PLAN_COUNT; ++i) out[i] = 0;
+  if (h->cfg.objective == MAVG_OBJ_MLP) mlp_step_plan(h, out);
+  return MAVG_OK;
+}
+
 mavg_status mavg_set_profiling(mavg_handle h, int32_t on) {
   CHECK_HANDLE(h);
   h->profiling = on != 0;

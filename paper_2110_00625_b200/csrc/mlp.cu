@@ -47,6 +47,10 @@ void mlp_teardown(mavg_ctx* c) {
   if (c->mlp) tc_teardown(c);
 }
 
+void mlp_step_plan(mavg_ctx* c, int32_t* out) {
+  if (c->mlp) tc_step_plan(c, out);
+}
+
 cudaError_t mlp_refresh_shared_operands(mavg_ctx* c) {
   if (use_tensor_cores(&c->cfg)) return tc_refresh_shared_operands(c);
   return cudaSuccess;

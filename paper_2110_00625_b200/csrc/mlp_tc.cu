@@ -219,6 +219,16 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.w16 = take((size_t)P * t.n16 * 2);
   t.w16g = take((size_t)t.n16 * 2);
   t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
+  {
+    // partial sums of the forward product that rides along with layer 1's weight-gradient launch:
+    // one 128 x B fp32 tile per (learner, row tile, run of column tiles) of that launch's plan
+    t.zpart_bytes = 16;
+    if (L >= 2 && B <= 128) {
+      const WgradPlan w = plan_wgrad_stream(cfg->dims[1], cfg->dims[0], B, P, sm_count, false, true, true);
+      t.zpart_bytes = (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float);
+    }
+    t.zpart = take(t.zpart_bytes);
+  }
   t.w16b_stride = L >= 3 ? (int64_t)up((size_t)cfg->dims[L - 2] * cfg->dims[L - 1], 64) : 0;
   t.w16b = take(L >= 3 ? (size_t)P * t.w16b_stride * 2 : 16);
   t.end = off;
@@ -490,6 +500,26 @@ mavg_status tc_setup(mavg_ctx* c) {
     for (int l = 2; l <= L; ++l)
       if (st->wgrad[l].slots != w1.slots || st->wgrad[l].a_bufs != w1.a_bufs) st->wgrad_merged = false;
   }
+  // Where layer 1's weight gradient is a launch of its own, it can take the next step's forward
+  // product of layer 1 along: the layer's plan gets room for the next step's input tile and long
+  // runs, and the gathered batch buffers get a view with 32-column boxes.
+  st->fuse_f1 = false;
+  if (!st->wgrad_merged && L >= 2 && B <= 128 && ok) {
+    const WgradPlan w = plan_wgrad_stream(cfg.dims[1], cfg.dims[0], B, P, c->sm_count, st->wgrad_mom,
+                                          !masters_fit_l2(c), true);
+    const size_t need = (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float);
+    if (w.slots >= 2 && need <= t.zpart_bytes) {
+      bool enc = true;
+      for (int i = 0; i < 2 && enc; ++i)
+        enc = encode_any(st, &st->x_next[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bf(t.xg[i]),
+                         cfg.dims[0], B, P, cfg.dims[0], (int64_t)B * cfg.dims[0], kWgradTileCols, B,
+                         CU_TENSOR_MAP_SWIZZLE_64B, &why);
+      if (enc) {
+        st->wgrad_f1 = w;
+        st->fuse_f1 = true;
+      }
+    }
+  }
   // the meta-update writes the bf16 copy of w~ itself where its vector kernel takes the whole model
   c->shadow.dst = (__nv_bfloat16*)(ws + t.w16g);
   c->shadow.L = L;
@@ -535,6 +565,15 @@ void tc_teardown(mavg_ctx* c) {
 int tc_get_w16_cur(mavg_ctx* c) { return c->mlp ? ((TcState*)c->mlp)->w16_cur : 0; }
 void tc_set_w16_cur(mavg_ctx* c, int cur) {
   if (c->mlp) ((TcState*)c->mlp)->w16_cur = cur;
+}
+
+void tc_step_plan(mavg_ctx* c, int32_t* out) {
+  const TcState* st = (const TcState*)c->mlp;
+  if (!st) return;
+  out[MAVG_PLAN_TENSOR_PATH] = 1;
+  out[MAVG_PLAN_WGRAD_MERGED] = st->wgrad_merged ? 1 : 0;
+  out[MAVG_PLAN_FWD_WITH_WGRAD] = st->fuse_f1 ? 1 : 0;
+  out[MAVG_PLAN_FWD_RUN_TILES] = st->fuse_f1 ? st->wgrad_f1.chunk : 0;
 }
 
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
@@ -586,6 +625,13 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   const bool fused_tail = st->tail_ok && c->schedule == 0;
   bool tail_on_side = false;
   const bool merged = st->wgrad_merged && c->schedule == 0;
+  // Layer 1's forward product of the NEXT step rides along with this step's weight-gradient
+  // launch of layer 1 (default schedule, that launch standing alone, a next step in this call).
+  // The step after finds the product as partial sums (f1_pending) and only finishes it.
+  const bool fuse_next = st->fuse_f1 && c->schedule == 0 && !merged && step < K;
+  if (step == 1) st->f1_pending = false;
+  const bool f1_here = st->f1_pending;
+  st->f1_pending = false;
   // Weight gradients of the last two layers beside the remaining dgrad products (their dZ comes
   // out of the fused last-layer kernel): layer L-1 then writes the other of its two bf16 copies,
   // because dgrad through it still reads the current one.
@@ -618,7 +664,11 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   // labels and indices are per step as well: they live beside the batch buffer they belong to
   int32_t* idx_b = idx;
   int32_t* labels_b = labels;
-  if (step == 1 || !overlap) {
+  if (step == 1) st->gathered_step = 0;
+  if (st->gathered_step == step) {
+    // the launch-by-launch form gathered this step's batch before the previous step's layer-1
+    // weight gradient, which read it
+  } else if (step == 1 || !overlap) {
     TC_TRY(launch_sample_gather(c, round, step, idx_b, labels_b, bfp(t.xg[xb]), bfp(t.xt[xb])));
   } else {
     // issued during the previous step on the gather stream
@@ -636,7 +686,10 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
     const CUtensorMap& wm = shared_w ? st->wg[l] : w_k(l);
     const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
-    if (l < L) {
+    if (l == 1 && f1_here) {
+      TC_TRY(launch_fwd_finish(c, st->wgrad_f1, ly.out, (const float*)(ws + t.zpart), ly.b_off,
+                               bfp(t.act[1]), bfp(t.act_t[1])));
+    } else if (l < L) {
       g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
       if (c->schedule == 0 && st->fwd_ks[l].splits > 1)
         TC_TRY(launch_gemm_ks(c, wm, l == 1 ? st->x_in_ks[xb] : st->act_in_ks[l], st->fwd_ks[l], g));
@@ -722,6 +775,19 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
       c->stream = main_s;
       side_used = true;
+    } else if (l == 1 && fuse_next) {
+      // this launch also reads the next step's gathered batch
+      const int nb = (step + 1) & 1;
+      if (overlap) {
+        TC_TRY(cudaStreamWaitEvent(main_s, st->ev_gather_done, 0));
+      } else {
+        TC_TRY(launch_sample_gather(c, round, step + 1, idx_b, labels_b, bfp(t.xg[nb]), bfp(t.xt[nb])));
+        st->gathered_step = step + 1;
+      }
+      TC_TRY(launch_wgrad_stream(c, st->wgrad_f1, st->dz_t[l], bm, st->w32[l], *w_st(l),
+                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom,
+                                 &st->x_next[nb], (float*)(ws + t.zpart)));
+      st->f1_pending = true;
     } else {
       TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));

@@ -20,6 +20,8 @@ struct TcLayout {
   size_t counters, counters_bytes;
   size_t w16, w16g;
   size_t tail_part;                          // partial sums of the fused last-layer kernel
+  size_t zpart, zpart_bytes;                 // partial sums of layer 1's forward product that rides
+                                             // along with the weight-gradient launch (wgrad_tc.cuh)
   size_t w16b;                               // second bf16 copy of layer L-1's weights [P, w16b_stride]
   int64_t w16b_stride;
   size_t end;
@@ -61,8 +63,18 @@ struct TcState {
   CUtensorMap w_b, w_mn_b, w16_st_b;
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   bool wgrad_merged = false;                  // all layers' weight gradients in one launch
+  // Layer 1's forward product of step k+1 formed inside step k's weight-gradient launch of that
+  // layer (see wgrad_tc.cuh): possible where that launch stands alone.  x_next[i]: the gathered
+  // batch buffer i as that launch reads it; f1_pending: the step about to be issued finds its
+  // first layer's product as partial sums; gathered_step: the step whose batch has already been
+  // gathered by the launch-by-launch form.
+  bool fuse_f1 = false;
+  bool f1_pending = false;
+  int gathered_step = 0;
+  CUtensorMap x_next[2];
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
+  WgradPlan wgrad_f1;                         // layer 1's plan for the launches that take the forward along
   // side streams and events for the branches of a step that may overlap
   cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,

@@ -19,6 +19,8 @@
 // Edge tiles need no predicates: TMA zero-fills loads and clips stores at the tensor bounds.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "mlp.cuh"
 #include "tc_ptx.cuh"
 #include "wgrad_tc.cuh"
@@ -40,6 +42,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
                                                                    // the first step of a round
                    const __grid_constant__ CUtensorMap tm_w16,   // bf16 [P, out, in] store
                    const __grid_constant__ CUtensorMap tm_u,     // fp32 [P, out, in] u^j, load + store (MOM)
+                   const __grid_constant__ CUtensorMap tm_xn,    // bf16 [P, B, in] next step's input (fwd_next)
                    const WgradArgs g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) WgradShared sh;
@@ -56,13 +59,16 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     tma_prefetch_desc(&tm_w32_in);
     tma_prefetch_desc(&tm_w16);
     if (MOM) tma_prefetch_desc(&tm_u);
+    if (g.fwd_next) tma_prefetch_desc(&tm_xn);
     wgrad_init_barriers(sh, g.slots);
     sh.abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
+  // two accumulators of 32 columns; with fwd_next a third of B columns behind them
+  const uint32_t tmem_cols = !g.fwd_next ? 64u : (g.batch <= 64 ? 128u : 256u);
   if (warp == 1) {
-    tmem_alloc(&sh.tmem_slot, 64);            // two accumulators of 32 columns
+    tmem_alloc(&sh.tmem_slot, tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -70,11 +76,11 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   tc_fence_after_sync();
   const uint32_t tmem_base = sh.tmem_slot;
   grid_dependency_wait();
-  wgrad_run<MOM>(tm_dzt, tm_at, tm_w32, tm_w32_in, tm_w16, tm_u, g, (int)blockIdx.x,
+  wgrad_run<MOM>(tm_dzt, tm_at, tm_w32, tm_w32_in, tm_w16, tm_u, tm_xn, g, (int)blockIdx.x,
                  (int)gridDim.x, smem, sh, tmem_base);
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, 64);
+  if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
 }
 
 // The same for several layers in one launch: every block makes one run per layer, in the order
@@ -117,13 +123,55 @@ k_wgrad_sgd_multi(const __grid_constant__ WgradMultiParams mp) {
   const int grid = (int)gridDim.x;
   for (int s = 0; s < mp.n; ++s) {
     const int vb = ((int)blockIdx.x + mp.rot[s]) % grid;
-    wgrad_run<MOM>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.g[s], vb,
-                   grid, smem, sh, tmem_base, tiles, items);
+    wgrad_run<MOM>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.w16[s],
+                   mp.g[s], vb, grid, smem, sh, tmem_base, tiles, items);
     wgrad_run_totals(mp.g[s], vb, grid, tiles, items);
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, 64);
+}
+
+// Finishes the forward product that rode along with the previous step's weight-gradient launch:
+// adds a row tile's partial sums (one per run of column tiles) in ascending run order, adds the
+// bias, applies ReLU and writes A_l as bf16 in both orientations.  grid (row tiles, P); a thread
+// takes one output row and eight consecutive batch columns at a time.
+__global__ void __launch_bounds__(256)
+k_fwd_finish(const float* __restrict__ zpart, int n_chunks, int m_tiles, int M, int B,
+             const float* __restrict__ rep, int64_t rep_stride, int64_t bias_off,
+             __nv_bfloat16* __restrict__ out_bm, __nv_bfloat16* __restrict__ out_mb) {
+  const int mt = blockIdx.x, p = blockIdx.y;
+  const size_t tile_floats = (size_t)B * kBM;
+  const float* base = zpart + ((size_t)p * m_tiles + mt) * n_chunks * tile_floats;
+  for (int u = threadIdx.x; u < kBM * (B / 8); u += blockDim.x) {
+    const int r = u & (kBM - 1), b0 = (u / kBM) * 8;
+    const int m = mt * kBM + r;
+    if (m >= M) continue;
+    float z[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) z[j] = 0.f;
+    for (int nc = 0; nc < n_chunks; ++nc) {
+      const float* src = base + (size_t)nc * tile_floats + (size_t)b0 * kBM + r;
+      float t[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) t[j] = __ldcs(src + (size_t)j * kBM);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) z[j] += t[j];
+    }
+    const float bias = rep[(size_t)p * rep_stride + bias_off + m];
+    uint32_t h4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a0 = z[2 * j] + bias, a1 = z[2 * j + 1] + bias;
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
+      h4[j] = *reinterpret_cast<uint32_t*>(&h2);
+    }
+    *reinterpret_cast<uint4*>(out_mb + ((size_t)p * M + m) * B + b0) =
+        make_uint4(h4[0], h4[1], h4[2], h4[3]);
+    const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(h4);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out_bm[((size_t)p * B + b0 + j) * M + m] = hh[j];
+  }
 }
 
 }  // namespace
@@ -145,11 +193,19 @@ constexpr long kWgradChunkCap = MAVG_WGRAD_CHUNK_CAP;
 #define MAVG_WGRAD_STREAM_SLOTS 4
 #endif
 constexpr long kWgradStreamChunk = MAVG_WGRAD_STREAM_CHUNK;
+#ifndef MAVG_WGRAD_FWD_CHUNK
+#define MAVG_WGRAD_FWD_CHUNK 64
+#endif
+constexpr long kWgradFwdChunk = MAVG_WGRAD_FWD_CHUNK;
+#ifndef MAVG_WGRAD_FWD_SLOTS
+#define MAVG_WGRAD_FWD_SLOTS 6
+#endif
+constexpr int kWgradFwdSlots = MAVG_WGRAD_FWD_SLOTS;
 constexpr int kWgradStreamSlots = MAVG_WGRAD_STREAM_SLOTS;
 constexpr int kWgradSlotCap = MAVG_WGRAD_SLOT_CAP < wgrad::kMaxSlots ? MAVG_WGRAD_SLOT_CAP : wgrad::kMaxSlots;
 
 WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum,
-                            bool streaming) {
+                            bool streaming, bool fwd_next) {
   WgradPlan w{};
   w.nkb = (B + kBK - 1) / kBK;
   w.m_tiles = (out + kBM - 1) / kBM;
@@ -159,6 +215,25 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   if (chunk < 1) chunk = 1;
   if (chunk > kWgradChunkCap) chunk = kWgradChunkCap;
   if (streaming && chunk > kWgradStreamChunk) chunk = kWgradStreamChunk;
+  // With the next step's forward product riding along, every work item ends with a 128 x B fp32
+  // partial sum going to global memory (and coming back once): long runs keep that traffic small
+  // against the 2 x 2 bytes per weight the fusion saves.
+  // Among the even splits of a row of column tiles, take the one whose busiest block finishes
+  // first: ceil(items / blocks) items of (run + one tile's worth of per-item work) each.
+  if (fwd_next) {
+    long best_cost = 0;
+    for (int nc = 1; nc <= w.n_tiles; ++nc) {
+      const long run = (w.n_tiles + nc - 1) / nc;
+      if (run > kWgradFwdChunk) continue;
+      if (run < 8 && best_cost) break;
+      const long items = (long)P * w.m_tiles * ((w.n_tiles + run - 1) / run);
+      const long cost = ((items + sm_count - 1) / sm_count) * (run + 1);
+      if (!best_cost || cost < best_cost) {
+        best_cost = cost;
+        chunk = run;
+      }
+    }
+  }
   if (chunk > w.n_tiles) chunk = w.n_tiles;
   w.chunk = (int)chunk;
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
@@ -166,7 +241,9 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   const int a_bytes = w.nkb * kBM * kBK * 2;
   const int b_bytes = w.nkb * kBN * kBK * 2;
   w.w16_on_b = b_bytes >= kW16Bytes ? 1 : 0;   // the bf16 output tile reuses the A^T slabs' space
-  const int slot_bytes = kW32Bytes + (momentum ? kW32Bytes : 0) + (w.w16_on_b ? 0 : kW16Bytes) + b_bytes;
+  w.xn_bytes = fwd_next ? B * kBN * 2 : 0;
+  const int slot_bytes = kW32Bytes + (momentum ? kW32Bytes : 0) + (w.w16_on_b ? 0 : kW16Bytes) +
+                         b_bytes + w.xn_bytes;
   const int budget = 220 * 1024;
   w.a_bufs = 2;
   w.slots = (budget - 2 * a_bytes) / slot_bytes;
@@ -175,7 +252,8 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
     w.slots = (budget - a_bytes) / slot_bytes;
   }
   if (w.slots > kWgradSlotCap) w.slots = kWgradSlotCap;
-  if (streaming && w.slots > kWgradStreamSlots) w.slots = kWgradStreamSlots;
+  const int stream_slots = fwd_next ? kWgradFwdSlots : kWgradStreamSlots;
+  if (streaming && w.slots > stream_slots) w.slots = stream_slots;
   w.smem = (size_t)w.a_bufs * a_bytes + (size_t)w.slots * slot_bytes + 1024;
   w.grid = w.items < sm_count ? w.items : sm_count;
   return w;
@@ -212,6 +290,11 @@ WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs&
   g.gamma = c->cfg.local_lr;
   g.beta = mom.beta;
   g.read_u = mom.read_u;
+  g.fwd_next = 0;
+  g.store_w16 = 1;
+  g.xn_bytes = w.xn_bytes;
+  g.batch = c->cfg.B;
+  g.zpart = nullptr;
   g.status = (int*)ws_ptr(c, c->ws.status);
   return g;
 }
@@ -258,23 +341,18 @@ cudaError_t launch_wgrad_multi(mavg_ctx* c, int n, const WgradLayerRef* layers, 
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
                                 const CUtensorMap& w16, const CUtensorMap* w32_shared,
-                                const CUtensorMap* u32, const MomArgs& mom) {
-  WgradArgs g{};
-  g.w32_in_batched = w32_shared ? 0 : 1;
-  g.nkb = w.nkb;
-  g.m_tiles = w.m_tiles;
-  g.n_tiles = w.n_tiles;
-  g.chunk = w.chunk;
-  g.n_chunks = w.n_chunks;
-  g.items = w.items;
-  g.slots = w.slots;
-  g.a_bufs = w.a_bufs;
-  g.w16_on_b = w.w16_on_b;
-  g.keep_w32 = c->l2_keep ? 1 : 0;
-  g.gamma = c->cfg.local_lr;
-  g.beta = mom.beta;
-  g.read_u = mom.read_u;
-  g.status = (int*)ws_ptr(c, c->ws.status);
+                                const CUtensorMap* u32, const MomArgs& mom,
+                                const CUtensorMap* xn, float* zpart) {
+  WgradArgs g = make_args(c, w, w32_shared != nullptr, mom);
+  if (xn) {
+    // the plan must have been made with fwd_next (room for the input tile in every slot)
+    if (w.xn_bytes == 0) return cudaErrorInvalidValue;
+    g.fwd_next = 1;
+    g.store_w16 = 0;       // the only reader of this layer's bf16 copy is the product fused here
+    g.zpart = zpart;
+  } else {
+    g.xn_bytes = w.xn_bytes;   // the slot keeps its shape; the tile is simply not loaded
+  }
   cudaLaunchConfig_t lc{};
   lc.gridDim = dim3((unsigned)w.grid);
   lc.blockDim = dim3(kThreads);
@@ -288,11 +366,21 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   prof_begin(c, MAVG_K_WGRAD_SGD);
   cudaError_t e = (mom.u && u32)
       ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<true>, dzt, at, w32,
-                           w32_shared ? *w32_shared : w32, w16, *u32, g)
+                           w32_shared ? *w32_shared : w32, w16, *u32, xn ? *xn : w16, g)
       : cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<false>, dzt, at, w32,
-                           w32_shared ? *w32_shared : w32, w16, w32, g);
+                           w32_shared ? *w32_shared : w32, w16, w32, xn ? *xn : w16, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_fwd_finish(mavg_ctx* c, const WgradPlan& w, int out, const float* zpart,
+                              int64_t bias_off, __nv_bfloat16* out_bm, __nv_bfloat16* out_mb) {
+  prof_begin(c, MAVG_K_FWD);
+  k_fwd_finish<<<dim3((unsigned)w.m_tiles, (unsigned)c->cfg.P), 256, 0, c->stream>>>(
+      zpart, w.n_chunks, w.m_tiles, out, c->cfg.B, c->buf.replicas, c->buf.replica_stride, bias_off,
+      out_bm, out_mb);
+  prof_end(c);
+  return cudaGetLastError();
 }
 
 }  // namespace mavg

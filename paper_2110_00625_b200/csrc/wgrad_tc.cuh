@@ -8,6 +8,7 @@ namespace mavg {
 
 struct WgradPlan {
   int nkb, m_tiles, n_tiles, chunk, n_chunks, items, slots, a_bufs, grid, w16_on_b;
+  int xn_bytes;   // room in every slot for the next step's input tile (plans made with fwd_next)
   size_t smem;
 };
 
@@ -18,8 +19,11 @@ constexpr int kWgradTileCols = 32;    // columns of in per tile
 // is a stream through HBM; the ring is then kept shallow and the runs of column tiles short
 // (measured on the large MLP, B = 64: 4 slots and runs of 4 to 8 tiles give 0.84 of the copy
 // bandwidth against 0.80 with 6 slots and runs of 16, and 0.67 with 3 slots).
+// fwd_next: the launch may also take the next step's forward product of this layer along (see
+// launch_wgrad_stream): every slot gets room for a [B, 32] tile of the next step's input and the
+// runs of column tiles get long.
 WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool momentum = false,
-                            bool streaming = false);
+                            bool streaming = false, bool fwd_next = false);
 cudaError_t wgrad_stream_prepare();
 // dzt: bf16 [P, out, B] box 64 x 128 (128B swizzle); at: bf16 [P, in, B] box 64 x 32 (128B swizzle);
 // w32: fp32 [P, out, in] box 32 x 128 (128B swizzle); w16: bf16 [P, out, in] box 32 x 128
@@ -27,10 +31,21 @@ cudaError_t wgrad_stream_prepare();
 // masters are then loaded from it for every learner (first step of a round, all w^j = w~) and
 // stored to w32 as always.  With learner-level momentum (mom.u set; the plan made with
 // momentum = true) u32 is the fp32 [P, out, in] view of the buffers u^j with w32's box.
+// xn, zpart (plans made with fwd_next only): xn is the bf16 [P, B, in] input of the NEXT local step
+// of this layer, box 32 x B (64B swizzle).  The launch then also forms that step's forward
+// product from the updated weight tiles while they are in shared memory,
+//   Z^T[out, B] = W_new[out, in] . Xn[B, in]^T,
+// as fp32 partial sums per work item in zpart (see WgradArgs), which launch_fwd_finish adds up,
+// and does NOT write the bf16 copy of the weights.
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
                                 const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr,
-                                const CUtensorMap* u32 = nullptr, const MomArgs& mom = MomArgs());
+                                const CUtensorMap* u32 = nullptr, const MomArgs& mom = MomArgs(),
+                                const CUtensorMap* xn = nullptr, float* zpart = nullptr);
+// A_l = relu(sum of the plan's partial sums in ascending run order + b_l), as bf16 in both
+// orientations: out_bm [P, B, out], out_mb [P, out, B].  Biases from the masters.
+cudaError_t launch_fwd_finish(mavg_ctx* c, const WgradPlan& w, int out, const float* zpart,
+                              int64_t bias_off, __nv_bfloat16* out_bm, __nv_bfloat16* out_mb);
 
 // Several layers' weight-gradient + SGD tiles in one persistent launch (layers listed in the
 // order their tiles should run).  All plans must come from the same batch size and momentum

@@ -12,7 +12,8 @@ namespace wgrad {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 32, kBK = 64;
-constexpr int kThreads = 352;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores
+constexpr int kThreads = 384;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores,
+                                // 11 forward MMAs (fwd_next)
 constexpr int kMaxSlots = 6;
 constexpr int kW32Bytes = kBM * kBN * 4;  // 16 KB, rows of 128 bytes, 128-byte swizzle
 constexpr int kW16Bytes = kBM * kBN * 2;  //  8 KB, rows of  64 bytes,  64-byte swizzle
@@ -61,6 +62,17 @@ struct WgradArgs {
   float gamma;
   float beta;              // learner momentum (MOM)
   int read_u;              // 0: the stored u counts as zero and is not loaded
+  // Next step's forward product of the same layer, taken from the freshly updated tiles while
+  // they are in shared memory (see wgrad_tc.cu): fwd_next = 1 adds, per tile,
+  //   Z^T[128 rows, B] += W16_tile[128, 32] . Xn[B, 32]^T
+  // into a third TMEM accumulator; per work item the fp32 partial sum goes to
+  //   zpart[((p * m_tiles + row tile) * n_chunks + chunk) * B * 128 + b * 128 + row].
+  int fwd_next;
+  int store_w16;           // 0: the bf16 tile is not written to global memory
+  int xn_bytes;            // room in a slot for the next step's input tile [B, 32] bf16 (loaded
+                           // only with fwd_next; part of the slot's size whenever the plan has it)
+  int batch;               // B
+  float* zpart;
   int* status;
 };
 
@@ -69,6 +81,8 @@ struct WgradShared {
   uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots], out_full[kMaxSlots];
   uint64_t tmem_full[2], tmem_empty[2];
   uint64_t a_full[2], a_empty[2];
+  uint64_t z_done[kMaxSlots];   // the forward MMAs that read this slot's bf16 tile have finished
+  uint64_t z_full, z_empty;     // the item's forward accumulator is complete / has been read
   uint32_t tmem_slot;
   int abort_flag;
 };
@@ -78,7 +92,10 @@ __device__ __forceinline__ void wgrad_init_barriers(WgradShared& sh, int slots) 
     mbar_init(&sh.slot_full[s], 1);
     mbar_init(&sh.slot_empty[s], 1);
     mbar_init(&sh.out_full[s], 4);
+    mbar_init(&sh.z_done[s], 1);
   }
+  mbar_init(&sh.z_full, 1);
+  mbar_init(&sh.z_empty, 4);
   for (int b = 0; b < 2; ++b) {
     mbar_init(&sh.tmem_full[b], 1);
     mbar_init(&sh.tmem_empty[b], 4);
@@ -107,6 +124,7 @@ template <bool MOM>
 __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUtensorMap& tm_at,
                                           const CUtensorMap& tm_w32, const CUtensorMap& tm_w32_in,
                                           const CUtensorMap& tm_w16, const CUtensorMap& tm_u,
+                                          const CUtensorMap& tm_xn,
                                           const WgradArgs& g, int vblock, int vgrid, uint8_t* smem,
                                           WgradShared& sh, uint32_t tmem_base,
                                           uint32_t tile_base = 0, uint32_t item_base = 0) {
@@ -120,7 +138,9 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
   constexpr int kUBytes = MOM ? kW32Bytes : 0;
   const int w16_off = kW32Bytes + kUBytes;
   const int b_off = g.w16_on_b ? w16_off : w16_off + kW16Bytes;
-  const int slot_bytes = b_off + b_bytes;                   // multiple of 1024
+  const int xn_off = b_off + b_bytes;                       // next step's input tile (fwd_next)
+  const int slot_bytes = xn_off + g.xn_bytes;               // multiple of 1024
+  constexpr uint32_t kZCol = 2 * kBN;                       // forward accumulator: B columns from here
   uint8_t* a_base = smem;
   uint8_t* slot_base = smem + (size_t)g.a_bufs * a_bytes;
   volatile int* abortp = &sh.abort_flag;
@@ -162,7 +182,9 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           const int i0 = (nt0 + j) * kBN;
           const bool load_u = MOM && g.read_u;
           mbar_arrive_expect_tx(&sh.slot_full[s],
-                                (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0)));
+                                (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0) +
+                                           (g.fwd_next ? g.xn_bytes : 0)));
+          if (g.fwd_next) tma_load_3d(sl + xn_off, &tm_xn, &sh.slot_full[s], i0, 0, p);
           tma_load_3d_hint(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0, pol);
           if (load_u) tma_load_3d(sl + kW32Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
@@ -214,9 +236,9 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
     const int grp = (warp - 2) >> 2;           // epilogue group = TMEM buffer = tile parity
     const int q = warp & 3;                    // TMEM lane quarter this warp may read
     const int r = q * 32 + lane;               // weight row inside the tile
-    uint32_t tile_ctr = tile_base;
+    uint32_t tile_ctr = tile_base, item_ctr = item_base;
     bool ok = true;
-    for (int item = vblock; item < g.items && ok; item += vgrid) {
+    for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
       int p, m0, nt0, nt;
       decode(item, p, m0, nt0, nt);
       for (int j = 0; j < nt; ++j, ++tile_ctr) {
@@ -272,15 +294,46 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           *reinterpret_cast<uint4*>(w16 + ((c ^ ((r >> 1) & 3)) << 4)) =
               make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
         fence_proxy_async();                   // generic-proxy writes -> visible to the TMA stores
-        __syncwarp();
+        __syncwarp();                          // (and to the forward MMAs, fwd_next)
         if (lane == 0) mbar_arrive(&sh.out_full[s]);
       }
+      if (g.fwd_next && grp == 0 && ok) {
+        // the item's share of the next step's forward product: fp32 partial to global memory,
+        // one weight row per lane, a batch column per store (128 bytes per warp)
+        if (!mbar_wait(&sh.z_full, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        float* zp = g.zpart +
+                    (((size_t)p * g.m_tiles + m0 / kBM) * g.n_chunks + nt0 / g.chunk) *
+                        ((size_t)g.batch * kBM) + r;
+        for (int c0 = 0; c0 < g.batch; c0 += 32) {
+          uint32_t acc[32];
+          if (c0 + 32 <= g.batch) {
+            tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, acc);
+          } else {                             // the batch is a multiple of 16
+            uint32_t h16[16];
+            tmem_ld_16cols(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, h16);
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) { acc[jj] = h16[jj]; acc[16 + jj] = 0u; }
+          }
+          tmem_ld_wait();
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj)
+            if (c0 + jj < g.batch) zp[(size_t)(c0 + jj) * kBM] = __uint_as_float(acc[jj]);
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.z_empty);
+      }
     }
-  } else {
+  } else if (warp == 10) {
     if (lane == 0) {
       uint32_t tile_ctr = tile_base;
       bool ok = true;
       int held = -1;          // slot whose stores are committed but not yet known to be read
+      uint32_t held_use = 0;
       const uint64_t pol = l2_policy(g.keep_w32 != 0);
       for (int item = vblock; item < g.items && ok; item += vgrid) {
         int p, m0, nt0, nt;
@@ -295,15 +348,20 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           uint8_t* sl = slot_base + (size_t)s * slot_bytes;
           const int i0 = (nt0 + j) * kBN;
           tma_store_3d_hint(&tm_w32, sl, i0, m0, p, pol);
-          tma_store_3d(&tm_w16, sl + w16_off, i0, m0, p);
+          if (g.store_w16) tma_store_3d(&tm_w16, sl + w16_off, i0, m0, p);
           if (MOM) tma_store_3d(&tm_u, sl + kW32Bytes, i0, m0, p);
           tma_store_commit();
           // A slot is free once its stores have read shared memory.  If the next tile is already
           // waiting to be stored, its stores go out first and this slot is handed back behind
           // them; if not, this thread has nothing else to do, waits for the read here and hands
           // the slot back a whole tile period earlier.
+          // (with fwd_next a slot is also still being read by its forward MMAs: z_done)
           if (held >= 0) {
             tma_store_wait_read<1>();
+            if (g.fwd_next && !mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE)) {
+              ok = false;
+              break;
+            }
             mbar_arrive(&sh.slot_empty[held]);
             held = -1;
           }
@@ -311,8 +369,13 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
             const uint32_t nx = tile_ctr + 1;
             if (mbar_try_wait(&sh.out_full[nx % g.slots], (nx / g.slots) & 1)) {
               held = s;
+              held_use = use;
             } else {
               tma_store_wait_read<0>();
+              if (g.fwd_next && !mbar_wait(&sh.z_done[s], use & 1, abortp, g.status, ERR_WG_STORE)) {
+                ok = false;
+                break;
+              }
               mbar_arrive(&sh.slot_empty[s]);
             }
           }
@@ -320,7 +383,44 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       }
       if (held >= 0) {
         tma_store_wait_read<0>();
-        mbar_arrive(&sh.slot_empty[held]);
+        if (!g.fwd_next || mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE))
+          mbar_arrive(&sh.slot_empty[held]);
+      }
+    }
+    __syncwarp();
+  } else {
+    // warp 11 (fwd_next): the forward MMAs of a tile, issued as soon as the epilogue has put the
+    // updated bf16 tile into its slot; they read that tile and the next step's input tile beside it
+    if (lane == 0 && g.fwd_next) {
+      const uint32_t idesc_z = idesc_bf16_f32(kBM, g.batch);
+      uint32_t tile_ctr = tile_base, item_ctr = item_base;
+      bool ok = true;
+      for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
+        int p, m0, nt0, nt;
+        decode(item, p, m0, nt0, nt);
+        for (int j = 0; j < nt; ++j, ++tile_ctr) {
+          const int s = tile_ctr % g.slots;
+          if (!mbar_wait(&sh.out_full[s], (tile_ctr / g.slots) & 1, abortp, g.status, ERR_WG_MMA)) {
+            ok = false;
+            break;
+          }
+          // the previous item's accumulator must have been read before this item's first
+          // forward MMA overwrites it
+          if (j == 0 && !mbar_wait(&sh.z_empty, (item_ctr & 1) ^ 1, abortp, g.status, ERR_WG_MMA)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint32_t base = smem_u32(slot_base + (size_t)s * slot_bytes);
+          const uint64_t adesc = smem_desc_k_sw64(base + w16_off);
+          const uint64_t bdesc = smem_desc_k_sw64(base + xn_off);
+#pragma unroll
+          for (int k = 0; k < kBN / 16; ++k)
+            umma_bf16(tmem_base + kZCol, adesc + 2 * k, bdesc + 2 * k, idesc_z,
+                      (uint32_t)((j | k) != 0));
+          umma_commit(&sh.z_done[s]);
+          if (j == nt - 1) umma_commit(&sh.z_full);
+        }
       }
     }
     __syncwarp();

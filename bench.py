@@ -235,24 +235,27 @@ NCU_TRAFFIC = {
 }
 
 
-def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=0):
+def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=()):
     """Bytes that must cross HBM per ROUND for each kernel class (weights streamed once per
-    product, activations in and out), and their total.  fwd_run_tiles > 0: in steps 1..K-1 the
-    layer-1 weight-gradient launch also forms the next step's layer-1 forward product (no bf16
-    copy of layer 1 written or read in those steps; instead one fp32 partial sum [128, B] per
-    learner, row tile and run of fwd_run_tiles column tiles, written there and read by the
-    kernel that finishes the layer, and the next batch read once more)."""
+    product, activations in and out), and their total.  fwd_run_tiles[l-1], layers l = 1..m: in
+    steps 1..K-1 the weight-gradient launch of layer l also forms the next step's forward product
+    of that layer: its bf16 weights are not read by a forward kernel in steps 2..K (layer 1's copy
+    is not even written); the layer's next input is read and its next activations are written by
+    the weight-gradient launch, which also writes and reads back one fp32 partial sum [128, B]
+    per learner, row tile and run of fwd_run_tiles[l-1] column tiles."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
     nW = [dims[l] * dims[l + 1] for l in range(L)]
     n = sum(nW) + sum(dims[1:])
     rows = P * B
     fwd_delta = wgrad_delta = 0
-    if fwd_run_tiles > 0 and K > 1:
-        n_tiles = -(-dims[0] // 32)
-        partial = P * -(-dims[1] // 128) * -(-n_tiles // fwd_run_tiles) * B * 128 * 4
-        fwd_delta = (K - 1) * (partial - 2 * P * nW[0] - 2 * rows * dims[0])
-        wgrad_delta = (K - 1) * (partial - 2 * P * nW[0] + 2 * rows * dims[0])
+    for i, run in enumerate(fwd_run_tiles if K > 1 else ()):
+        n_tiles = -(-dims[i] // 32)
+        runs = -(-n_tiles // run)
+        partial = P * -(-dims[i + 1] // 128) * runs * B * 128 * 4 if runs > 1 else 0
+        moved = 2 * rows * dims[i] + 4 * rows * dims[i + 1]     # the layer's input read, A_l written twice
+        fwd_delta -= (K - 1) * (2 * P * nW[i] + moved)
+        wgrad_delta += (K - 1) * (moved + 2 * partial - (2 * P * nW[0] if i == 0 else 0))
     per_round = {
         # replicas, w~, v read; v, w~ and (unless the copies are deferred) the replicas written
         "meta_update": dict(bytes=((4 if deferred else 8) * P + 16) * n, flops=0),
@@ -274,7 +277,7 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_
 
 
 def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False,
-                     fwd_run_tiles=0):
+                     fwd_run_tiles=()):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
     per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles)
     out = {}
@@ -507,7 +510,7 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
     prof = g.get_profile(reset=True)
     g.set_profiling(False)
     plan = g.get_step_plan()
-    fwd_run_tiles = plan["fwd_run_tiles"] if plan["fwd_with_wgrad"] and args.schedule == 0 else 0
+    fwd_run_tiles = tuple(plan["fwd_run_tiles"]) if args.schedule == 0 else ()
     kern = kernel_rooflines(cfg, prof, psteps, peaks, mode == 1, deferred=not args.no_defer,
                             momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles)
     n = g.n
@@ -611,9 +614,10 @@ def run_mavg(args):
                        "l2_keep": bool(args.l2_keep),
                        "schedule": {0: "CUDA graph of per-product launches",
                                     2: "CUDA graph of per-product launches, plain tensor-core tiles"}[args.schedule],
-                       "layer1_forward": ("inside the layer's weight-gradient launch of the step before "
-                                          f"(steps 2..K; partial sums per {r['fwd_run_tiles']} column tiles)"
-                                          if r["fwd_run_tiles"] else "a launch of its own"),
+                       "forward_products": (f"layers 1..{len(r['fwd_run_tiles'])} inside their weight-gradient "
+                                            "launch of the step before (steps 2..K; partial sums per "
+                                            f"{list(r['fwd_run_tiles'])} column tiles)"
+                                            if r["fwd_run_tiles"] else "launches of their own"),
                        "l2": "flushed between steps by a 256 MiB memset, outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],

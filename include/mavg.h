@@ -210,12 +210,13 @@ mavg_status mavg_get_launch_count(mavg_handle h, int64_t *count);
 typedef enum {
   MAVG_PLAN_TENSOR_PATH = 0,    /* 1: the products run on the tensor cores (bf16 operands) */
   MAVG_PLAN_WGRAD_MERGED = 1,   /* 1: all layers' weight gradients + SGD share one launch */
-  MAVG_PLAN_FWD_WITH_WGRAD = 2, /* 1: under the default schedule, layer 1's weight-gradient launch
-                                   of steps 1..K-1 also forms the next step's layer-1 forward
-                                   product from the updated tiles (no bf16 copy of layer 1 is
-                                   written in those steps) */
-  MAVG_PLAN_FWD_RUN_TILES = 3,  /* with FWD_WITH_WGRAD: column tiles per partial sum */
-  MAVG_PLAN_COUNT = 4
+  MAVG_PLAN_FWD_WITH_WGRAD = 2, /* m >= 0: under the default schedule, in steps 1..K-1 the
+                                   weight-gradient launches of layers 1..m also form the next
+                                   step's forward product of their layer from the updated tiles
+                                   (m <= L-1; layer 1's bf16 copy is not written in those steps) */
+  MAVG_PLAN_FWD_RUN_TILES = 3,  /* first of MAVG_MAX_LAYERS entries: for layer l <= m, entry
+                                   3 + l - 1 is the number of column tiles per partial sum */
+  MAVG_PLAN_COUNT = 3 + MAVG_MAX_LAYERS
 } mavg_plan_entry;
 mavg_status mavg_get_step_plan(mavg_handle h, int32_t *out);
 

@@ -24,7 +24,6 @@ EXPORTS = ["mavg_workspace_bytes", "mavg_create", "mavg_local_steps", "mavg_meta
            "mavg_get_step_plan", "mavg_set_profiling", "mavg_set_schedule", "mavg_get_profile", "mavg_sync",
            "mavg_set_wait_limit", "mavg_selftest_wait", "mavg_cache_release", "mavg_last_error",
            "mavg_batch_indices_noalloc", "mavg_destroy"]
-PLAN_ENTRIES = ["tensor_path", "wgrad_merged", "fwd_with_wgrad", "fwd_run_tiles"]
 KERNEL_CLASSES = ["meta_update", "broadcast", "pseudograd_steps", "batch_gather", "fwd_gemm",
                   "loss", "dgrad_gemm", "wgrad_sgd_gemm", "aux"]
 
@@ -269,9 +268,13 @@ class Mavg:
         return r.value
 
     def get_step_plan(self):
-        out = (C.c_int32 * len(PLAN_ENTRIES))()
+        """How a local step is laid out in launches: tensor_path, wgrad_merged, fwd_with_wgrad
+        (layers 1..m whose next-step forward product rides on their weight-gradient launch) and
+        fwd_run_tiles (per such layer, column tiles per partial sum)."""
+        out = (C.c_int32 * (3 + MAX_LAYERS))()
         self._check(self.lib.mavg_get_step_plan(self.handle, out))
-        return dict(zip(PLAN_ENTRIES, out))
+        return {"tensor_path": out[0], "wgrad_merged": out[1], "fwd_with_wgrad": out[2],
+                "fwd_run_tiles": list(out[3:3 + out[2]])}
 
     def set_profiling(self, on):
         self._check(self.lib.mavg_set_profiling(self.handle, int(bool(on))))

@@ -196,6 +196,8 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
     if (l < L) {
       t.act[l] = take(rows * d * 2);
       t.act_t[l] = take(rows * d * 2);
+      t.act_b[l] = take(rows * d * 2);
+      t.act_t_b[l] = take(rows * d * 2);
       t.dz[l] = take(rows * d * 2);
     } else {
       t.dz[l] = take(rows * t.cpad * 2);
@@ -220,13 +222,18 @@ TcLayout make_layout(const mavg_config* cfg, size_t base, int sm_count) {
   t.w16g = take((size_t)t.n16 * 2);
   t.tail_part = take(tail_fused_supported(cfg) ? tail_fused_part_bytes(cfg) : 16);
   {
-    // partial sums of the forward product that rides along with layer 1's weight-gradient launch:
-    // one 128 x B fp32 tile per (learner, row tile, run of column tiles) of that launch's plan
+    // partial sums of a forward product that rides along with a weight-gradient launch: one
+    // 128 x B fp32 tile per (learner, row tile, run of column tiles) of that launch's plan; the
+    // layers use the space one after the other
     t.zpart_bytes = 16;
-    if (L >= 2 && B <= 128) {
-      const WgradPlan w = plan_wgrad_stream(cfg->dims[1], cfg->dims[0], B, P, sm_count, false, true, true);
-      t.zpart_bytes = (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float);
-    }
+    t.zcount_bytes = 16;
+    if (B <= 128)
+      for (int l = 1; l < L; ++l) {
+        const WgradPlan w = plan_wgrad_stream(cfg->dims[l], cfg->dims[l - 1], B, P, sm_count, false, true, true);
+        t.zpart_bytes = std::max(t.zpart_bytes, (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float));
+        t.zcount_bytes = std::max(t.zcount_bytes, (size_t)P * w.m_tiles * sizeof(int));
+      }
+    t.zcount = take(t.zcount_bytes);
     t.zpart = take(t.zpart_bytes);
   }
   t.w16b_stride = L >= 3 ? (int64_t)up((size_t)cfg->dims[L - 2] * cfg->dims[L - 1], 64) : 0;
@@ -454,6 +461,14 @@ mavg_status tc_setup(mavg_ctx* c) {
       if (st->fwd_ks[l].splits > 1)
         ok = ok && encode_map(st, &st->act_in_ks[l], bf(t.act[l - 1]), in, B, P, in,
                               (int64_t)B * in, B, &why);
+      // the same three views of the second set of activation buffers
+      ok = ok && encode_map(st, &st->act_in_b[l], bf(t.act_b[l - 1]), in, B, P, in, (int64_t)B * in,
+                            st->fwd[l].BN, &why);
+      ok = ok && encode_map(st, &st->act_in_t_b[l], bf(t.act_t_b[l - 1]), B, in, P, B,
+                            (int64_t)B * in, kWgradTileCols, &why);
+      if (st->fwd_ks[l].splits > 1)
+        ok = ok && encode_map(st, &st->act_in_ks_b[l], bf(t.act_b[l - 1]), in, B, P, in,
+                              (int64_t)B * in, B, &why);
     }
     ok = ok && encode_map(st, &st->dz_t[l], bf(t.dz_t[l]), B, out, P, B, (int64_t)B * out, kBM,
                           &why);
@@ -500,24 +515,28 @@ mavg_status tc_setup(mavg_ctx* c) {
     for (int l = 2; l <= L; ++l)
       if (st->wgrad[l].slots != w1.slots || st->wgrad[l].a_bufs != w1.a_bufs) st->wgrad_merged = false;
   }
-  // Where layer 1's weight gradient is a launch of its own, it can take the next step's forward
-  // product of layer 1 along: the layer's plan gets room for the next step's input tile and long
-  // runs, and the gathered batch buffers get a view with 32-column boxes.
-  st->fuse_f1 = false;
+  // Where the weight gradients are launches of their own, the launch of layer l can take the
+  // next step's forward product of layer l along (layers 1..fuse_upto, a prefix of the hidden
+  // layers): its plan gets room for the next step's input tile and long runs, and the input
+  // buffers get a view with 32-column boxes.
+  st->fuse_upto = 0;
   if (!st->wgrad_merged && L >= 2 && B <= 128 && ok) {
-    const WgradPlan w = plan_wgrad_stream(cfg.dims[1], cfg.dims[0], B, P, c->sm_count, st->wgrad_mom,
-                                          !masters_fit_l2(c), true);
-    const size_t need = (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float);
-    if (w.slots >= 2 && need <= t.zpart_bytes) {
+    for (int l = 1; l < L; ++l) {
+      const int in = cfg.dims[l - 1], out = cfg.dims[l];
+      const WgradPlan w = plan_wgrad_stream(out, in, B, P, c->sm_count, st->wgrad_mom,
+                                            !masters_fit_l2(c), true);
+      const size_t need = (size_t)P * w.m_tiles * w.n_chunks * B * kBM * sizeof(float);
+      if (w.slots < 2 || need > t.zpart_bytes || (size_t)P * w.m_tiles * sizeof(int) > t.zcount_bytes)
+        break;
       bool enc = true;
-      for (int i = 0; i < 2 && enc; ++i)
-        enc = encode_any(st, &st->x_next[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bf(t.xg[i]),
-                         cfg.dims[0], B, P, cfg.dims[0], (int64_t)B * cfg.dims[0], kWgradTileCols, B,
-                         CU_TENSOR_MAP_SWIZZLE_64B, &why);
-      if (enc) {
-        st->wgrad_f1 = w;
-        st->fuse_f1 = true;
+      for (int i = 0; i < 2 && enc; ++i) {
+        const size_t src = l == 1 ? t.xg[i] : (i == 0 ? t.act[l - 1] : t.act_b[l - 1]);
+        enc = encode_any(st, &st->a_next[l][i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bf(src), in, B,
+                         P, in, (int64_t)B * in, kWgradTileCols, B, CU_TENSOR_MAP_SWIZZLE_64B, &why);
       }
+      if (!enc) break;
+      st->wgrad_f[l] = w;
+      st->fuse_upto = l;
     }
   }
   // the meta-update writes the bf16 copy of w~ itself where its vector kernel takes the whole model
@@ -539,6 +558,7 @@ mavg_status tc_setup(mavg_ctx* c) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ws + t.counters, 0, t.counters_bytes, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + t.zcount, 0, t.zcount_bytes, c->stream);
 
   if (e != cudaSuccess) {
     c->err = std::string("tensor-core path set-up: ") + cudaGetErrorString(e);
@@ -572,8 +592,8 @@ void tc_step_plan(mavg_ctx* c, int32_t* out) {
   if (!st) return;
   out[MAVG_PLAN_TENSOR_PATH] = 1;
   out[MAVG_PLAN_WGRAD_MERGED] = st->wgrad_merged ? 1 : 0;
-  out[MAVG_PLAN_FWD_WITH_WGRAD] = st->fuse_f1 ? 1 : 0;
-  out[MAVG_PLAN_FWD_RUN_TILES] = st->fuse_f1 ? st->wgrad_f1.chunk : 0;
+  out[MAVG_PLAN_FWD_WITH_WGRAD] = st->fuse_upto;
+  for (int l = 1; l <= st->fuse_upto; ++l) out[MAVG_PLAN_FWD_RUN_TILES + l - 1] = st->wgrad_f[l].chunk;
 }
 
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
@@ -625,13 +645,19 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
   const bool fused_tail = st->tail_ok && c->schedule == 0;
   bool tail_on_side = false;
   const bool merged = st->wgrad_merged && c->schedule == 0;
-  // Layer 1's forward product of the NEXT step rides along with this step's weight-gradient
-  // launch of layer 1 (default schedule, that launch standing alone, a next step in this call).
-  // The step after finds the product as partial sums (f1_pending) and only finishes it.
-  const bool fuse_next = st->fuse_f1 && c->schedule == 0 && !merged && step < K;
-  if (step == 1) st->f1_pending = false;
-  const bool f1_here = st->f1_pending;
-  st->f1_pending = false;
+  // Forward products of the NEXT step ride along with this step's weight-gradient launches of
+  // layers 1..ride (default schedule, those launches standing alone, a next step in this call);
+  // the step after finds the activations of its first fwd_done layers in place.
+  const int ride = (c->schedule == 0 && !merged && step < K) ? st->fuse_upto : 0;
+  const int done = step == 1 ? 0 : st->fwd_done;
+  st->fwd_done = 0;
+  // activation buffers of this step and of the next
+  const int ab = st->fuse_upto >= 1 ? (step & 1) : 0;
+  auto act_of = [&](int l, int set) { return bfp(set ? t.act_b[l] : t.act[l]); };
+  auto act_t_of = [&](int l, int set) { return bfp(set ? t.act_t_b[l] : t.act_t[l]); };
+  auto act_in = [&](int l) -> const CUtensorMap& { return ab ? st->act_in_b[l] : st->act_in[l]; };
+  auto act_in_t = [&](int l) -> const CUtensorMap& { return ab ? st->act_in_t_b[l] : st->act_in_t[l]; };
+  auto act_in_ks = [&](int l) -> const CUtensorMap& { return ab ? st->act_in_ks_b[l] : st->act_in_ks[l]; };
   // Weight gradients of the last two layers beside the remaining dgrad products (their dZ comes
   // out of the fused last-layer kernel): layer L-1 then writes the other of its two bf16 copies,
   // because dgrad through it still reads the current one.
@@ -650,7 +676,7 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     WgradLayerRef r{};
     r.plan = &st->wgrad[l];
     r.dzt = &st->dz_t[l];
-    r.at = l == 1 ? &st->x_in_t[xb] : &st->act_in_t[l];
+    r.at = l == 1 ? &st->x_in_t[xb] : &act_in_t(l);
     r.w32 = &st->w32[l];
     r.w16 = w_st(l);
     r.w32_shared = shared_w ? &st->w32g[l] : nullptr;
@@ -685,20 +711,19 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     g.bias_in = shared_w ? c->buf.global_w : c->buf.replicas;
     g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
     const CUtensorMap& wm = shared_w ? st->wg[l] : w_k(l);
-    const CUtensorMap& am = l == 1 ? st->x_in[xb] : st->act_in[l];
-    if (l == 1 && f1_here) {
-      TC_TRY(launch_fwd_finish(c, st->wgrad_f1, ly.out, (const float*)(ws + t.zpart), ly.b_off,
-                               bfp(t.act[1]), bfp(t.act_t[1])));
+    const CUtensorMap& am = l == 1 ? st->x_in[xb] : act_in(l);
+    if (l <= done) {
+      // A_l of this step came out of the previous step's weight-gradient launch of this layer
     } else if (l < L) {
-      g.out_bm = bfp(t.act[l]); g.out_mb = bfp(t.act_t[l]);
+      g.out_bm = act_of(l, ab); g.out_mb = act_t_of(l, ab);
       if (c->schedule == 0 && st->fwd_ks[l].splits > 1)
-        TC_TRY(launch_gemm_ks(c, wm, l == 1 ? st->x_in_ks[xb] : st->act_in_ks[l], st->fwd_ks[l], g));
+        TC_TRY(launch_gemm_ks(c, wm, l == 1 ? st->x_in_ks[xb] : act_in_ks(l), st->fwd_ks[l], g));
       else
         TC_TRY(launch_gemm<EPI_FWD_HIDDEN>(c, MAVG_K_FWD, wm, am, st->fwd[l], g));
     } else if (fused_tail) {
       // last layer forward, loss, dZ_L and dgrad_L in one CUDA-core kernel
       TailLaunch tl{};
-      tl.a_bm = L >= 2 ? bfp(t.act[L - 1]) : bfp(t.xg[xb]);
+      tl.a_bm = L >= 2 ? act_of(L - 1, ab) : bfp(t.xg[xb]);
       tl.w16 = (shared_w ? bfp(t.w16g) : bfp(t.w16)) + t.sh_off[L - 1];
       tl.w16_stride = shared_w ? 0 : t.n16;
       tl.shared_w = shared_w;
@@ -759,14 +784,15 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
       g.bias_in = shared_w ? c->buf.global_w : c->buf.replicas;
       g.bias_in_stride = shared_w ? 0 : c->buf.replica_stride;
       g.out_bm = bfp(t.dz[l - 1]); g.out_mb = bfp(t.dz_t[l - 1]);
-      g.mask_mb = bfp(t.act_t[l - 1]);
+      g.mask_mb = act_t_of(l - 1, ab);
       g.a_mn = 1;
       g.mom = mom;
       TC_TRY(launch_gemm<EPI_DGRAD>(c, MAVG_K_DGRAD, shared_w ? st->wg_mn[l] : w_mn(l),
                                     st->dz[l], st->dgrad[l], g));
     }
-    const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : st->act_in_t[l];
+    const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : act_in_t(l);
     if (merged) continue;        // all layers' weight gradients follow in one launch
+    if (l <= ride) continue;     // after the dgrad chain, in ascending order (below)
     if (overlap && l > 1) {
       TC_TRY(cudaEventRecord(st->ev_fork, main_s));
       TC_TRY(cudaStreamWaitEvent(st->s_wgrad, st->ev_fork, 0));
@@ -775,23 +801,40 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
                                  shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
       c->stream = main_s;
       side_used = true;
-    } else if (l == 1 && fuse_next) {
-      // this launch also reads the next step's gathered batch
-      const int nb = (step + 1) & 1;
+    } else {
+      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
+                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
+    }
+  }
+  // Layers whose launch takes the next step's forward product along: layer l's needs A_{l-1} of
+  // the next step, so they run in ascending order, each leaving A_l of the next step behind (in
+  // the other set of activation buffers: this step's A_l is still an operand of layer l+1's
+  // launch).  Layer 1 reads the next step's gathered
+  // batch; only layer 1's bf16 copy has no other reader and is left unwritten.
+  for (int l = 1; l <= ride; ++l) {
+    const MlpLayer& ly = c->layers[l - 1];
+    const int nb = (step + 1) & 1;
+    if (l == 1) {
       if (overlap) {
         TC_TRY(cudaStreamWaitEvent(main_s, st->ev_gather_done, 0));
       } else {
         TC_TRY(launch_sample_gather(c, round, step + 1, idx_b, labels_b, bfp(t.xg[nb]), bfp(t.xt[nb])));
         st->gathered_step = step + 1;
       }
-      TC_TRY(launch_wgrad_stream(c, st->wgrad_f1, st->dz_t[l], bm, st->w32[l], *w_st(l),
-                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom,
-                                 &st->x_next[nb], (float*)(ws + t.zpart)));
-      st->f1_pending = true;
-    } else {
-      TC_TRY(launch_wgrad_stream(c, st->wgrad[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
-                                 shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom));
     }
+    const CUtensorMap& bm = l == 1 ? st->x_in_t[xb] : act_in_t(l);
+    WgradFwdNext fn{};
+    fn.xn = &st->a_next[l][nb];
+    fn.zpart = (float*)(ws + t.zpart);
+    fn.zcount = (int*)(ws + t.zcount);
+    fn.bias_off = ly.b_off;
+    fn.out_rows = ly.out;
+    fn.out_bm = act_of(l, nb);
+    fn.out_mb = act_t_of(l, nb);
+    fn.store_w16 = l > 1;
+    TC_TRY(launch_wgrad_stream(c, st->wgrad_f[l], st->dz_t[l], bm, st->w32[l], *w_st(l),
+                               shared_w ? &st->w32g[l] : nullptr, &st->u32[l], mom, &fn));
+    st->fwd_done = l;
   }
   if (merged) {
     // largest layer first, so that the small ones fill the ragged end of the launch

@@ -15,13 +15,18 @@ struct TcLayout {
   int64_t sh_off[MAVG_MAX_LAYERS];
   size_t xg[2], xt[2];                       // gathered batch, two buffers used by alternate steps
   size_t act[MAVG_MAX_LAYERS + 1], act_t[MAVG_MAX_LAYERS + 1];
+  // second set of activation buffers: odd steps use it where a step's weight-gradient launches
+  // already produce the next step's activations (TcState::fuse_upto)
+  size_t act_b[MAVG_MAX_LAYERS + 1], act_t_b[MAVG_MAX_LAYERS + 1];
   size_t dz[MAVG_MAX_LAYERS + 1], dz_t[MAVG_MAX_LAYERS + 1];
   size_t part, part_bytes;
   size_t counters, counters_bytes;
   size_t w16, w16g;
   size_t tail_part;                          // partial sums of the fused last-layer kernel
-  size_t zpart, zpart_bytes;                 // partial sums of layer 1's forward product that rides
-                                             // along with the weight-gradient launch (wgrad_tc.cuh)
+  size_t zcount, zcount_bytes;               // arrival counters of those partial sums
+  size_t zpart, zpart_bytes;                 // partial sums of a forward product that rides along
+                                             // with a weight-gradient launch (wgrad_tc.cuh); one
+                                             // layer at a time
   size_t w16b;                               // second bf16 copy of layer L-1's weights [P, w16b_stride]
   int64_t w16b_stride;
   size_t end;
@@ -63,18 +68,25 @@ struct TcState {
   CUtensorMap w_b, w_mn_b, w16_st_b;
   bool tail_ok = false;                       // the fused last-layer kernel covers the shape
   bool wgrad_merged = false;                  // all layers' weight gradients in one launch
-  // Layer 1's forward product of step k+1 formed inside step k's weight-gradient launch of that
-  // layer (see wgrad_tc.cuh): possible where that launch stands alone.  x_next[i]: the gathered
-  // batch buffer i as that launch reads it; f1_pending: the step about to be issued finds its
-  // first layer's product as partial sums; gathered_step: the step whose batch has already been
-  // gathered by the launch-by-launch form.
-  bool fuse_f1 = false;
-  bool f1_pending = false;
+  // Forward products of step k+1 formed inside step k's weight-gradient launches (see
+  // wgrad_tc.cuh), for layers 1..fuse_upto (0: none; at most L-1).  Possible where those launches
+  // stand alone.  Step k then runs, after its dgrad chain, for l = 1..fuse_upto: weight gradient +
+  // SGD of layer l with the forward product of W_l(k+1) and A_{l-1}(k+1) riding along, which
+  // leaves A_l(k+1) behind.  Steps alternate between two sets of
+  // activation buffers (A_l(k) is still read by layer l+1's weight gradient when A_l(k+1) is
+  // written); *_b are the views of the second set, a_next[l][i] the input of layer l in set i
+  // (l = 1: gather buffer i) as the riding product reads it.  fwd_done: how many leading
+  // layers of the step about to be issued already have their activations; gathered_step: the
+  // step whose batch has already been gathered by the launch-by-launch form.
+  int fuse_upto = 0;
+  int fwd_done = 0;
   int gathered_step = 0;
-  CUtensorMap x_next[2];
+  CUtensorMap act_in_b[MAVG_MAX_LAYERS + 1], act_in_t_b[MAVG_MAX_LAYERS + 1],
+      act_in_ks_b[MAVG_MAX_LAYERS + 1];
+  CUtensorMap a_next[MAVG_MAX_LAYERS + 1][2];
+  WgradPlan wgrad_f[MAVG_MAX_LAYERS + 1];     // plans of the launches that take a forward along
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
-  WgradPlan wgrad_f1;                         // layer 1's plan for the launches that take the forward along
   // side streams and events for the branches of a step that may overlap
   cudaStream_t s_wgrad = nullptr, s_gather = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_wgrad_done = nullptr, ev_gather_done = nullptr,

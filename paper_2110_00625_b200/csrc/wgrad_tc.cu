@@ -32,8 +32,8 @@ namespace {
 using namespace tc;
 using namespace wgrad;
 
-template <bool MOM>
-__global__ void __launch_bounds__(kThreads)
+template <bool MOM, bool FWD>
+__global__ void __launch_bounds__(FWD ? kThreadsFwd : kThreads)
 k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out, B]  load
                    const __grid_constant__ CUtensorMap tm_at,    // bf16 [P, in, B]   load
                    const __grid_constant__ CUtensorMap tm_w32,   // fp32 [P, out, in] store
@@ -59,14 +59,14 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
     tma_prefetch_desc(&tm_w32_in);
     tma_prefetch_desc(&tm_w16);
     if (MOM) tma_prefetch_desc(&tm_u);
-    if (g.fwd_next) tma_prefetch_desc(&tm_xn);
+    if (FWD && g.fwd_next) tma_prefetch_desc(&tm_xn);
     wgrad_init_barriers(sh, g.slots);
     sh.abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
   // two accumulators of 32 columns; with fwd_next a third of B columns behind them
-  const uint32_t tmem_cols = !g.fwd_next ? 64u : (g.batch <= 64 ? 128u : 256u);
+  const uint32_t tmem_cols = !(FWD && g.fwd_next) ? 64u : (g.batch <= 64 ? 128u : 256u);
   if (warp == 1) {
     tmem_alloc(&sh.tmem_slot, tmem_cols);
     tmem_relinquish();
@@ -76,7 +76,7 @@ k_wgrad_sgd_stream(const __grid_constant__ CUtensorMap tm_dzt,   // bf16 [P, out
   tc_fence_after_sync();
   const uint32_t tmem_base = sh.tmem_slot;
   grid_dependency_wait();
-  wgrad_run<MOM>(tm_dzt, tm_at, tm_w32, tm_w32_in, tm_w16, tm_u, tm_xn, g, (int)blockIdx.x,
+  wgrad_run<MOM, FWD>(tm_dzt, tm_at, tm_w32, tm_w32_in, tm_w16, tm_u, tm_xn, g, (int)blockIdx.x,
                  (int)gridDim.x, smem, sh, tmem_base);
   tc_fence_before_sync();
   __syncthreads();
@@ -123,55 +123,13 @@ k_wgrad_sgd_multi(const __grid_constant__ WgradMultiParams mp) {
   const int grid = (int)gridDim.x;
   for (int s = 0; s < mp.n; ++s) {
     const int vb = ((int)blockIdx.x + mp.rot[s]) % grid;
-    wgrad_run<MOM>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.w16[s],
+    wgrad_run<MOM, false>(mp.dzt[s], mp.at[s], mp.w32[s], mp.w32_in[s], mp.w16[s], mp.u[s], mp.w16[s],
                    mp.g[s], vb, grid, smem, sh, tmem_base, tiles, items);
     wgrad_run_totals(mp.g[s], vb, grid, tiles, items);
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, 64);
-}
-
-// Finishes the forward product that rode along with the previous step's weight-gradient launch:
-// adds a row tile's partial sums (one per run of column tiles) in ascending run order, adds the
-// bias, applies ReLU and writes A_l as bf16 in both orientations.  grid (row tiles, P); a thread
-// takes one output row and eight consecutive batch columns at a time.
-__global__ void __launch_bounds__(256)
-k_fwd_finish(const float* __restrict__ zpart, int n_chunks, int m_tiles, int M, int B,
-             const float* __restrict__ rep, int64_t rep_stride, int64_t bias_off,
-             __nv_bfloat16* __restrict__ out_bm, __nv_bfloat16* __restrict__ out_mb) {
-  const int mt = blockIdx.x, p = blockIdx.y;
-  const size_t tile_floats = (size_t)B * kBM;
-  const float* base = zpart + ((size_t)p * m_tiles + mt) * n_chunks * tile_floats;
-  for (int u = threadIdx.x; u < kBM * (B / 8); u += blockDim.x) {
-    const int r = u & (kBM - 1), b0 = (u / kBM) * 8;
-    const int m = mt * kBM + r;
-    if (m >= M) continue;
-    float z[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) z[j] = 0.f;
-    for (int nc = 0; nc < n_chunks; ++nc) {
-      const float* src = base + (size_t)nc * tile_floats + (size_t)b0 * kBM + r;
-      float t[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) t[j] = __ldcs(src + (size_t)j * kBM);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) z[j] += t[j];
-    }
-    const float bias = rep[(size_t)p * rep_stride + bias_off + m];
-    uint32_t h4[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float a0 = z[2 * j] + bias, a1 = z[2 * j + 1] + bias;
-      __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
-      h4[j] = *reinterpret_cast<uint32_t*>(&h2);
-    }
-    *reinterpret_cast<uint4*>(out_mb + ((size_t)p * M + m) * B + b0) =
-        make_uint4(h4[0], h4[1], h4[2], h4[3]);
-    const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(h4);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) out_bm[((size_t)p * B + b0 + j) * M + m] = hh[j];
-  }
 }
 
 }  // namespace
@@ -260,17 +218,17 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
 }
 
 cudaError_t wgrad_stream_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(k_wgrad_sgd_stream<false>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_wgrad_sgd_stream<true>,
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_wgrad_sgd_multi<false>,
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_wgrad_sgd_multi<true>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  const void* kernels[] = {(const void*)k_wgrad_sgd_stream<false, false>,
+                           (const void*)k_wgrad_sgd_stream<true, false>,
+                           (const void*)k_wgrad_sgd_stream<false, true>,
+                           (const void*)k_wgrad_sgd_stream<true, true>,
+                           (const void*)k_wgrad_sgd_multi<false>,
+                           (const void*)k_wgrad_sgd_multi<true>};
+  for (const void* k : kernels) {
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 namespace {
@@ -342,20 +300,27 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
                                 const CUtensorMap& at, const CUtensorMap& w32,
                                 const CUtensorMap& w16, const CUtensorMap* w32_shared,
                                 const CUtensorMap* u32, const MomArgs& mom,
-                                const CUtensorMap* xn, float* zpart) {
+                                const WgradFwdNext* fn) {
   WgradArgs g = make_args(c, w, w32_shared != nullptr, mom);
-  if (xn) {
+  if (fn) {
     // the plan must have been made with fwd_next (room for the input tile in every slot)
-    if (w.xn_bytes == 0) return cudaErrorInvalidValue;
+    if (w.xn_bytes == 0 || !fn->xn) return cudaErrorInvalidValue;
     g.fwd_next = 1;
-    g.store_w16 = 0;       // the only reader of this layer's bf16 copy is the product fused here
-    g.zpart = zpart;
+    g.store_w16 = fn->store_w16 ? 1 : 0;
+    g.zpart = fn->zpart;
+    g.zcount = fn->zcount;
+    g.bias_rep = c->buf.replicas;
+    g.rep_stride = c->buf.replica_stride;
+    g.bias_off = fn->bias_off;
+    g.out_rows = fn->out_rows;
+    g.out_bm = fn->out_bm;
+    g.out_mb = fn->out_mb;
   } else {
     g.xn_bytes = w.xn_bytes;   // the slot keeps its shape; the tile is simply not loaded
   }
   cudaLaunchConfig_t lc{};
   lc.gridDim = dim3((unsigned)w.grid);
-  lc.blockDim = dim3(kThreads);
+  lc.blockDim = dim3(fn ? kThreadsFwd : kThreads);
   lc.dynamicSmemBytes = w.smem;
   lc.stream = c->stream;
   cudaLaunchAttribute at_[1];
@@ -363,24 +328,19 @@ cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorM
   at_[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at_;
   lc.numAttrs = 1;
+  const bool with_u = mom.u && u32;
+  const CUtensorMap& w32_in = w32_shared ? *w32_shared : w32;
+  const CUtensorMap& um = with_u ? *u32 : w32;
   prof_begin(c, MAVG_K_WGRAD_SGD);
-  cudaError_t e = (mom.u && u32)
-      ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<true>, dzt, at, w32,
-                           w32_shared ? *w32_shared : w32, w16, *u32, xn ? *xn : w16, g)
-      : cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<false>, dzt, at, w32,
-                           w32_shared ? *w32_shared : w32, w16, w32, xn ? *xn : w16, g);
+  cudaError_t e;
+  if (fn)
+    e = with_u ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<true, true>, dzt, at, w32, w32_in, w16, um, *fn->xn, g)
+               : cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<false, true>, dzt, at, w32, w32_in, w16, um, *fn->xn, g);
+  else
+    e = with_u ? cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<true, false>, dzt, at, w32, w32_in, w16, um, w16, g)
+               : cudaLaunchKernelEx(&lc, k_wgrad_sgd_stream<false, false>, dzt, at, w32, w32_in, w16, um, w16, g);
   prof_end(c);
   return e != cudaSuccess ? e : cudaGetLastError();
-}
-
-cudaError_t launch_fwd_finish(mavg_ctx* c, const WgradPlan& w, int out, const float* zpart,
-                              int64_t bias_off, __nv_bfloat16* out_bm, __nv_bfloat16* out_mb) {
-  prof_begin(c, MAVG_K_FWD);
-  k_fwd_finish<<<dim3((unsigned)w.m_tiles, (unsigned)c->cfg.P), 256, 0, c->stream>>>(
-      zpart, w.n_chunks, w.m_tiles, out, c->cfg.B, c->buf.replicas, c->buf.replica_stride, bias_off,
-      out_bm, out_mb);
-  prof_end(c);
-  return cudaGetLastError();
 }
 
 }  // namespace mavg

@@ -31,21 +31,29 @@ cudaError_t wgrad_stream_prepare();
 // masters are then loaded from it for every learner (first step of a round, all w^j = w~) and
 // stored to w32 as always.  With learner-level momentum (mom.u set; the plan made with
 // momentum = true) u32 is the fp32 [P, out, in] view of the buffers u^j with w32's box.
-// xn, zpart (plans made with fwd_next only): xn is the bf16 [P, B, in] input of the NEXT local step
-// of this layer, box 32 x B (64B swizzle).  The launch then also forms that step's forward
-// product from the updated weight tiles while they are in shared memory,
-//   Z^T[out, B] = W_new[out, in] . Xn[B, in]^T,
-// as fp32 partial sums per work item in zpart (see WgradArgs), which launch_fwd_finish adds up,
-// and does NOT write the bf16 copy of the weights.
+// fn (plans made with fwd_next only): the launch also forms the NEXT local step's forward product
+// of this layer from the updated weight tiles while they are in shared memory,
+//   Z^T[out, B] = W_new[out, in] . Xn[B, in]^T,       A_next = relu(Z + b)  (bf16),
+// accumulated in tensor memory over each run of column tiles.  With several runs per row the
+// runs leave fp32 partial sums in zpart and the run that finishes last adds them up in ascending
+// run order (so the result does not depend on which one that was).
+struct WgradFwdNext {
+  const CUtensorMap* xn;   // bf16 [P, B, in]: the layer's input of the next step, box 32 x B (64B swizzle)
+  float* zpart;            // P x row tiles x runs x B x 128 floats
+  int* zcount;             // P x row tiles arrival counters, zero before (and again after) the launch
+  int64_t bias_off;        // the layer's bias in a learner's master vector
+  int out_rows;            // rows of the layer
+  __nv_bfloat16* out_bm;   // A_next [P, B, out]
+  __nv_bfloat16* out_mb;   // A_next [P, out, B]
+  bool store_w16;          // false: the bf16 copy of the weights is not written (a layer whose
+                           // copy nothing else reads before the next launch that writes it:
+                           // layer 1, which has no dgrad product)
+};
 cudaError_t launch_wgrad_stream(mavg_ctx* c, const WgradPlan& w, const CUtensorMap& dzt,
                                 const CUtensorMap& at, const CUtensorMap& w32,
                                 const CUtensorMap& w16, const CUtensorMap* w32_shared = nullptr,
                                 const CUtensorMap* u32 = nullptr, const MomArgs& mom = MomArgs(),
-                                const CUtensorMap* xn = nullptr, float* zpart = nullptr);
-// A_l = relu(sum of the plan's partial sums in ascending run order + b_l), as bf16 in both
-// orientations: out_bm [P, B, out], out_mb [P, out, B].  Biases from the masters.
-cudaError_t launch_fwd_finish(mavg_ctx* c, const WgradPlan& w, int out, const float* zpart,
-                              int64_t bias_off, __nv_bfloat16* out_bm, __nv_bfloat16* out_mb);
+                                const WgradFwdNext* fn = nullptr);
 
 // Several layers' weight-gradient + SGD tiles in one persistent launch (layers listed in the
 // order their tiles should run).  All plans must come from the same batch size and momentum

@@ -12,8 +12,8 @@ namespace wgrad {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 32, kBK = 64;
-constexpr int kThreads = 384;   // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores,
-                                // 11 forward MMAs (fwd_next)
+constexpr int kThreads = 352;      // warp 0 producer, 1 MMA, 2-5 / 6-9 epilogue groups, 10 stores
+constexpr int kThreadsFwd = 512;   // + warp 11 forward MMAs, 12-15 forward accumulator (fwd_next)
 constexpr int kMaxSlots = 6;
 constexpr int kW32Bytes = kBM * kBN * 4;  // 16 KB, rows of 128 bytes, 128-byte swizzle
 constexpr int kW16Bytes = kBM * kBN * 2;  //  8 KB, rows of  64 bytes,  64-byte swizzle
@@ -66,13 +66,24 @@ struct WgradArgs {
   // they are in shared memory (see wgrad_tc.cu): fwd_next = 1 adds, per tile,
   //   Z^T[128 rows, B] += W16_tile[128, 32] . Xn[B, 32]^T
   // into a third TMEM accumulator; per work item the fp32 partial sum goes to
-  //   zpart[((p * m_tiles + row tile) * n_chunks + chunk) * B * 128 + b * 128 + row].
+  //   zpart[((p * m_tiles + row tile) * n_chunks + chunk) * B * 128 + b * 128 + row]
+  // (not with a single run per row: then the accumulator is the whole product).
   int fwd_next;
   int store_w16;           // 0: the bf16 tile is not written to global memory
   int xn_bytes;            // room in a slot for the next step's input tile [B, 32] bf16 (loaded
                            // only with fwd_next; part of the slot's size whenever the plan has it)
   int batch;               // B
   float* zpart;
+  // the work item that completes a row tile's product last adds the partial sums up in ascending
+  // run order, adds the bias, applies ReLU and writes A_l of the next step as bf16 in both
+  // orientations (out_bm [P, B, out], out_mb [P, out, B]); zcount: one arrival counter per
+  // (learner, row tile), zero before and after the launch
+  int* zcount;
+  const float* bias_rep;   // masters [P, rep_stride]; the layer's bias at bias_off
+  int64_t rep_stride, bias_off;
+  int out_rows;            // rows of the layer (the last row tile may be ragged)
+  __nv_bfloat16* out_bm;
+  __nv_bfloat16* out_mb;
   int* status;
 };
 
@@ -83,6 +94,8 @@ struct WgradShared {
   uint64_t a_full[2], a_empty[2];
   uint64_t z_done[kMaxSlots];   // the forward MMAs that read this slot's bf16 tile have finished
   uint64_t z_full, z_empty;     // the item's forward accumulator is complete / has been read
+  uint64_t z_part, z_flag;      // the item's partial sum is in global memory / z_last is set
+  int z_last;                   // this item completed its row tile's product last
   uint32_t tmem_slot;
   int abort_flag;
 };
@@ -96,6 +109,8 @@ __device__ __forceinline__ void wgrad_init_barriers(WgradShared& sh, int slots) 
   }
   mbar_init(&sh.z_full, 1);
   mbar_init(&sh.z_empty, 4);
+  mbar_init(&sh.z_part, 4);
+  mbar_init(&sh.z_flag, 1);
   for (int b = 0; b < 2; ++b) {
     mbar_init(&sh.tmem_full[b], 1);
     mbar_init(&sh.tmem_empty[b], 4);
@@ -120,7 +135,8 @@ __device__ __forceinline__ void wgrad_run_totals(const WgradArgs& g, int vblock,
 // A block that makes several runs keeps using the same barriers (g.slots and g.a_bufs must not
 // change): tile_base and item_base are the tiles and items of its earlier runs, see
 // wgrad_run_totals.
-template <bool MOM>
+// FWD = false compiles the roles of the riding forward product out (g.fwd_next must be 0).
+template <bool MOM, bool FWD>
 __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUtensorMap& tm_at,
                                           const CUtensorMap& tm_w32, const CUtensorMap& tm_w32_in,
                                           const CUtensorMap& tm_w16, const CUtensorMap& tm_u,
@@ -128,6 +144,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
                                           const WgradArgs& g, int vblock, int vgrid, uint8_t* smem,
                                           WgradShared& sh, uint32_t tmem_base,
                                           uint32_t tile_base = 0, uint32_t item_base = 0) {
+  const bool fwd_next = FWD && g.fwd_next != 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = g.nkb * kBM * kBK * 2;         // dZ^T tile: nkb slabs of 16 KB
   const int b_bytes = g.nkb * kBN * kBK * 2;         // A^T tile:  nkb slabs of 4 KB
@@ -183,8 +200,8 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           const bool load_u = MOM && g.read_u;
           mbar_arrive_expect_tx(&sh.slot_full[s],
                                 (uint32_t)(kW32Bytes + b_bytes + (load_u ? kUBytes : 0) +
-                                           (g.fwd_next ? g.xn_bytes : 0)));
-          if (g.fwd_next) tma_load_3d(sl + xn_off, &tm_xn, &sh.slot_full[s], i0, 0, p);
+                                           (fwd_next ? g.xn_bytes : 0)));
+          if (fwd_next) tma_load_3d(sl + xn_off, &tm_xn, &sh.slot_full[s], i0, 0, p);
           tma_load_3d_hint(sl, &tm_w32_in, &sh.slot_full[s], i0, m0, g.w32_in_batched ? p : 0, pol);
           if (load_u) tma_load_3d(sl + kW32Bytes, &tm_u, &sh.slot_full[s], i0, m0, p);
           for (int kb = 0; kb < g.nkb; ++kb)
@@ -236,9 +253,9 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
     const int grp = (warp - 2) >> 2;           // epilogue group = TMEM buffer = tile parity
     const int q = warp & 3;                    // TMEM lane quarter this warp may read
     const int r = q * 32 + lane;               // weight row inside the tile
-    uint32_t tile_ctr = tile_base, item_ctr = item_base;
+    uint32_t tile_ctr = tile_base;
     bool ok = true;
-    for (int item = vblock; item < g.items && ok; item += vgrid, ++item_ctr) {
+    for (int item = vblock; item < g.items && ok; item += vgrid) {
       int p, m0, nt0, nt;
       decode(item, p, m0, nt0, nt);
       for (int j = 0; j < nt; ++j, ++tile_ctr) {
@@ -297,36 +314,6 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
         __syncwarp();                          // (and to the forward MMAs, fwd_next)
         if (lane == 0) mbar_arrive(&sh.out_full[s]);
       }
-      if (g.fwd_next && grp == 0 && ok) {
-        // the item's share of the next step's forward product: fp32 partial to global memory,
-        // one weight row per lane, a batch column per store (128 bytes per warp)
-        if (!mbar_wait(&sh.z_full, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
-          ok = false;
-          break;
-        }
-        tc_fence_after_sync();
-        float* zp = g.zpart +
-                    (((size_t)p * g.m_tiles + m0 / kBM) * g.n_chunks + nt0 / g.chunk) *
-                        ((size_t)g.batch * kBM) + r;
-        for (int c0 = 0; c0 < g.batch; c0 += 32) {
-          uint32_t acc[32];
-          if (c0 + 32 <= g.batch) {
-            tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, acc);
-          } else {                             // the batch is a multiple of 16
-            uint32_t h16[16];
-            tmem_ld_16cols(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, h16);
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) { acc[jj] = h16[jj]; acc[16 + jj] = 0u; }
-          }
-          tmem_ld_wait();
-#pragma unroll
-          for (int jj = 0; jj < 32; ++jj)
-            if (c0 + jj < g.batch) zp[(size_t)(c0 + jj) * kBM] = __uint_as_float(acc[jj]);
-        }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.z_empty);
-      }
     }
   } else if (warp == 10) {
     if (lane == 0) {
@@ -358,7 +345,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
           // (with fwd_next a slot is also still being read by its forward MMAs: z_done)
           if (held >= 0) {
             tma_store_wait_read<1>();
-            if (g.fwd_next && !mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE)) {
+            if (fwd_next && !mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE)) {
               ok = false;
               break;
             }
@@ -372,7 +359,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
               held_use = use;
             } else {
               tma_store_wait_read<0>();
-              if (g.fwd_next && !mbar_wait(&sh.z_done[s], use & 1, abortp, g.status, ERR_WG_STORE)) {
+              if (fwd_next && !mbar_wait(&sh.z_done[s], use & 1, abortp, g.status, ERR_WG_STORE)) {
                 ok = false;
                 break;
               }
@@ -383,15 +370,15 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       }
       if (held >= 0) {
         tma_store_wait_read<0>();
-        if (!g.fwd_next || mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE))
+        if (!fwd_next || mbar_wait(&sh.z_done[held], held_use & 1, abortp, g.status, ERR_WG_STORE))
           mbar_arrive(&sh.slot_empty[held]);
       }
     }
     __syncwarp();
-  } else {
-    // warp 11 (fwd_next): the forward MMAs of a tile, issued as soon as the epilogue has put the
+  } else if (warp == 11) {
+    // (fwd_next) the forward MMAs of a tile, issued as soon as the epilogue has put the
     // updated bf16 tile into its slot; they read that tile and the next step's input tile beside it
-    if (lane == 0 && g.fwd_next) {
+    if (lane == 0 && fwd_next) {
       const uint32_t idesc_z = idesc_bf16_f32(kBM, g.batch);
       uint32_t tile_ctr = tile_base, item_ctr = item_base;
       bool ok = true;
@@ -424,6 +411,113 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       }
     }
     __syncwarp();
+  } else if (fwd_next) {
+    // warps 12-15: the forward accumulator of every work item.  One weight row per lane (warp w
+    // reads TMEM lanes 32 (w % 4) ...), 32 batch columns at a time.
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const bool single = g.n_chunks == 1;
+    const size_t tile_floats = (size_t)g.batch * kBM;
+    uint32_t item_ctr = item_base;
+    for (int item = vblock; item < g.items; item += vgrid, ++item_ctr) {
+      int p, m0, nt0, nt;
+      decode(item, p, m0, nt0, nt);
+      const int mt = m0 / kBM;
+      const int m = m0 + r;
+      const bool row_ok = m < g.out_rows;
+      const float bias = row_ok ? g.bias_rep[(size_t)p * g.rep_stride + g.bias_off + m] : 0.f;
+      // A_l of the next step from 32 (or the last 16) finished columns of this lane's row
+      auto emit = [&](int c0, const float* z) {
+        if (!row_ok) return;
+        const int nc = min(32, g.batch - c0);
+        uint32_t h[16];
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+          const float a0 = z[2 * jj] + bias, a1 = z[2 * jj + 1] + bias;
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 > 0.f ? a0 : 0.f, a1 > 0.f ? a1 : 0.f);
+          h[jj] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        uint4* dmb = reinterpret_cast<uint4*>(g.out_mb + ((size_t)p * g.out_rows + m) * g.batch + c0);
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          if (8 * v < nc) dmb[v] = make_uint4(h[4 * v], h[4 * v + 1], h[4 * v + 2], h[4 * v + 3]);
+        const __nv_bfloat16* hh = reinterpret_cast<const __nv_bfloat16*>(h);
+        __nv_bfloat16* dbm = g.out_bm + ((size_t)p * g.batch + c0) * g.out_rows + m;
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj)
+          if (jj < nc) dbm[(size_t)jj * g.out_rows] = hh[jj];
+      };
+      if (!mbar_wait_relaxed(&sh.z_full, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE, 400)) break;
+      tc_fence_after_sync();
+      float* zbase = g.zpart + ((size_t)p * g.m_tiles + mt) * g.n_chunks * tile_floats + r;
+      float* zp = zbase + (size_t)(nt0 / g.chunk) * tile_floats;
+      for (int c0 = 0; c0 < g.batch; c0 += 32) {
+        uint32_t acc[32];
+        if (c0 + 32 <= g.batch) {
+          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, acc);
+        } else {                             // the batch is a multiple of 16
+          uint32_t h16[16];
+          tmem_ld_16cols(tmem_base + ((uint32_t)(q * 32) << 16) + kZCol + (uint32_t)c0, h16);
+#pragma unroll
+          for (int jj = 0; jj < 16; ++jj) { acc[jj] = h16[jj]; acc[16 + jj] = 0u; }
+        }
+        tmem_ld_wait();
+        if (single) {
+          emit(c0, reinterpret_cast<const float*>(acc));
+        } else {
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj)
+            if (c0 + jj < g.batch) zp[(size_t)(c0 + jj) * kBM] = __uint_as_float(acc[jj]);
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.z_empty);
+      if (single) continue;
+      // Whichever item of the row tile gets here last finishes the row tile.  The 128 lanes'
+      // partial-sum stores are ordered before one lane's gpu-scope release on the counter by the
+      // block-scope arrive/wait on z_part (the orders compose); on the other side that lane's
+      // acquire on the counter is ordered before the 128 lanes' loads by z_flag, and the loads
+      // go to the L2 (no stale L1 line can serve them).
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.z_part);
+      if (warp == 12 && lane == 0 &&
+          mbar_wait(&sh.z_part, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
+        int* cnt = g.zcount + (size_t)p * g.m_tiles + mt;
+        int old;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
+        const int last = old == g.n_chunks - 1;
+        if (last) *cnt = 0;
+        sh.z_last = last;
+        mbar_arrive(&sh.z_flag);
+      }
+      __syncwarp();
+      if (!mbar_wait(&sh.z_flag, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) break;
+      if (!sh.z_last) continue;
+      for (int c0 = 0; c0 < g.batch; c0 += 32) {
+        float z[32];
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) z[jj] = 0.f;
+        // two runs' loads in flight at a time; the sums are formed in ascending run order
+        for (int nc = 0; nc < g.n_chunks; nc += 2) {
+          const float* s0 = zbase + (size_t)nc * tile_floats + (size_t)c0 * kBM;
+          const bool two = nc + 1 < g.n_chunks;
+          float a[32], b[32];
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            const bool in = c0 + jj < g.batch;
+            a[jj] = in ? __ldcg(s0 + (size_t)jj * kBM) : 0.f;
+            b[jj] = in && two ? __ldcg(s0 + tile_floats + (size_t)jj * kBM) : 0.f;
+          }
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            z[jj] += a[jj];
+            if (two) z[jj] += b[jj];
+          }
+        }
+        emit(c0, z);
+      }
+    }
   }
 }
 

@@ -319,35 +319,49 @@ def test_tc_mixed_call_sequences_keep_the_same_bits():
         assert np.array_equal(x, y)
 
 
-# A model whose first layer has more weight tiles than the one-launch-for-all-layers form takes
-# (13 x 8 x 96 > 64 per SM): its layer-1 weight gradient is a launch of its own, and that launch
-# also forms the NEXT step's layer-1 forward product from the updated tiles (steps 1..K-1).
-FUSED_DIMS, FUSED_P, FUSED_B = [3072, 1024, 10], 13, 16
+# Models whose first layer has more weight tiles than the one-launch-for-all-layers form takes
+# (13 x 8 x 96 > 64 per SM): every layer's weight gradient is a launch of its own, and the launches
+# of the hidden layers also form the NEXT step's forward product of their layer from the updated
+# tiles (steps 1..K-1): one hidden layer, and two (the second one's launch reads the activations
+# the first one's has just produced, and still writes its bf16 copy for the dgrad product).
+FUSED_SHAPES = [[3072, 1024, 10], [3072, 1024, 512, 10]]
+FUSED_P, FUSED_B = 13, 16
 
 
-def _fused_handle(K, **kw):
+def _fused_handle(dims, K, **kw):
     m = _mavg()
     cfg = dict(m.workloads.CONFIGS["C2"])
-    cfg.update(dims=FUSED_DIMS, P=FUSED_P, K=K, B=FUSED_B, S=4096)
+    cfg.update(dims=dims, P=FUSED_P, K=K, B=FUSED_B, S=4096)
     x, y = m.workloads.make_dataset(cfg, S=cfg["S"])
     w1 = m.workloads.mlp_init(cfg["dims"])
     g = m.Mavg(w1, P=FUSED_P, K=K, local_lr=cfg["gamma"], mu=cfg["mu"], B=FUSED_B,
-               seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=FUSED_DIMS, gemm_bf16=1,
+               seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=dims, gemm_bf16=1,
                x=x, y=y, x_bf16=True, **kw)
     return g, cfg, x, y, w1
 
 
+# Per-tile bounds: with 16 samples per batch a single ReLU decision that differs between the two
+# roundings moves a whole weight row's gradient by 1/16 of itself, and three steps through two
+# hidden layers collect more of those than the one-hidden-layer model (measured: the schedule that
+# does not ride shows the same per-tile distances to the oracle, worst 0.033 against 0.034, and the
+# two schedules are 0.004 apart); a wrong tile is off by ~1.
+FUSED_TILE_TOL = {2: dict(l2_tol=2e-2, frac=0.05), 3: dict(l2_tol=5e-2, frac=0.15)}
+FUSED_STEP_TOL = {2: 3e-2, 3: 5e-2}        # whole step of a learner; 5e-2 is the bf16 gate
+
+
+@pytest.mark.parametrize("dims", FUSED_SHAPES)
 @pytest.mark.parametrize("beta", [0.0, 0.9])
-def test_forward_riding_on_the_weight_gradient_against_the_oracle(oracle, beta):
-    # K = 3 local steps from identical replicas: step 1 plain, steps 2 and 3 take their first
-    # layer's forward product from the partial sums the step before left; per learner, per tile
-    g, cfg, x, y, w1 = _fused_handle(3, learner_momentum=beta)
+def test_forward_riding_on_the_weight_gradient_against_the_oracle(oracle, dims, beta):
+    # K = 3 local steps from identical replicas: step 1 plain, steps 2 and 3 take their hidden
+    # layers' forward products from the partial sums the step before left; per learner, per tile
+    g, cfg, x, y, w1 = _fused_handle(dims, 3, learner_momentum=beta)
     plan = g.get_step_plan()
-    assert plan["tensor_path"] == 1 and plan["wgrad_merged"] == 0 and plan["fwd_with_wgrad"] == 1
-    assert 8 <= plan["fwd_run_tiles"] <= FUSED_DIMS[0] // 32
+    assert plan["tensor_path"] == 1 and plan["wgrad_merged"] == 0
+    assert plan["fwd_with_wgrad"] == len(dims) - 2
+    assert all(8 <= r <= d // 32 for r, d in zip(plan["fwd_run_tiles"], dims))
     xq = oracle.bf16_round(x)             # the GPU holds the dataset in bf16
     o = oracle.Mavg(w1, P=FUSED_P, K=3, gamma=cfg["gamma"], mu=cfg["mu"], B=FUSED_B,
-                    seed=_mavg().workloads.BASE_SEED, objective=oracle.OBJ_MLP, dims=FUSED_DIMS,
+                    seed=_mavg().workloads.BASE_SEED, objective=oracle.OBJ_MLP, dims=dims,
                     bf16=True, x=xq, y=y, stride=g.stride, beta=beta)
     g.local_steps()
     losses_o, _ = o.local_steps()
@@ -357,8 +371,8 @@ def test_forward_riding_on_the_weight_gradient_against_the_oracle(oracle, beta):
     for j in range(FUSED_P):
         step_g = gr[j, :g.n].astype(np.float64) - w1
         step_o = o.replicas[j, :g.n].astype(np.float64) - w1
-        assert l2_rel(step_g, step_o) <= 3e-2, j
-        assert_tiles_close(step_g, step_o, FUSED_DIMS, what=f"learner {j}")
+        assert l2_rel(step_g, step_o) <= FUSED_STEP_TOL[len(dims) - 1], j
+        assert_tiles_close(step_g, step_o, dims, what=f"learner {j}", **FUSED_TILE_TOL[len(dims) - 1])
     # the bf16 copy of layer 1 is valid again after the call's last step: a second call without a
     # meta-update in between starts from the learners' own weights and must agree as well
     g.local_steps()
@@ -368,10 +382,11 @@ def test_forward_riding_on_the_weight_gradient_against_the_oracle(oracle, beta):
     g.close()
 
 
-def test_forward_riding_on_the_weight_gradient_graph_equals_launch_by_launch():
+@pytest.mark.parametrize("dims", FUSED_SHAPES)
+def test_forward_riding_on_the_weight_gradient_graph_equals_launch_by_launch(dims):
     outs = []
     for profiled in (False, False, True):
-        g, *_ = _fused_handle(4)
+        g, *_ = _fused_handle(dims, 4)
         g.set_profiling(profiled)
         losses = [g.round(want_loss=True) for _ in range(2)]
         g.local_steps(); g.local_steps(); g.meta_update()      # a call that starts from diverged replicas
@@ -382,11 +397,14 @@ def test_forward_riding_on_the_weight_gradient_graph_equals_launch_by_launch():
         assert np.array_equal(outs[0][0], other[0]) and np.array_equal(outs[0][1], other[1])
         assert outs[0][2] == other[2] and np.array_equal(outs[0][3], other[3])
     # and it computes what the plain-tiles schedule computes, to rounding order
-    a, *_ = _fused_handle(4)
-    b, *_ = _fused_handle(4)
+    a, *_, a_w1 = _fused_handle(dims, 4)
+    b, *_ = _fused_handle(dims, 4)
     b.set_schedule(2)
     la, lb = a.round(want_loss=True), b.round(want_loss=True)
     a.sync(); b.sync()
     assert abs(la - lb) <= 1e-3 * abs(lb)
     assert l2_rel(a.v.cpu().numpy(), b.v.cpu().numpy()) <= 2e-2
+    ra, rb = a.replicas.cpu().numpy(), b.replicas.cpu().numpy()    # re-broadcast: all rows = w~
+    assert_tiles_close(ra[0, :a.n].astype(np.float64) - a_w1, rb[0, :a.n].astype(np.float64) - a_w1,
+                       dims, what="riding against plain tiles", l2_tol=2e-2, frac=0.05)
     a.close(); b.close()

@@ -216,7 +216,11 @@ typedef enum {
                                    (m <= L-1; layer 1's bf16 copy is not written in those steps) */
   MAVG_PLAN_FWD_RUN_TILES = 3,  /* first of MAVG_MAX_LAYERS entries: for layer l <= m, entry
                                    3 + l - 1 is the number of column tiles per partial sum */
-  MAVG_PLAN_COUNT = 3 + MAVG_MAX_LAYERS
+  MAVG_PLAN_DENSE_FIRST_STEP = 3 + MAVG_MAX_LAYERS, /* bit l-1 set: under the default schedule the
+                                   forward product of hidden layer l at the first step of a round
+                                   (all learners hold w~) is one dense product over the batch rows
+                                   of all learners, the weights read once */
+  MAVG_PLAN_COUNT = 4 + MAVG_MAX_LAYERS
 } mavg_plan_entry;
 mavg_status mavg_get_step_plan(mavg_handle h, int32_t *out);
 

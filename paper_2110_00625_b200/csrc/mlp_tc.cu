@@ -539,6 +539,22 @@ mavg_status tc_setup(mavg_ctx* c) {
       st->fuse_upto = l;
     }
   }
+  // First step of a round: the hidden layers' forward products as one dense product each, where
+  // that gives enough tiles (the input buffers seen as one [P*B, in] array).
+  for (int l = 1; l <= L; ++l) st->dense[l] = DensePlan{};
+  for (int l = 1; l < L && ok; ++l) {
+    const int in = cfg.dims[l - 1];
+    DensePlan pl = plan_fwd_dense(cfg.dims[l], in, B, P, c->sm_count);
+    if (!pl.ok) continue;
+    bool enc = true;
+    for (int i = 0; i < 2 && enc; ++i) {
+      const size_t src = l == 1 ? t.xg[i] : (i == 0 ? t.act[l - 1] : t.act_b[l - 1]);
+      enc = encode_map(st, &st->in2d[l][i], bf(src), in, P * B, 1, in, (int64_t)P * B * in,
+                       kDenseCols, &why);
+    }
+    if (enc) st->dense[l] = pl;
+  }
+  if (e == cudaSuccess) e = fwd_dense_prepare();
   // the meta-update writes the bf16 copy of w~ itself where its vector kernel takes the whole model
   c->shadow.dst = (__nv_bfloat16*)(ws + t.w16g);
   c->shadow.L = L;
@@ -594,6 +610,8 @@ void tc_step_plan(mavg_ctx* c, int32_t* out) {
   out[MAVG_PLAN_WGRAD_MERGED] = st->wgrad_merged ? 1 : 0;
   out[MAVG_PLAN_FWD_WITH_WGRAD] = st->fuse_upto;
   for (int l = 1; l <= st->fuse_upto; ++l) out[MAVG_PLAN_FWD_RUN_TILES + l - 1] = st->wgrad_f[l].chunk;
+  for (int l = 1; l <= MAVG_MAX_LAYERS; ++l)
+    if (st->dense[l].ok) out[MAVG_PLAN_DENSE_FIRST_STEP] |= 1 << (l - 1);
 }
 
 cudaError_t tc_refresh_shared_operands(mavg_ctx* c) {
@@ -714,6 +732,10 @@ cudaError_t tc_step(mavg_ctx* c, int64_t round, int step) {
     const CUtensorMap& am = l == 1 ? st->x_in[xb] : act_in(l);
     if (l <= done) {
       // A_l of this step came out of the previous step's weight-gradient launch of this layer
+    } else if (l < L && shared_w && c->schedule == 0 && st->dense[l].ok) {
+      // every learner holds w~: one dense product over the batch rows of all learners
+      TC_TRY(launch_fwd_dense(c, st->dense[l], st->wg[l], st->in2d[l][l == 1 ? xb : ab], ly.out,
+                              c->buf.global_w + ly.b_off, act_of(l, ab), act_t_of(l, ab)));
     } else if (l < L) {
       g.out_bm = act_of(l, ab); g.out_mb = act_t_of(l, ab);
       if (c->schedule == 0 && st->fwd_ks[l].splits > 1)

@@ -4,6 +4,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "fwd_dense.cuh"
 #include "wgrad_tc.cuh"
 
 namespace mavg {
@@ -85,6 +86,11 @@ struct TcState {
       act_in_ks_b[MAVG_MAX_LAYERS + 1];
   CUtensorMap a_next[MAVG_MAX_LAYERS + 1][2];
   WgradPlan wgrad_f[MAVG_MAX_LAYERS + 1];     // plans of the launches that take a forward along
+  // First local step of a round (all learners hold w~): hidden layer l's forward as one dense
+  // product over the batch rows of all learners (fwd_dense.cuh) where dense[l].ok; in2d[l][i]:
+  // the layer's input in buffer set i (l = 1: gather buffer i) as one [P*B, d_{l-1}] array.
+  DensePlan dense[MAVG_MAX_LAYERS + 1];
+  CUtensorMap in2d[MAVG_MAX_LAYERS + 1][2];
   GemmPlan fwd[MAVG_MAX_LAYERS + 1], dgrad[MAVG_MAX_LAYERS + 1];
   WgradPlan wgrad[MAVG_MAX_LAYERS + 1];
   // side streams and events for the branches of a step that may overlap

@@ -408,3 +408,43 @@ def test_forward_riding_on_the_weight_gradient_graph_equals_launch_by_launch(dim
     assert_tiles_close(ra[0, :a.n].astype(np.float64) - a_w1, rb[0, :a.n].astype(np.float64) - a_w1,
                        dims, what="riding against plain tiles", l2_tol=2e-2, frac=0.05)
     a.close(); b.close()
+
+
+def test_dense_first_step_forward_against_the_oracle(oracle):
+    # At the first step of a round all learners hold w~ and the hidden layers' forward products
+    # run as one dense product over the batch rows of all learners (128 x 256 tiles).  Shape with
+    # a contraction tail (200 = 3 x 64 + 8), a ragged last row tile (520 = 4 x 128 + 8) and a last
+    # batch tile that is three quarters full (39 x 64 = 9.75 x 256); K = 2, so that the second
+    # step (per-learner weights, per-learner tiles) starts from what the dense step produced.
+    m = _mavg()
+    dims, B, P, K = [200, 1024, 520, 10], 64, 39, 2
+    S = 4 * P * B
+    r = np.random.default_rng(23)
+    x = r.standard_normal((S, dims[0])).astype(np.float32)
+    y = r.integers(0, dims[-1], S).astype(np.int32)
+    w1 = m.workloads.mlp_init(dims, seed=6)
+    g = m.Mavg(w1, P=P, K=K, local_lr=0.05, mu=0.9, B=B, seed=77, objective=m.OBJ_MLP, dims=dims,
+               gemm_bf16=1, x=x, y=y)
+    assert g.get_step_plan()["dense_first_step"] == [1, 2]
+    o = oracle.Mavg(w1, P=P, K=K, gamma=0.05, mu=0.9, B=B, seed=77, objective=oracle.OBJ_MLP,
+                    dims=dims, bf16=True, x=x, y=y, stride=g.stride)
+    g.local_steps()
+    losses_o, _ = o.local_steps()
+    g.sync()
+    gr = g.replicas.cpu().numpy()
+    # the first step's losses depend on nothing but the dense products and the last layer
+    assert np.abs(g.get_losses()[:, 0] - losses_o[:, 0]).max() <= 2e-3 * losses_o[:, 0].max()
+    assert np.abs(g.get_losses() - losses_o).max() <= 2e-2 * losses_o.max()
+    for j in (0, 3, 17, P - 2, P - 1):          # first and last learners of full and ragged tiles
+        step_g = gr[j, :g.n].astype(np.float64) - w1
+        step_o = o.replicas[j, :g.n].astype(np.float64) - w1
+        assert l2_rel(step_g, step_o) <= 3e-2, j
+        assert_tiles_close(step_g, step_o, dims, what=f"learner {j}")
+    # the plain-tiles schedule forms the same first-step products per learner: same losses
+    h = m.Mavg(w1, P=P, K=K, local_lr=0.05, mu=0.9, B=B, seed=77, objective=m.OBJ_MLP, dims=dims,
+               gemm_bf16=1, x=x, y=y)
+    h.set_schedule(2)
+    h.local_steps()
+    h.sync()
+    assert np.abs(h.get_losses()[:, 0] - g.get_losses()[:, 0]).max() <= 1e-4 * losses_o[:, 0].max()
+    g.close(); h.close()

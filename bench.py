@@ -235,20 +235,25 @@ NCU_TRAFFIC = {
 }
 
 
-def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=()):
+def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=(),
+                      dense_layers=()):
     """Bytes that must cross HBM per ROUND for each kernel class (weights streamed once per
     product, activations in and out), and their total.  fwd_run_tiles[l-1], layers l = 1..m: in
     steps 1..K-1 the weight-gradient launch of layer l also forms the next step's forward product
     of that layer: its bf16 weights are not read by a forward kernel in steps 2..K (layer 1's copy
     is not even written); the layer's next input is read and its next activations are written by
     the weight-gradient launch, which also writes and reads back one fp32 partial sum [128, B]
-    per learner, row tile and run of fwd_run_tiles[l-1] column tiles."""
+    per learner, row tile and run of fwd_run_tiles[l-1] column tiles; the flops move with them.
+    dense_layers: hidden layers whose first-step forward is one dense product over all learners'
+    batch rows, reading the (shared) weights once instead of once per learner."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
     L = len(dims) - 1
     nW = [dims[l] * dims[l + 1] for l in range(L)]
     n = sum(nW) + sum(dims[1:])
     rows = P * B
-    fwd_delta = wgrad_delta = 0
+    fwd_delta = wgrad_delta = flop_delta = 0
+    for l in dense_layers:
+        fwd_delta -= 2 * (P - 1) * nW[l - 1]
     for i, run in enumerate(fwd_run_tiles if K > 1 else ()):
         n_tiles = -(-dims[i] // 32)
         runs = -(-n_tiles // run)
@@ -256,6 +261,7 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_
         moved = 2 * rows * dims[i] + 4 * rows * dims[i + 1]     # the layer's input read, A_l written twice
         fwd_delta -= (K - 1) * (2 * P * nW[i] + moved)
         wgrad_delta += (K - 1) * (moved + 2 * partial - (2 * P * nW[0] if i == 0 else 0))
+        flop_delta += (K - 1) * 2 * rows * nW[i]
     per_round = {
         # replicas, w~, v read; v, w~ and (unless the copies are deferred) the replicas written
         "meta_update": dict(bytes=((4 if deferred else 8) * P + 16) * n, flops=0),
@@ -272,14 +278,16 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_
                                flops=K * 2 * rows * sum(nW)),
     }
     per_round["fwd_gemm"]["bytes"] += fwd_delta
+    per_round["fwd_gemm"]["flops"] -= flop_delta
     per_round["wgrad_sgd_gemm"]["bytes"] += wgrad_delta
+    per_round["wgrad_sgd_gemm"]["flops"] += flop_delta
     return per_round
 
 
 def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False,
-                     fwd_run_tiles=()):
+                     fwd_run_tiles=(), dense_layers=()):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
-    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles)
+    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles, dense_layers)
     out = {}
     for name, (ms, cnt) in prof.items():
         if cnt == 0 or ms <= 0:
@@ -511,8 +519,10 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
     g.set_profiling(False)
     plan = g.get_step_plan()
     fwd_run_tiles = tuple(plan["fwd_run_tiles"]) if args.schedule == 0 else ()
+    dense_layers = tuple(plan["dense_first_step"]) if args.schedule == 0 else ()
     kern = kernel_rooflines(cfg, prof, psteps, peaks, mode == 1, deferred=not args.no_defer,
-                            momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles)
+                            momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles,
+                            dense_layers=dense_layers)
     n = g.n
     g.close()
     del g, flush
@@ -545,11 +555,13 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
             roof["traffic"] = NCU_TRAFFIC.get(name, {}).get(dom)
     # the whole round against the HBM roofline: every class's algorithmic bytes / the round's time
     per_round = algorithmic_bytes(cfg, mode == 1, deferred=not args.no_defer,
-                                  momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles)
+                                  momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles,
+                                  dense_layers=dense_layers)
     round_bytes = sum(v["bytes"] for v in per_round.values())
     ms_round = total_ms / steps
     return dict(
-        cfg=cfg, n=n, units=units, fwd_run_tiles=fwd_run_tiles, total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
+        cfg=cfg, n=n, units=units, fwd_run_tiles=fwd_run_tiles, dense_layers=dense_layers,
+        total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
         clocks=clocks, cpu=cpu, kern=kern, roof=roof, t_wall=t_wall, mode=mode,
         meta_in_round={"ms": statistics.median(meta_ms),
                        "gbs": per_round["meta_update"]["bytes"] / statistics.median(meta_ms) / 1e6},
@@ -618,6 +630,9 @@ def run_mavg(args):
                                             "launch of the step before (steps 2..K; partial sums per "
                                             f"{list(r['fwd_run_tiles'])} column tiles)"
                                             if r["fwd_run_tiles"] else "launches of their own"),
+                       "first_step_forward": (f"layers {list(r['dense_layers'])}: one dense product over the "
+                                              "batch rows of all learners" if r["dense_layers"]
+                                              else "per-learner tiles reading the one bf16 copy of the global model"),
                        "l2": "flushed between steps by a 256 MiB memset, outside the step's events",
                        "kernel_timing": "second pass over the same steps with one event pair per launch"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],

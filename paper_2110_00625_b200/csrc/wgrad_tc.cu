@@ -177,15 +177,19 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   // partial sum going to global memory (and coming back once): long runs keep that traffic small
   // against the 2 x 2 bytes per weight the fusion saves.
   // Among the even splits of a row of column tiles, take the one whose busiest block finishes
-  // first: ceil(items / blocks) items of (run + one tile's worth of per-item work) each.
+  // first: ceil(items / blocks) items of (run + per-item work) each.  The per-item work -- the
+  // next dZ^T tile, reading the forward accumulator, the partial sum and its share of the sums
+  // over all runs of a row, during which the next item's forward products wait -- is worth about
+  // six tile periods (measured with 8 learners: runs of 8 tiles took 150 us per launch where runs
+  // of 32 to 48 take 75 us).
   if (fwd_next) {
     long best_cost = 0;
     for (int nc = 1; nc <= w.n_tiles; ++nc) {
       const long run = (w.n_tiles + nc - 1) / nc;
       if (run > kWgradFwdChunk) continue;
-      if (run < 8 && best_cost) break;
+      if (run < 16 && best_cost) break;
       const long items = (long)P * w.m_tiles * ((w.n_tiles + run - 1) / run);
-      const long cost = ((items + sm_count - 1) / sm_count) * (run + 1);
+      const long cost = ((items + sm_count - 1) / sm_count) * (run + 6);
       if (!best_cost || cost < best_cost) {
         best_cost = cost;
         chunk = run;

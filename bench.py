@@ -229,9 +229,9 @@ def run_reference(args):
 # kernels and tile plans) and scaled by 4, since every kernel's traffic is proportional to P.
 NCU_TRAFFIC = {
     "C2": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
-    # profiles/step_kernels_c4_p8.md: sums over one step's launches of the class at P = 8, times 4,
-    # divided by the launches of the class (4 weight-gradient, 4 forward, 3 dgrad launches per step)
-    "C4": {"wgrad_sgd_gemm": None, "fwd_gemm": None, "dgrad_gemm": None},
+    # profiles/step_kernels_c4_p8.md: sums over a middle step's launches of the class at P = 8,
+    # times 4, divided by the launches of the class (4 weight-gradient, 1 forward, 3 dgrad)
+    "C4": {"wgrad_sgd_gemm": 954.2e6, "fwd_gemm": 10.2e6, "dgrad_gemm": 198.4e6},
 }
 
 

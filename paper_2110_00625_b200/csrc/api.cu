@@ -544,6 +544,7 @@ mavg_status mavg_sync(mavg_handle h) {
     char msg[96];
     snprintf(msg, sizeof msg, "a device-side wait ran out (code %d)", flag);
     cudaMemsetAsync(ws_ptr(h, h->ws.status), 0, sizeof(int32_t), h->stream);
+    if (h->cfg.objective == MAVG_OBJ_MLP) mlp_reset_counters(h);
     return set_err(h, MAVG_ERR_TIMEOUT, msg);
   }
   return MAVG_OK;

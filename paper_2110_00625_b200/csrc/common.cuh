@@ -174,6 +174,7 @@ mavg_status mlp_setup(mavg_ctx* c);
 void mlp_teardown(mavg_ctx* c);
 cudaError_t mlp_refresh_shared_operands(mavg_ctx* c);   // after w~ changed
 cudaError_t mlp_local_steps(mavg_ctx* c, int64_t round);
+void mlp_reset_counters(mavg_ctx* c);                    // after an abandoned device-side wait
 void mlp_step_plan(mavg_ctx* c, int32_t* out);           // entries of mavg_plan_entry
 cudaError_t mlp_indices_only(mavg_ctx* c, int64_t round, int learner, int step, int32_t* dev_out);
 

@@ -47,6 +47,10 @@ void mlp_teardown(mavg_ctx* c) {
   if (c->mlp) tc_teardown(c);
 }
 
+void mlp_reset_counters(mavg_ctx* c) {
+  if (c->mlp) tc_reset_counters(c);
+}
+
 void mlp_step_plan(mavg_ctx* c, int32_t* out) {
   if (c->mlp) tc_step_plan(c, out);
 }

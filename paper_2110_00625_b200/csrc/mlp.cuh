@@ -61,6 +61,7 @@ cudaError_t tail_fused_prepare();
 cudaError_t launch_tail_fused(mavg_ctx* c, const TailLaunch& t);    // the products, dZ, partial sums
 cudaError_t launch_tail_finish(mavg_ctx* c, const TailLaunch& t);   // bias steps and loss from the partials
 
+void tc_reset_counters(mavg_ctx* c);          // after an abandoned device-side wait
 void tc_step_plan(mavg_ctx* c, int32_t* out);  // entries of mavg_plan_entry
 int tc_get_w16_cur(mavg_ctx* c);            // which bf16 copy of the doubled layer is current
 void tc_set_w16_cur(mavg_ctx* c, int cur);

@@ -603,6 +603,17 @@ void tc_set_w16_cur(mavg_ctx* c, int cur) {
   if (c->mlp) ((TcState*)c->mlp)->w16_cur = cur;
 }
 
+// After an abandoned wait the arrival counters of split tiles and of riding forward products may
+// have been left mid-count: zero them (stream-ordered), so that the handle's next launches count
+// from a clean state.
+void tc_reset_counters(mavg_ctx* c) {
+  const TcState* st = (const TcState*)c->mlp;
+  if (!st) return;
+  char* ws = (char*)c->buf.workspace;
+  cudaMemsetAsync(ws + st->lay.counters, 0, st->lay.counters_bytes, c->stream);
+  cudaMemsetAsync(ws + st->lay.zcount, 0, st->lay.zcount_bytes, c->stream);
+}
+
 void tc_step_plan(mavg_ctx* c, int32_t* out) {
   const TcState* st = (const TcState*)c->mlp;
   if (!st) return;

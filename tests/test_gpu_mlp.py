@@ -393,6 +393,13 @@ def test_forward_riding_on_the_weight_gradient_graph_equals_launch_by_launch(dim
         g.sync()
         outs.append((g.w.cpu().numpy(), g.v.cpu().numpy(), losses, g.get_losses()))
         g.close()
+    # the same calls with the re-broadcast left to the next round's first step
+    g, *_ = _fused_handle(dims, 4, defer_broadcast=True)
+    losses = [g.round(want_loss=True) for _ in range(2)]
+    g.local_steps(); g.local_steps(); g.meta_update()
+    g.sync()
+    outs.append((g.w.cpu().numpy(), g.v.cpu().numpy(), losses, g.get_losses()))
+    g.close()
     for other in outs[1:]:
         assert np.array_equal(outs[0][0], other[0]) and np.array_equal(outs[0][1], other[1])
         assert outs[0][2] == other[2] and np.array_equal(outs[0][3], other[3])

@@ -236,14 +236,15 @@ NCU_TRAFFIC = {
 
 
 def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_tiles=(),
-                      dense_layers=()):
+                      dense_layers=(), fwd_whole_rows=()):
     """Bytes that must cross HBM per ROUND for each kernel class (weights streamed once per
     product, activations in and out), and their total.  fwd_run_tiles[l-1], layers l = 1..m: in
     steps 1..K-1 the weight-gradient launch of layer l also forms the next step's forward product
     of that layer: its bf16 weights are not read by a forward kernel in steps 2..K (layer 1's copy
     is not even written); the layer's next input is read and its next activations are written by
     the weight-gradient launch, which also writes and reads back one fp32 partial sum [128, B]
-    per learner, row tile and run of fwd_run_tiles[l-1] column tiles; the flops move with them.
+    per learner, row tile and run of fwd_run_tiles[l-1] column tiles (not for the fwd_whole_rows[l-1]
+    (learner, row tile) pairs that are taken as one run); the flops move with them.
     dense_layers: hidden layers whose first-step forward is one dense product over all learners'
     batch rows, reading the (shared) weights once instead of once per learner."""
     dims, P, K, B = cfg["dims"], cfg["P"], cfg["K"], cfg["B"]
@@ -257,7 +258,8 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_
     for i, run in enumerate(fwd_run_tiles if K > 1 else ()):
         n_tiles = -(-dims[i] // 32)
         runs = -(-n_tiles // run)
-        partial = P * -(-dims[i + 1] // 128) * runs * B * 128 * 4 if runs > 1 else 0
+        split_rows = P * -(-dims[i + 1] // 128) - (fwd_whole_rows[i] if i < len(fwd_whole_rows) else 0)
+        partial = split_rows * runs * B * 128 * 4 if runs > 1 else 0
         moved = 2 * rows * dims[i] + 4 * rows * dims[i + 1]     # the layer's input read, A_l written twice
         fwd_delta -= (K - 1) * (2 * P * nW[i] + moved)
         wgrad_delta += (K - 1) * (moved + 2 * partial - (2 * P * nW[0] if i == 0 else 0))
@@ -285,9 +287,10 @@ def algorithmic_bytes(cfg, tensor_path, deferred=False, momentum=False, fwd_run_
 
 
 def kernel_rooflines(cfg, prof, steps, peaks, tensor_path, deferred=False, momentum=False,
-                     fwd_run_tiles=(), dense_layers=()):
+                     fwd_run_tiles=(), dense_layers=(), fwd_whole_rows=()):
     """Per kernel class: algorithmic bytes or flops of all its launches / its summed device time."""
-    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles, dense_layers)
+    per_round = algorithmic_bytes(cfg, tensor_path, deferred, momentum, fwd_run_tiles, dense_layers,
+                                  fwd_whole_rows)
     out = {}
     for name, (ms, cnt) in prof.items():
         if cnt == 0 or ms <= 0:
@@ -520,9 +523,10 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
     plan = g.get_step_plan()
     fwd_run_tiles = tuple(plan["fwd_run_tiles"]) if args.schedule == 0 else ()
     dense_layers = tuple(plan["dense_first_step"]) if args.schedule == 0 else ()
+    fwd_whole_rows = tuple(plan["fwd_whole_rows"]) if args.schedule == 0 else ()
     kern = kernel_rooflines(cfg, prof, psteps, peaks, mode == 1, deferred=not args.no_defer,
                             momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles,
-                            dense_layers=dense_layers)
+                            dense_layers=dense_layers, fwd_whole_rows=fwd_whole_rows)
     n = g.n
     g.close()
     del g, flush
@@ -556,12 +560,12 @@ def measure_mlp(name, args, m, torch, dist, peaks, world, rank, local, steps, wi
     # the whole round against the HBM roofline: every class's algorithmic bytes / the round's time
     per_round = algorithmic_bytes(cfg, mode == 1, deferred=not args.no_defer,
                                   momentum=args.beta != 0.0, fwd_run_tiles=fwd_run_tiles,
-                                  dense_layers=dense_layers)
+                                  dense_layers=dense_layers, fwd_whole_rows=fwd_whole_rows)
     round_bytes = sum(v["bytes"] for v in per_round.values())
     ms_round = total_ms / steps
     return dict(
         cfg=cfg, n=n, units=units, fwd_run_tiles=fwd_run_tiles, dense_layers=dense_layers,
-        total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
+        fwd_whole_rows=fwd_whole_rows, total_ms=total_ms, e2e_ms=e2e_ms, launches=launches,
         clocks=clocks, cpu=cpu, kern=kern, roof=roof, t_wall=t_wall, mode=mode,
         meta_in_round={"ms": statistics.median(meta_ms),
                        "gbs": per_round["meta_update"]["bytes"] / statistics.median(meta_ms) / 1e6},
@@ -628,7 +632,8 @@ def run_mavg(args):
                                     2: "CUDA graph of per-product launches, plain tensor-core tiles"}[args.schedule],
                        "forward_products": (f"layers 1..{len(r['fwd_run_tiles'])} inside their weight-gradient "
                                             "launch of the step before (steps 2..K; partial sums per "
-                                            f"{list(r['fwd_run_tiles'])} column tiles)"
+                                            f"{list(r['fwd_run_tiles'])} column tiles, after {list(r['fwd_whole_rows'])} "
+                                            "(learner, row tile) pairs taken whole)"
                                             if r["fwd_run_tiles"] else "launches of their own"),
                        "first_step_forward": (f"layers {list(r['dense_layers'])}: one dense product over the "
                                               "batch rows of all learners" if r["dense_layers"]

@@ -220,7 +220,11 @@ typedef enum {
                                    forward product of hidden layer l at the first step of a round
                                    (all learners hold w~) is one dense product over the batch rows
                                    of all learners, the weights read once */
-  MAVG_PLAN_COUNT = 4 + MAVG_MAX_LAYERS
+  MAVG_PLAN_FWD_WHOLE_ROWS = 4 + MAVG_MAX_LAYERS, /* first of MAVG_MAX_LAYERS entries: for layer
+                                   l <= m, how many of its P x ceil(out / 128) (learner, row tile)
+                                   pairs are taken as one run over all column tiles (no partial
+                                   sums); the others are cut into runs of FWD_RUN_TILES tiles */
+  MAVG_PLAN_COUNT = 4 + 2 * MAVG_MAX_LAYERS
 } mavg_plan_entry;
 mavg_status mavg_get_step_plan(mavg_handle h, int32_t *out);
 

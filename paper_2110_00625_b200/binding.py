@@ -270,12 +270,14 @@ class Mavg:
     def get_step_plan(self):
         """How a local step is laid out in launches: tensor_path, wgrad_merged, fwd_with_wgrad
         (layers 1..m whose next-step forward product rides on their weight-gradient launch) and
-        fwd_run_tiles (per such layer, column tiles per partial sum), dense_first_step (hidden
+        fwd_run_tiles (per such layer, column tiles per partial sum), fwd_whole_rows (per such
+        layer, the (learner, row tile) pairs taken as one run, without partial sums), dense_first_step (hidden
         layers whose first-step forward is one dense product over all learners' batch rows)."""
-        out = (C.c_int32 * (4 + MAX_LAYERS))()
+        out = (C.c_int32 * (4 + 2 * MAX_LAYERS))()
         self._check(self.lib.mavg_get_step_plan(self.handle, out))
         return {"tensor_path": out[0], "wgrad_merged": out[1], "fwd_with_wgrad": out[2],
                 "fwd_run_tiles": list(out[3:3 + out[2]]),
+                "fwd_whole_rows": list(out[4 + MAX_LAYERS:4 + MAX_LAYERS + out[2]]),
                 "dense_first_step": [l + 1 for l in range(MAX_LAYERS) if out[3 + MAX_LAYERS] >> l & 1]}
 
     def set_profiling(self, on):

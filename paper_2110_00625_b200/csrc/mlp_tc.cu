@@ -620,7 +620,10 @@ void tc_step_plan(mavg_ctx* c, int32_t* out) {
   out[MAVG_PLAN_TENSOR_PATH] = 1;
   out[MAVG_PLAN_WGRAD_MERGED] = st->wgrad_merged ? 1 : 0;
   out[MAVG_PLAN_FWD_WITH_WGRAD] = st->fuse_upto;
-  for (int l = 1; l <= st->fuse_upto; ++l) out[MAVG_PLAN_FWD_RUN_TILES + l - 1] = st->wgrad_f[l].chunk;
+  for (int l = 1; l <= st->fuse_upto; ++l) {
+    out[MAVG_PLAN_FWD_RUN_TILES + l - 1] = st->wgrad_f[l].chunk;
+    out[MAVG_PLAN_FWD_WHOLE_ROWS + l - 1] = st->wgrad_f[l].whole_rows;
+  }
   for (int l = 1; l <= MAVG_MAX_LAYERS; ++l)
     if (st->dense[l].ok) out[MAVG_PLAN_DENSE_FIRST_STEP] |= 1 << (l - 1);
 }

@@ -151,10 +151,6 @@ constexpr long kWgradChunkCap = MAVG_WGRAD_CHUNK_CAP;
 #define MAVG_WGRAD_STREAM_SLOTS 4
 #endif
 constexpr long kWgradStreamChunk = MAVG_WGRAD_STREAM_CHUNK;
-#ifndef MAVG_WGRAD_FWD_CHUNK
-#define MAVG_WGRAD_FWD_CHUNK 64
-#endif
-constexpr long kWgradFwdChunk = MAVG_WGRAD_FWD_CHUNK;
 #ifndef MAVG_WGRAD_FWD_SLOTS
 #define MAVG_WGRAD_FWD_SLOTS 6
 #endif
@@ -173,33 +169,42 @@ WgradPlan plan_wgrad_stream(int out, int in, int B, int P, int sm_count, bool mo
   if (chunk < 1) chunk = 1;
   if (chunk > kWgradChunkCap) chunk = kWgradChunkCap;
   if (streaming && chunk > kWgradStreamChunk) chunk = kWgradStreamChunk;
-  // With the next step's forward product riding along, every work item ends with a 128 x B fp32
-  // partial sum going to global memory (and coming back once): long runs keep that traffic small
-  // against the 2 x 2 bytes per weight the fusion saves.
-  // Among the even splits of a row of column tiles, take the one whose busiest block finishes
-  // first: ceil(items / blocks) items of (run + per-item work) each.  The per-item work -- the
-  // next dZ^T tile, reading the forward accumulator, the partial sum and its share of the sums
-  // over all runs of a row, during which the next item's forward products wait -- is worth about
-  // six tile periods (measured with 8 learners: runs of 8 tiles took 150 us per launch where runs
-  // of 32 to 48 take 75 us).
+  // With a riding forward product every run ends with per-run work -- reading the forward
+  // accumulator, the partial sum and its share of the sums over all runs of a row, during which
+  // the next run's forward products wait -- worth about eight tile periods (measured with 8
+  // learners: runs of 8 tiles took 150 us per launch where runs of 32 to 48 take 75 us).  So: as
+  // many whole waves of whole rows as pay (one item per (learner, row tile), no partial sums at
+  // all), then the remaining rows cut evenly into runs of at least 16 tiles; taken is the
+  // combination whose busiest block finishes first.
+  long whole_rows = 0;
   if (fwd_next) {
-    long best_cost = 0;
-    for (int nc = 1; nc <= w.n_tiles; ++nc) {
-      const long run = (w.n_tiles + nc - 1) / nc;
-      if (run > kWgradFwdChunk) continue;
-      if (run < 16 && best_cost) break;
-      const long items = (long)P * w.m_tiles * ((w.n_tiles + run - 1) / run);
-      const long cost = ((items + sm_count - 1) / sm_count) * (run + 6);
-      if (!best_cost || cost < best_cost) {
-        best_cost = cost;
-        chunk = run;
+    const long rows = (long)P * w.m_tiles, per_run = 8;
+    long best_cost = -1;
+    for (long waves = 0; waves * sm_count <= rows; ++waves) {
+      const long rest = rows - waves * sm_count;
+      const long head = waves * (w.n_tiles + per_run);
+      if (rest == 0) {
+        if (best_cost < 0 || head < best_cost) { best_cost = head; whole_rows = rows; chunk = w.n_tiles; }
+        break;
+      }
+      for (int nc = 1; nc <= w.n_tiles; ++nc) {
+        const long run = (w.n_tiles + nc - 1) / nc;
+        if (run < 16 && nc > 1) break;
+        const long items = rest * ((w.n_tiles + run - 1) / run);
+        const long cost = head + ((items + sm_count - 1) / sm_count) * (run + per_run);
+        if (best_cost < 0 || cost < best_cost) {
+          best_cost = cost;
+          whole_rows = waves * sm_count;
+          chunk = run;
+        }
       }
     }
   }
   if (chunk > w.n_tiles) chunk = w.n_tiles;
   w.chunk = (int)chunk;
   w.n_chunks = (w.n_tiles + w.chunk - 1) / w.chunk;
-  w.items = P * w.m_tiles * w.n_chunks;
+  w.whole_rows = (int)whole_rows;
+  w.items = w.whole_rows + (P * w.m_tiles - w.whole_rows) * w.n_chunks;
   const int a_bytes = w.nkb * kBM * kBK * 2;
   const int b_bytes = w.nkb * kBN * kBK * 2;
   w.w16_on_b = b_bytes >= kW16Bytes ? 1 : 0;   // the bf16 output tile reuses the A^T slabs' space
@@ -245,6 +250,7 @@ WgradArgs make_args(mavg_ctx* c, const WgradPlan& w, bool shared, const MomArgs&
   g.chunk = w.chunk;
   g.n_chunks = w.n_chunks;
   g.items = w.items;
+  g.whole_rows = w.whole_rows;
   g.slots = w.slots;
   g.a_bufs = w.a_bufs;
   g.w16_on_b = w.w16_on_b;

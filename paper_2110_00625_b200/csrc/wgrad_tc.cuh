@@ -8,6 +8,8 @@ namespace mavg {
 
 struct WgradPlan {
   int nkb, m_tiles, n_tiles, chunk, n_chunks, items, slots, a_bufs, grid, w16_on_b;
+  int whole_rows; // (learner, row tile) pairs taken as one run of all column tiles (plans made with
+                  // fwd_next: whole waves of such items first, the remaining rows cut into runs)
   int xn_bytes;   // room in every slot for the next step's input tile (plans made with fwd_next)
   size_t smem;
 };

@@ -52,7 +52,11 @@ struct WgradArgs {
   int m_tiles, n_tiles;    // 128-row tiles of out, 32-column tiles of in
   int chunk;               // column tiles per work item
   int n_chunks;            // ceil(n_tiles / chunk)
-  int items;               // P * m_tiles * n_chunks
+  int items;               // whole_rows + (P * m_tiles - whole_rows) * n_chunks
+  int whole_rows;          // the first whole_rows (learner, row tile) pairs are one work item each:
+                           // all n_tiles column tiles in one run; the others are cut into
+                           // n_chunks runs of chunk tiles (0 everywhere but in plans that balance
+                           // a riding forward product's long runs over the blocks)
   int slots;               // ring depth
   int a_bufs;              // 1 or 2 buffers for the dZ^T tile
   int w16_on_b;            // 1: the bf16 output tile is written over the slot's A^T slabs
@@ -124,8 +128,8 @@ __device__ __forceinline__ void wgrad_init_barriers(WgradShared& sh, int slots) 
 __device__ __forceinline__ void wgrad_run_totals(const WgradArgs& g, int vblock, int vgrid,
                                                  uint32_t& tiles, uint32_t& items) {
   for (int item = vblock; item < g.items; item += vgrid) {
-    const int nt0 = (item % g.n_chunks) * g.chunk;
-    tiles += (uint32_t)min(g.chunk, g.n_tiles - nt0);
+    const int nt0 = ((item - g.whole_rows) % g.n_chunks) * g.chunk;
+    tiles += (uint32_t)(item < g.whole_rows ? g.n_tiles : min(g.chunk, g.n_tiles - nt0));
     items += 1;
   }
 }
@@ -164,13 +168,20 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
 
   // work item -> (learner p, row tile, first column tile, number of column tiles)
   auto decode = [&](int item, int& p, int& m0, int& nt0, int& nt) {
-    const int nc = item % g.n_chunks;
-    const int rest = item / g.n_chunks;
-    const int mt = rest % g.m_tiles;
-    p = rest / g.m_tiles;
+    int row;                       // (learner, row tile) pair
+    if (item < g.whole_rows) {
+      row = item;
+      nt0 = 0;
+      nt = g.n_tiles;
+    } else {
+      const int idx = item - g.whole_rows;
+      row = g.whole_rows + idx / g.n_chunks;
+      nt0 = (idx % g.n_chunks) * g.chunk;
+      nt = min(g.chunk, g.n_tiles - nt0);
+    }
+    const int mt = row % g.m_tiles;
+    p = row / g.m_tiles;
     m0 = mt * kBM;
-    nt0 = nc * g.chunk;
-    nt = min(g.chunk, g.n_tiles - nt0);
   };
 
   if (warp == 0) {
@@ -416,12 +427,13 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
     // reads TMEM lanes 32 (w % 4) ...), 32 batch columns at a time.
     const int q = warp & 3;
     const int r = q * 32 + lane;
-    const bool single = g.n_chunks == 1;
     const size_t tile_floats = (size_t)g.batch * kBM;
     uint32_t item_ctr = item_base;
+    uint32_t split_ctr = 0;          // items so far that went through z_part / z_flag
     for (int item = vblock; item < g.items; item += vgrid, ++item_ctr) {
       int p, m0, nt0, nt;
       decode(item, p, m0, nt0, nt);
+      const bool single = nt == g.n_tiles;     // the accumulator is the whole product
       const int mt = m0 / kBM;
       const int m = m0 + r;
       const bool row_ok = m < g.out_rows;
@@ -482,7 +494,7 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.z_part);
       if (warp == 12 && lane == 0 &&
-          mbar_wait(&sh.z_part, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
+          mbar_wait(&sh.z_part, split_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) {
         int* cnt = g.zcount + (size_t)p * g.m_tiles + mt;
         int old;
         asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
@@ -492,7 +504,8 @@ __device__ __forceinline__ void wgrad_run(const CUtensorMap& tm_dzt, const CUten
         mbar_arrive(&sh.z_flag);
       }
       __syncwarp();
-      if (!mbar_wait(&sh.z_flag, item_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) break;
+      if (!mbar_wait(&sh.z_flag, split_ctr & 1, abortp, g.status, ERR_WG_EPILOGUE)) break;
+      ++split_ctr;
       if (!sh.z_last) continue;
       for (int c0 = 0; c0 < g.batch; c0 += 32) {
         float z[32];

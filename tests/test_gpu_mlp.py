@@ -323,8 +323,10 @@ def test_tc_mixed_call_sequences_keep_the_same_bits():
 # (13 x 8 x 96 > 64 per SM): every layer's weight gradient is a launch of its own, and the launches
 # of the hidden layers also form the NEXT step's forward product of their layer from the updated
 # tiles (steps 1..K-1): one hidden layer, and two (the second one's launch reads the activations
-# the first one's has just produced, and still writes its bf16 copy for the dgrad product).
-FUSED_SHAPES = [[3072, 1024, 10], [3072, 1024, 512, 10]]
+# the first one's has just produced, and still writes its bf16 copy for the dgrad product); and one
+# with more (learner, row tile) pairs than SMs (13 x 16 = 208), whose plan takes the first 148 pairs
+# as whole rows and cuts the other 60 into two runs each (both kinds of work item in one launch).
+FUSED_SHAPES = [[3072, 1024, 10], [3072, 1024, 512, 10], [3072, 2048, 10]]
 FUSED_P, FUSED_B = 13, 16
 
 
@@ -358,7 +360,11 @@ def test_forward_riding_on_the_weight_gradient_against_the_oracle(oracle, dims, 
     plan = g.get_step_plan()
     assert plan["tensor_path"] == 1 and plan["wgrad_merged"] == 0
     assert plan["fwd_with_wgrad"] == len(dims) - 2
-    assert all(8 <= r <= d // 32 for r, d in zip(plan["fwd_run_tiles"], dims))
+    assert all(16 <= r <= d // 32 for r, d in zip(plan["fwd_run_tiles"], dims))
+    rows = [FUSED_P * -(-d // 128) for d in dims[1:-1]]
+    assert all(0 <= wr <= n for wr, n in zip(plan["fwd_whole_rows"], rows))
+    if dims[1] == 2048:
+        assert 0 < plan["fwd_whole_rows"][0] < rows[0]
     xq = oracle.bf16_round(x)             # the GPU holds the dataset in bf16
     o = oracle.Mavg(w1, P=FUSED_P, K=3, gamma=cfg["gamma"], mu=cfg["mu"], B=FUSED_B,
                     seed=_mavg().workloads.BASE_SEED, objective=oracle.OBJ_MLP, dims=dims,

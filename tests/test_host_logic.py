@@ -102,7 +102,7 @@ def test_workspace_size_and_buffer_checks(lib):
     assert lib.mavg_set_wait_limit(None, 100) == 1
     assert lib.mavg_selftest_wait(None) == 1
     assert lib.mavg_set_schedule(None, 0) == 1
-    assert lib.mavg_get_step_plan(None, (C.c_int32 * 12)()) == 1
+    assert lib.mavg_get_step_plan(None, (C.c_int32 * 20)()) == 1
 
 
 def test_create_without_a_device_fails_cleanly(lib):

@@ -17,6 +17,20 @@
 // same slot (unless the momentum is reset at this step), updated in place (u <- beta u - gamma dW;
 // W <- W + u) and stored back, 18 bytes per weight instead of 10.
 // Edge tiles need no predicates: TMA zero-fills loads and clips stores at the tensor bounds.
+//
+// The 512-thread instantiation (FWD) lets the NEXT local step's forward product of the same layer
+// ride along: the epilogue has just put the updated bf16 tile W16[128, 32] into the slot, and the
+// producer has loaded the matching [B, 32] tile of the next step's input Xn beside it, so
+//   forward warp    one thread issues W16_tile . Xn_tile^T (M=128, N=B, K=32) into a third TMEM
+//                   accumulator that collects a whole run of column tiles; the slot is released
+//                   only after these MMAs have read it;
+//   4 more warps    read that accumulator once per run.  A run that covers its whole row adds the
+//                   bias, applies ReLU and writes the next step's activations (bf16, both
+//                   orientations) at once; the runs of a row that is cut leave fp32 partial sums
+//                   and bump the row's arrival counter, and the one that arrives last adds the
+//                   partial sums in ascending run order and finishes the row.
+// Per weight and step this removes the forward product's read of the bf16 copy and, for a layer
+// without a dgrad product (layer 1), the copy itself.
 #include <cuda.h>
 
 #include <algorithm>

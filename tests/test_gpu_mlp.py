@@ -461,3 +461,50 @@ def test_dense_first_step_forward_against_the_oracle(oracle):
     h.sync()
     assert np.abs(h.get_losses()[:, 0] - g.get_losses()[:, 0]).max() <= 1e-4 * losses_o[:, 0].max()
     g.close(); h.close()
+
+
+@pytest.mark.parametrize("dims,B", [([3072, 1024, 10], 48), ([3072, 1024, 10], 128),
+                                    ([3048, 1000, 10], 64)])
+def test_forward_riding_other_batch_sizes_and_ragged_edges(oracle, dims, B):
+    # B = 48: the forward accumulator's last 16 columns are read on their own (the batch is not a
+    # multiple of 32); B = 128: two 64-wide contraction slabs, the bf16 tile on top of the dead
+    # operand slabs, 256 columns of tensor memory.  Two local steps from identical replicas: the
+    # second step's hidden activations come out of the first step's weight-gradient launch.
+    # Against the plain-tiles schedule per tile (itself checked against the oracle at these batch
+    # sizes by the shape tests above), and for B = 48 against the oracle directly.
+    # 3048 x 1000: the last column tile has 8 of 32 columns and the last row tile 104 of 128 rows
+    # (zero-filled operand tiles, clipped stores, rows beyond the layer not written).
+    m = _mavg()
+    P, K = 13, 2
+    cfg = dict(m.workloads.CONFIGS["C2"])
+    cfg.update(dims=dims, P=P, K=K, B=B, S=4096)
+    x, y = m.workloads.make_dataset(cfg, S=cfg["S"])
+    w1 = m.workloads.mlp_init(dims)
+
+    def run(schedule):
+        g = m.Mavg(w1, P=P, K=K, local_lr=cfg["gamma"], mu=cfg["mu"], B=B,
+                   seed=m.workloads.BASE_SEED, objective=m.OBJ_MLP, dims=dims, gemm_bf16=1,
+                   x=x, y=y, x_bf16=True)
+        assert g.get_step_plan()["fwd_with_wgrad"] == 1
+        g.set_schedule(schedule)
+        g.local_steps()
+        g.sync()
+        out = g.replicas.cpu().numpy()[:, :g.n].astype(np.float64), g.get_losses(), g.stride
+        g.close()
+        return out
+
+    ra, la, stride = run(0)
+    rb, lb, _ = run(2)
+    assert np.abs(la - lb).max() <= 2e-3 * np.abs(lb).max()
+    for j in (0, P // 2, P - 1):
+        assert_tiles_close(ra[j] - w1, rb[j] - w1, dims, what=f"learner {j}, riding against plain")
+    if B != 128:
+        o = oracle.Mavg(w1, P=P, K=K, gamma=cfg["gamma"], mu=cfg["mu"], B=B,
+                        seed=m.workloads.BASE_SEED, objective=oracle.OBJ_MLP, dims=dims, bf16=True,
+                        x=oracle.bf16_round(x), y=y, stride=stride)
+        losses_o, _ = o.local_steps()
+        assert np.abs(la - losses_o).max() <= 2e-2 * losses_o.max()
+        for j in (0, P - 1):
+            step_o = o.replicas[j, :len(w1)].astype(np.float64) - w1
+            assert l2_rel(ra[j] - w1, step_o) <= 3e-2, j
+            assert_tiles_close(ra[j] - w1, step_o, dims, what=f"learner {j}")
